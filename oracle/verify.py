@@ -1,0 +1,142 @@
+"""Relaxed acceptance of one draft tree (oracle; test infrastructure).
+
+Follows Sec. 4 (multiplicative bound, relaxed accept probability), App. A.2
+Eq. 1-2 (accept test, residual resampling) and Sec. 2.1 (tree verification).
+p = drafter, q = target.  All arithmetic in double on the distributions that
+postprocess_row returns.
+
+Readings where the paper is silent:
+ * the neighbour list excludes the draft token x itself; x always belongs to A
+ * A is the longest prefix of the distance-ordered list for which the running
+   sum stays strictly below lambda * q(x)  (Sec. 4, display with "<")
+ * siblings are tested one after another in stored order; after a rejection
+   the mass of A is moved onto x (q~), the target becomes the normalised
+   positive part of q~ - p (Eq. 2), and the drafter is renormalised without x
+ * the token drawn when no child is accepted (or at a leaf) uses inverse-CDF
+   sampling in token-id order
+"""
+
+import numpy as np
+
+from .postprocess import postprocess_row
+from .tree import tree_children
+
+
+def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes):
+    """Sec. 4: m = sum of q over A_{k,lambda}(x) and the members of A besides x."""
+    cum = q_cur[x]
+    bound = lam * q_cur[x]
+    members = []
+    code = x - code_offset
+    if 0 <= code < n_codes:
+        for r in range(k):
+            a = code_offset + int(nbr_idx[code][r])
+            if cum + q_cur[a] < bound:
+                cum = cum + q_cur[a]
+                members.append(a)
+            else:
+                break
+    return cum, members
+
+
+def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
+                code_offset, n_codes):
+    """Process one tree node.
+
+    q: target distribution of the node; p: drafter distribution (None at a leaf)
+    child_ids: its children in stored order; tokens[c]: draft token of node c
+    (a negative token means "no draft" and is skipped).
+    Returns (next_child or -1, sampled token or -1, {child: (m, thr)}).
+    """
+    q_cur = np.array(q, dtype=np.float64)
+    p_cur = None if p is None else np.array(p, dtype=np.float64)
+    tested = {}
+    for c in child_ids:
+        x = int(tokens[c])
+        if x < 0:
+            continue
+        m, members = relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes)
+        if p_cur[x] > 0:
+            thr = min(1.0, m / p_cur[x])          # Sec. 4, final accept probability
+        else:
+            thr = 1.0 if m > 0 else 0.0
+        tested[c] = (m, thr)
+        if float(u_accept[c]) < thr:
+            return c, -1, tested
+        q_t = q_cur.copy()                         # q~: mass of A moved onto x
+        q_t[x] = m
+        for a in members:
+            q_t[a] = 0.0
+        r = np.maximum(q_t - p_cur, 0.0)           # Eq. 2
+        Z = r.sum()
+        q_cur = r / Z if Z > 0 else q_t
+        w = 1.0 - p_cur[x]
+        p_cur[x] = 0.0
+        if w > 0:
+            p_cur = p_cur / w
+    cdf = np.cumsum(q_cur)
+    target = float(u_resample) * cdf[-1]
+    j = int(np.argmax(cdf > target))
+    return -1, j, tested
+
+
+def walk(node_next, node_token, tokens):
+    """Sec. 2.1 / App. A.2: follow accepted children from the root; the accepted
+    draft tokens are kept, then one token drawn at the node where the walk
+    stops.  Returns (accept_len, out_tokens, out_nodes); the lists have
+    accept_len + 1 entries."""
+    cur = 0
+    out_tokens, out_nodes = [], []
+    while node_next[cur] >= 0:
+        cur = int(node_next[cur])
+        out_tokens.append(int(tokens[cur]))
+        out_nodes.append(cur)
+    out_tokens.append(int(node_token[cur]))
+    out_nodes.append(cur)
+    return len(out_tokens) - 1, out_tokens, out_nodes
+
+
+def verify_sequence(parent, target_cond, target_uncond, draft_cond, draft_uncond, tokens,
+                    u_accept, u_resample, nbr_idx, *, cfg_scale=1.0, temperature=1.0,
+                    top_k_target=0, top_k_draft=0, lam=1.0, k=0, code_offset=0, n_codes=0,
+                    allowed_begin=0, allowed_end=None):
+    """Verify one sequence's tree.  Logit arrays are [N][V]; uncond may be None.
+
+    Returns a dict with node_next, node_token (int arrays [N]), node_mass,
+    node_thresh (double [N], -1 where a node was not tested), accept_len,
+    out_tokens, out_nodes.
+    """
+    children = tree_children(parent)
+    N = len(parent)
+    node_next = np.full(N, -1, dtype=np.int64)
+    node_token = np.full(N, -1, dtype=np.int64)
+    node_mass = np.full(N, -1.0)
+    node_thresh = np.full(N, -1.0)
+    for n in range(N):
+        q, _ = postprocess_row(target_cond[n], None if target_uncond is None else target_uncond[n],
+                               cfg_scale, temperature, top_k_target, allowed_begin, allowed_end)
+        p = None
+        if children[n]:
+            p, _ = postprocess_row(draft_cond[n], None if draft_uncond is None else draft_uncond[n],
+                                   cfg_scale, temperature, top_k_draft, allowed_begin, allowed_end)
+        nxt, tok, tested = verify_node(q, p, children[n], tokens, u_accept, u_resample[n],
+                                       nbr_idx, k, lam, code_offset, n_codes)
+        node_next[n], node_token[n] = nxt, tok
+        for c, (m, thr) in tested.items():
+            node_mass[c], node_thresh[c] = m, thr
+    accept_len, out_tokens, out_nodes = walk(node_next, node_token, tokens)
+    return dict(node_next=node_next, node_token=node_token, node_mass=node_mass,
+                node_thresh=node_thresh, accept_len=accept_len, out_tokens=out_tokens,
+                out_nodes=out_nodes)
+
+
+def verify_batch(parent, target_cond, target_uncond, draft_cond, draft_uncond, tokens,
+                 u_accept, u_resample, nbr_idx, **params):
+    """verify_sequence over the leading batch dimension; returns a list of dicts."""
+    out = []
+    for b in range(len(tokens)):
+        out.append(verify_sequence(
+            parent, target_cond[b], None if target_uncond is None else target_uncond[b],
+            draft_cond[b], None if draft_uncond is None else draft_uncond[b],
+            tokens[b], u_accept[b], u_resample[b], nbr_idx, **params))
+    return out
