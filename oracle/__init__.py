@@ -16,6 +16,6 @@ its tables needs trained models and captions that are not available.
 from .postprocess import fma_f32, combine_f32, postprocess_row  # noqa: F401
 from .neighbors import neighbor_table, neighbor_row  # noqa: F401
 from .tree import tree_children  # noqa: F401
-from .verify import relaxed_mass, verify_node, verify_sequence, walk, verify_batch  # noqa: F401
+from .verify import relaxed_mass, moved_mass, sibling_loop, inverse_cdf, verify_node, verify_sequence, walk, verify_batch  # noqa: F401
 from .sampler import sample_children, sample_draft_tree  # noqa: F401
 from .philox import philox4x32_10, uniform_open, uniform_halfopen, stream_uniforms  # noqa: F401

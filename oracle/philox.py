@@ -42,8 +42,8 @@ def philox4x32_10(counter, key):
 
 
 def uniform_open(x):
-    """32 random bits -> float32 in (0,1): ((x >> 8) + 0.5) * 2^-24."""
-    return ((np.asarray(x, dtype=np.uint32) >> 8).astype(np.float64) + 0.5) * 2.0 ** -24
+    """32 random bits -> float32 in (0,1): ((x >> 9) + 0.5) * 2^-23 (exact in float32)."""
+    return ((np.asarray(x, dtype=np.uint32) >> 9).astype(np.float64) + 0.5) * 2.0 ** -23
 
 
 def uniform_halfopen(x):

@@ -39,15 +39,20 @@ def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes):
     return cum, members
 
 
-def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
-                code_offset, n_codes):
-    """Process one tree node.
+def moved_mass(q_cur, x, m, members):
+    """q~: the target distribution with the mass of A concentrated on x."""
+    q_t = np.array(q_cur, dtype=np.float64)
+    q_t[x] = m
+    for a in members:
+        q_t[a] = 0.0
+    return q_t
 
-    q: target distribution of the node; p: drafter distribution (None at a leaf)
-    child_ids: its children in stored order; tokens[c]: draft token of node c
-    (a negative token means "no draft" and is skipped).
-    Returns (next_child or -1, sampled token or -1, {child: (m, thr)}).
-    """
+
+def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset, n_codes):
+    """Test the children of one node in stored order (Sec. 4; App. A.2 Eq. 1-2).
+
+    Returns (accepted child or -1, q_cur, {child: (m, thr)}): q_cur is the
+    target distribution left after the rejections (q itself at a leaf)."""
     q_cur = np.array(q, dtype=np.float64)
     p_cur = None if p is None else np.array(p, dtype=np.float64)
     tested = {}
@@ -62,11 +67,8 @@ def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
             thr = 1.0 if m > 0 else 0.0
         tested[c] = (m, thr)
         if float(u_accept[c]) < thr:
-            return c, -1, tested
-        q_t = q_cur.copy()                         # q~: mass of A moved onto x
-        q_t[x] = m
-        for a in members:
-            q_t[a] = 0.0
+            return c, q_cur, tested
+        q_t = moved_mass(q_cur, x, m, members)
         r = np.maximum(q_t - p_cur, 0.0)           # Eq. 2
         Z = r.sum()
         q_cur = r / Z if Z > 0 else q_t
@@ -74,10 +76,29 @@ def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
         p_cur[x] = 0.0
         if w > 0:
             p_cur = p_cur / w
-    cdf = np.cumsum(q_cur)
-    target = float(u_resample) * cdf[-1]
-    j = int(np.argmax(cdf > target))
-    return -1, j, tested
+    return -1, q_cur, tested
+
+
+def inverse_cdf(dist, u):
+    """Smallest token j whose cumulative mass exceeds u * total."""
+    cdf = np.cumsum(dist)
+    return int(np.argmax(cdf > float(u) * cdf[-1]))
+
+
+def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
+                code_offset, n_codes):
+    """Process one tree node.
+
+    q: target distribution of the node; p: drafter distribution (None at a leaf)
+    child_ids: its children in stored order; tokens[c]: draft token of node c
+    (a negative token means "no draft" and is skipped).
+    Returns (next_child or -1, sampled token or -1, {child: (m, thr)}).
+    """
+    nxt, q_cur, tested = sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam,
+                                      code_offset, n_codes)
+    if nxt >= 0:
+        return nxt, -1, tested
+    return -1, inverse_cdf(q_cur, u_resample), tested
 
 
 def walk(node_next, node_token, tokens):

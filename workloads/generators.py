@@ -64,10 +64,10 @@ def make_uniforms(B, N, seed, device="cpu"):
 
 
 def make_gumbel_uniforms(B, N, V, seed, device="cpu"):
-    """[B][N][V] float32 uniforms in (0,1) on the grid (i + 0.5) * 2^-24."""
+    """[B][N][V] float32 uniforms in (0,1) on the grid (i + 0.5) * 2^-23 (exact in float32)."""
     g = _gen(seed, device)
-    i = torch.randint(0, 1 << 24, (B, N, V), generator=g, device=device).to(torch.float32)
-    return (i + 0.5) * (2.0 ** -24)
+    i = torch.randint(0, 1 << 23, (B, N, V), generator=g, device=device).to(torch.float32)
+    return (i + 0.5) * (2.0 ** -23)
 
 
 def random_sibling_tokens(parent, B, lo, hi, seed, device="cpu"):
