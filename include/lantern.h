@@ -1,0 +1,177 @@
+/*
+ * lantern.h -- C ABI of the relaxed tree-verification hot path (LANTERN++).
+ *
+ * Notation follows the paper (Sec. 2 "Notations"): p is the DRAFTER
+ * distribution, q is the TARGET distribution; a draft token x is accepted with
+ * probability min(1, sum_{a in A(x)} q(a) / p(x)).
+ *
+ * Conventions for every entry point
+ *  - Pointers are DEVICE pointers owned by the caller unless marked "host".
+ *  - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *    default stream).  Nothing synchronises; outputs are valid once the stream
+ *    has reached the end of the call.  Outputs are fully overwritten.
+ *  - Errors come back as a lantern_status.  Invalid arguments are detected on the
+ *    host before anything is launched.  Problems that only the device can see
+ *    (a table index out of range, a copy that did not complete in time) are
+ *    OR-ed into *device_status as LANTERN_DEV_* bits; the kernels never trap.
+ *  - Same inputs and same uniforms / seed give the same bytes.
+ *  - Only lantern_tree_create allocates (a few hundred bytes per tree).
+ */
+#ifndef LANTERN_H_
+#define LANTERN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LANTERN_OK = 0,
+  LANTERN_ERR_INVALID_ARG = 1,  /* NULL required pointer, bad range, misaligned rows, bad tree  */
+  LANTERN_ERR_UNSUPPORTED = 2,  /* size beyond what the kernels are built for                   */
+  LANTERN_ERR_WORKSPACE = 3,    /* workspace missing or smaller than *_workspace() reports      */
+  LANTERN_ERR_CUDA = 4          /* a CUDA runtime call failed (launch, copy, allocation)        */
+} lantern_status;
+
+typedef enum { LANTERN_F32 = 0, LANTERN_BF16 = 1 } lantern_dtype;
+
+/* bits of *device_status */
+enum {
+  LANTERN_DEV_BAD_INDEX = 1,    /* a token or neighbour index fell outside the vocabulary; it was
+                                   treated as probability 0                                     */
+  LANTERN_DEV_TIMEOUT = 2,      /* a bounded on-chip wait expired; the data was re-read with
+                                   plain loads                                                  */
+  LANTERN_DEV_EMPTY_ROW = 4     /* a row had no finite logit                                    */
+};
+
+const char* lantern_status_string(lantern_status s);
+
+/* ---- static draft tree (Sec. 2.1 "Tree Drafting and Verification") -------------------------
+ * Node 0 stands for the last committed token; every other node carries one draft token.
+ * Nodes are numbered breadth first: parent[0] = -1, 0 <= parent[i] < i, parent[] non-decreasing,
+ * so the children of a node are contiguous and stored in the order they were drawn (rank order).
+ * At most LANTERN_MAX_CHILDREN children per node, at most LANTERN_MAX_NODES nodes.
+ * `parent` is a HOST array; it is copied, the caller keeps ownership. */
+#define LANTERN_MAX_CHILDREN 8
+#define LANTERN_MAX_NODES 1024
+typedef struct lantern_tree lantern_tree;
+lantern_status lantern_tree_create(const int32_t* parent /* host [n_nodes] */, int32_t n_nodes,
+                                   lantern_tree** out);
+lantern_status lantern_tree_destroy(lantern_tree* tree);
+int32_t lantern_tree_max_depth(const lantern_tree* tree);  /* depth of the deepest node */
+
+/* ---- parameters (App. B "Models": guidance, temperature, top-k; Sec. 4: k, lambda) ---------
+ * Row post-processing, identical for target rows (-> q) and drafter rows (-> p):
+ *   z_j = fma(cfg_scale, cond_j - uncond_j, uncond_j) * (1/temperature)      (float32 ops)
+ *   z_j = cond_j * (1/temperature)                         when the uncond pointer is NULL
+ *   tokens outside [allowed_begin, allowed_end) get -inf
+ *   top_k > 0: every z_j below the top_k-th largest value becomes -inf (ties at it are kept)
+ *   distribution = softmax(z)                                                                  */
+typedef struct {
+  float cfg_scale;
+  float temperature;       /* > 0 */
+  int32_t top_k_target;    /* 0 = off */
+  int32_t top_k_draft;     /* 0 = off */
+  float lambda;            /* multiplicative bound of Sec. 4, >= 1; 1 = no relaxation */
+  int32_t k;               /* neighbours considered per draft token, 0..k_table; 0 = standard
+                              speculative sampling                                              */
+  int32_t vocab;           /* V, logits per row */
+  int32_t code_offset;     /* token t has latent code t - code_offset ...                       */
+  int32_t n_codes;         /* ... iff 0 <= t - code_offset < n_codes (the table's row count L)  */
+  int32_t allowed_begin;   /* tokens outside [allowed_begin, allowed_end) are masked            */
+  int32_t allowed_end;     /* 0 means V                                                         */
+  uint64_t seed;           /* Philox-4x32-10 key; used only where uniforms are not supplied     */
+  uint64_t step;           /* counter base, < 2^62: change it every decode step                 */
+} lantern_params;
+
+/* ---- (1) latent-neighbour table -------------------------------------------------------------
+ * Sec. 2.2 / Sec. 4: B_k(x) = the k nearest neighbours of codebook vector c_x (App. A.1:
+ * C = {c_1..c_L}, c_i in R^d).  Metric: squared Euclidean distance on the raw rows.  For every
+ * row i the k rows j != i with the smallest (distance, j), ascending; exact (distances are
+ * evaluated in double precision before ranking), so duplicate rows tie by index.
+ *   codebook  [L][d] row-major, dt = F32 or BF16            nbr_idx  [L][k] int32
+ *   nbr_dist  [L][k] float32 squared distances, or NULL
+ *   workspace device scratch of at least lantern_build_neighbors_workspace() bytes, 256-B aligned
+ * Requires 1 <= k <= min(L-1, 1024), 1 <= d <= 4096.                                            */
+size_t lantern_build_neighbors_workspace(lantern_dtype dt, int32_t L, int32_t d, int32_t k);
+lantern_status lantern_build_neighbors(const void* codebook, lantern_dtype dt, int32_t L, int32_t d,
+                                       int32_t k, int32_t* nbr_idx, float* nbr_dist,
+                                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- (3) stochastic static-tree drafting ----------------------------------------------------
+ * Sec. 2.1: at a node with s children the drafter samples s tokens from p(. | path).  Drawn
+ * without replacement by Gumbel-top-s: key_j = log p_j - log(-log U_j); the s largest keys in
+ * descending order (ties: lower token id) become the children's tokens, in stored order.
+ * Expands the parents with node id in [parent_begin, parent_end) (one tree level, or 0..N for the
+ * whole tree when all drafter rows are known).
+ *   draft_cond / draft_uncond  [B][N][V] logits, row n = drafter output at node n; uncond NULL =
+ *                              no guidance.  Element (b, n, j) at  b*seq_stride + n*row_stride + j
+ *                              (strides in elements; rows must start 16-byte aligned).
+ *   gumbel_uniforms            [B][N][V] float32 in (0,1) indexed like the rows (contiguous), or
+ *                              NULL: Philox stream 0, U = ((x >> 9) + 0.5) * 2^-23
+ *   tokens                     [B][N] int32, entries of the expanded parents' children are
+ *                              written (-1 where fewer than s tokens have positive probability)
+ *   draft_prob                 [B][N] float32 p(token) under the parent's row, or NULL           */
+lantern_status lantern_sample_draft_tree(const lantern_params* params, const lantern_tree* tree,
+                                         const void* draft_cond, const void* draft_uncond,
+                                         lantern_dtype dt, int64_t row_stride, int64_t seq_stride,
+                                         int32_t batch, int32_t parent_begin, int32_t parent_end,
+                                         const float* gumbel_uniforms, int32_t* tokens,
+                                         float* draft_prob, int32_t* device_status, void* stream);
+
+/* ---- (2) relaxed verification of the tree ---------------------------------------------------
+ * Sec. 4 and App. A.2 (Eq. 1-2), per node n with children c_1..c_s in stored order:
+ *   q_cur = q(n), p_cur = p(n)
+ *   for each child c with token x:
+ *     A = {x} + longest prefix of x's neighbour list (first k entries of the table row) whose
+ *         running sum of q_cur, q_cur(x) included, stays < lambda * q_cur(x);   m = sum_A q_cur
+ *     accept c iff u_accept[c] < min(1, m / p_cur(x))
+ *     on rejection: move A's mass onto x, q_cur = normalise([q~ - p_cur]_+), drop x from p_cur
+ *   if no child was accepted (or n is a leaf): node_token[n] = inverse-CDF sample of q_cur with
+ *   u_resample[n], in token-id order.
+ * Then the walk (Sec. 2.1): from the root follow accepted children; out_tokens holds the accepted
+ * draft tokens followed by the token sampled where the walk stops.
+ *   nbr_idx        [n_codes][k_table] table of (1); may be NULL when params->k == 0
+ *   target_* / draft_*  [B][N][V] logits as in (3); draft rows of leaves are never read
+ *   tokens         [B][N] draft tokens (entry 0 unused; negative = no draft, skipped)
+ *   u_accept, u_resample  [B][N] float32 in [0,1), or NULL: Philox streams 1 / 2,
+ *                  u = (x >> 8) * 2^-24
+ *   accept_len     [B]            number of accepted draft tokens
+ *   out_tokens, out_nodes  [B][max_depth+1]; entries beyond accept_len+1 are set to -1
+ *   node_next, node_token  [B][N] or NULL (then they live in the workspace)
+ *   node_mass, node_thresh [B][N] float32 m and accept probability per tested child, -1 where
+ *                  a node was not tested; or NULL
+ *   device_status  one int32, OR-ed with LANTERN_DEV_* bits; or NULL
+ *   workspace      device scratch >= lantern_verify_tree_workspace() bytes (0 bytes needed when
+ *                  node_next and node_token are both given), 256-byte aligned                    */
+size_t lantern_verify_tree_workspace(const lantern_tree* tree, int32_t batch);
+lantern_status lantern_verify_tree(const lantern_params* params, const lantern_tree* tree,
+                                   const int32_t* nbr_idx, int32_t k_table,
+                                   const void* target_cond, const void* target_uncond,
+                                   const void* draft_cond, const void* draft_uncond,
+                                   lantern_dtype dt, int64_t row_stride, int64_t seq_stride,
+                                   int32_t batch, const int32_t* tokens,
+                                   const float* u_accept, const float* u_resample,
+                                   int32_t* accept_len, int32_t* out_tokens, int32_t* out_nodes,
+                                   int32_t* node_next, int32_t* node_token,
+                                   float* node_mass, float* node_thresh,
+                                   int32_t* device_status, void* workspace, size_t workspace_bytes,
+                                   void* stream);
+
+/* Raw Philox-4x32-10 words (Salmon et al., SC 2011) for counters (first + i, c1, c2, c3), i in
+ * [0, n): out[i][0..3].  Exists so that the generator can be checked against other
+ * implementations.  out is a device pointer to n*4 uint32.                                      */
+lantern_status lantern_philox_raw(uint64_t seed, uint32_t first, uint32_t c1, uint32_t c2,
+                                  uint32_t c3, int32_t n, uint32_t* out, void* stream);
+
+/* Tuning knob, process-wide: number of CTAs a logit row is split over (a thread-block cluster),
+ * 0 = choose automatically.  Returns the previous value.  Results do not depend on it beyond
+ * float32 summation order.                                                                      */
+int32_t lantern_set_cluster_size(int32_t ctas_per_row);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LANTERN_H_ */
