@@ -14,11 +14,12 @@ from .postprocess import postprocess_row
 from .tree import tree_children
 
 
-def sample_children(p, uniforms, s):
+def sample_children(p, uniforms, s, return_gaps=False):
     """Tokens of s children drawn from distribution p with uniforms U [V].
 
     Returns (tokens, probs): tokens by descending key (ties: lower id first);
-    -1 where fewer than s tokens have positive probability."""
+    -1 where fewer than s tokens have positive probability.  With return_gaps
+    also the key gap between rank r and rank r+1 for r < s (diagnostic)."""
     p = np.asarray(p, dtype=np.float64)
     U = np.asarray(uniforms, dtype=np.float64)
     support = np.nonzero(p > 0)[0]
@@ -29,6 +30,10 @@ def sample_children(p, uniforms, s):
     for r in range(min(s, len(order))):
         toks[r] = int(support[order[r]])
         probs[r] = float(p[toks[r]])
+    if return_gaps:
+        ks = key[order[: s + 1]]
+        gaps = [float(ks[r] - ks[r + 1]) if r + 1 < len(ks) else np.inf for r in range(s)]
+        return toks, probs, gaps
     return toks, probs
 
 

@@ -22,8 +22,11 @@ from .postprocess import postprocess_row
 from .tree import tree_children
 
 
-def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes):
-    """Sec. 4: m = sum of q over A_{k,lambda}(x) and the members of A besides x."""
+def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None):
+    """Sec. 4: m = sum of q over A_{k,lambda}(x) and the members of A besides x.
+
+    If `margins` is a list, |running sum - bound| of every comparison made is
+    appended to it (diagnostic for near-tie accounting; no effect on the result)."""
     cum = q_cur[x]
     bound = lam * q_cur[x]
     members = []
@@ -31,6 +34,8 @@ def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes):
     if 0 <= code < n_codes:
         for r in range(k):
             a = code_offset + int(nbr_idx[code][r])
+            if margins is not None:
+                margins.append(abs(cum + q_cur[a] - bound))
             if cum + q_cur[a] < bound:
                 cum = cum + q_cur[a]
                 members.append(a)
@@ -51,8 +56,9 @@ def moved_mass(q_cur, x, m, members):
 def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset, n_codes):
     """Test the children of one node in stored order (Sec. 4; App. A.2 Eq. 1-2).
 
-    Returns (accepted child or -1, q_cur, {child: (m, thr)}): q_cur is the
-    target distribution left after the rejections (q itself at a leaf)."""
+    Returns (accepted child or -1, q_cur, {child: (m, thr, cut_margin)}): q_cur
+    is the target distribution left after the rejections (q itself at a leaf);
+    cut_margin is the smallest |running sum - bound| met while forming A."""
     q_cur = np.array(q, dtype=np.float64)
     p_cur = None if p is None else np.array(p, dtype=np.float64)
     tested = {}
@@ -60,12 +66,13 @@ def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset
         x = int(tokens[c])
         if x < 0:
             continue
-        m, members = relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes)
+        margins = []
+        m, members = relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins)
         if p_cur[x] > 0:
             thr = min(1.0, m / p_cur[x])          # Sec. 4, final accept probability
         else:
             thr = 1.0 if m > 0 else 0.0
-        tested[c] = (m, thr)
+        tested[c] = (m, thr, min(margins) if margins else np.inf)
         if float(u_accept[c]) < thr:
             return c, q_cur, tested
         q_t = moved_mass(q_cur, x, m, members)
@@ -79,10 +86,15 @@ def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset
     return -1, q_cur, tested
 
 
-def inverse_cdf(dist, u):
-    """Smallest token j whose cumulative mass exceeds u * total."""
+def inverse_cdf(dist, u, return_margin=False):
+    """Smallest token j whose cumulative mass exceeds u * total.  With
+    return_margin also min_j |u * total - cdf_j| / total (diagnostic)."""
     cdf = np.cumsum(dist)
-    return int(np.argmax(cdf > float(u) * cdf[-1]))
+    target = float(u) * cdf[-1]
+    j = int(np.argmax(cdf > target))
+    if return_margin:
+        return j, float(np.abs(cdf - target).min() / cdf[-1])
+    return j
 
 
 def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
@@ -92,13 +104,16 @@ def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
     q: target distribution of the node; p: drafter distribution (None at a leaf)
     child_ids: its children in stored order; tokens[c]: draft token of node c
     (a negative token means "no draft" and is skipped).
-    Returns (next_child or -1, sampled token or -1, {child: (m, thr)}).
+    Returns (next_child or -1, sampled token or -1, {child: (m, thr, cut_margin)});
+    tested["resample_margin"] is set when a token was drawn.
     """
     nxt, q_cur, tested = sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam,
                                       code_offset, n_codes)
     if nxt >= 0:
         return nxt, -1, tested
-    return -1, inverse_cdf(q_cur, u_resample), tested
+    j, margin = inverse_cdf(q_cur, u_resample, return_margin=True)
+    tested["resample_margin"] = margin
+    return -1, j, tested
 
 
 def walk(node_next, node_token, tokens):
@@ -133,6 +148,8 @@ def verify_sequence(parent, target_cond, target_uncond, draft_cond, draft_uncond
     node_token = np.full(N, -1, dtype=np.int64)
     node_mass = np.full(N, -1.0)
     node_thresh = np.full(N, -1.0)
+    cut_margin = np.full(N, np.inf)
+    resample_margin = np.full(N, np.inf)
     for n in range(N):
         q, _ = postprocess_row(target_cond[n], None if target_uncond is None else target_uncond[n],
                                cfg_scale, temperature, top_k_target, allowed_begin, allowed_end)
@@ -143,12 +160,13 @@ def verify_sequence(parent, target_cond, target_uncond, draft_cond, draft_uncond
         nxt, tok, tested = verify_node(q, p, children[n], tokens, u_accept, u_resample[n],
                                        nbr_idx, k, lam, code_offset, n_codes)
         node_next[n], node_token[n] = nxt, tok
-        for c, (m, thr) in tested.items():
-            node_mass[c], node_thresh[c] = m, thr
+        resample_margin[n] = tested.pop("resample_margin", np.inf)
+        for c, (m, thr, cm) in tested.items():
+            node_mass[c], node_thresh[c], cut_margin[c] = m, thr, cm
     accept_len, out_tokens, out_nodes = walk(node_next, node_token, tokens)
     return dict(node_next=node_next, node_token=node_token, node_mass=node_mass,
                 node_thresh=node_thresh, accept_len=accept_len, out_tokens=out_tokens,
-                out_nodes=out_nodes)
+                out_nodes=out_nodes, cut_margin=cut_margin, resample_margin=resample_margin)
 
 
 def verify_batch(parent, target_cond, target_uncond, draft_cond, draft_uncond, tokens,

@@ -1,0 +1,18 @@
+"""Relaxed (LANTERN++) tree verification on B200: CUDA kernels behind a C ABI.
+
+p is the DRAFTER distribution and q the TARGET distribution, as in the paper.
+Every function here only marshals arguments for liblantern.so; all arithmetic
+runs in the CUDA kernels.  Importing fails loudly if the library is missing.
+"""
+from .binding import (  # noqa: F401
+    LIB_PATH,
+    LanternError,
+    Params,
+    Tree,
+    build_neighbors,
+    sample_draft_tree,
+    verify_tree,
+    philox_raw,
+    set_cluster_size,
+    lib,
+)

@@ -1,0 +1,236 @@
+"""ctypes binding of include/lantern.h.  Same names, argument marshalling only.
+
+Tensors are torch CUDA tensors (PyTorch supplies device memory and streams);
+pointers, strides and the current stream are handed to the C ABI.
+"""
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblantern.so")
+
+STATUS = {0: "ok", 1: "invalid argument", 2: "unsupported size", 3: "workspace", 4: "CUDA runtime error"}
+DEV_BAD_INDEX, DEV_TIMEOUT, DEV_EMPTY_ROW = 1, 2, 4
+
+
+class LanternError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, STATUS.get(status, "?"), status))
+
+
+class _CParams(ctypes.Structure):
+    _fields_ = [
+        ("cfg_scale", ctypes.c_float), ("temperature", ctypes.c_float),
+        ("top_k_target", ctypes.c_int32), ("top_k_draft", ctypes.c_int32),
+        ("lam", ctypes.c_float), ("k", ctypes.c_int32), ("vocab", ctypes.c_int32),
+        ("code_offset", ctypes.c_int32), ("n_codes", ctypes.c_int32),
+        ("allowed_begin", ctypes.c_int32), ("allowed_end", ctypes.c_int32),
+        ("seed", ctypes.c_uint64), ("step", ctypes.c_uint64),
+    ]
+
+
+@dataclass
+class Params:
+    """Mirror of lantern_params (see include/lantern.h)."""
+    vocab: int
+    cfg_scale: float = 1.0
+    temperature: float = 1.0
+    top_k_target: int = 0
+    top_k_draft: int = 0
+    lam: float = 1.0
+    k: int = 0
+    code_offset: int = 0
+    n_codes: int = 0
+    allowed_begin: int = 0
+    allowed_end: int = 0
+    seed: int = 0
+    step: int = 0
+
+    def c(self):
+        return _CParams(self.cfg_scale, self.temperature, self.top_k_target, self.top_k_draft,
+                        self.lam, self.k, self.vocab, self.code_offset, self.n_codes,
+                        self.allowed_begin, self.allowed_end, self.seed, self.step)
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "liblantern.so is missing: build it with `python -m paper_2502_06352_b200.build` "
+            "(needs nvcc; there is no CPU fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    L.lantern_status_string.restype = ctypes.c_char_p
+    L.lantern_status_string.argtypes = [ctypes.c_int]
+    L.lantern_tree_create.restype = ctypes.c_int
+    L.lantern_tree_create.argtypes = [vp, i32, ctypes.POINTER(vp)]
+    L.lantern_tree_destroy.restype = ctypes.c_int
+    L.lantern_tree_destroy.argtypes = [vp]
+    L.lantern_tree_max_depth.restype = i32
+    L.lantern_tree_max_depth.argtypes = [vp]
+    L.lantern_build_neighbors_workspace.restype = sz
+    L.lantern_build_neighbors_workspace.argtypes = [ctypes.c_int, i32, i32, i32]
+    L.lantern_build_neighbors.restype = ctypes.c_int
+    L.lantern_build_neighbors.argtypes = [vp, ctypes.c_int, i32, i32, i32, vp, vp, vp, sz, vp]
+    L.lantern_sample_draft_tree.restype = ctypes.c_int
+    L.lantern_sample_draft_tree.argtypes = [ctypes.POINTER(_CParams), vp, vp, vp, ctypes.c_int, i64, i64,
+                                            i32, i32, i32, vp, vp, vp, vp, vp]
+    L.lantern_verify_tree_workspace.restype = sz
+    L.lantern_verify_tree_workspace.argtypes = [vp, i32]
+    L.lantern_verify_tree.restype = ctypes.c_int
+    L.lantern_verify_tree.argtypes = [ctypes.POINTER(_CParams), vp, vp, i32, vp, vp, vp, vp, ctypes.c_int,
+                                      i64, i64, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.lantern_philox_raw.restype = ctypes.c_int
+    L.lantern_philox_raw.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
+                                     ctypes.c_uint32, i32, vp, vp]
+    L.lantern_set_cluster_size.restype = i32
+    L.lantern_set_cluster_size.argtypes = [i32]
+    return L
+
+
+lib = _load()
+
+
+def _check(status, where):
+    if status != 0:
+        raise LanternError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t):
+    if t.dtype == torch.float32:
+        return 0
+    if t.dtype == torch.bfloat16:
+        return 1
+    raise TypeError("logits / codebook must be float32 or bfloat16")
+
+
+class Tree:
+    """Static draft tree handle (lantern_tree_create / lantern_tree_destroy)."""
+
+    def __init__(self, parent):
+        self.parent = [int(x) for x in parent]
+        self.n_nodes = len(self.parent)
+        arr = (ctypes.c_int32 * self.n_nodes)(*self.parent)
+        h = ctypes.c_void_p()
+        _check(lib.lantern_tree_create(arr, self.n_nodes, ctypes.byref(h)), "lantern_tree_create")
+        self.handle = h
+        self.max_depth = lib.lantern_tree_max_depth(h)
+
+    def __del__(self):
+        h = getattr(self, "handle", None)
+        if h is not None and lib is not None:
+            lib.lantern_tree_destroy(h)
+            self.handle = None
+
+
+def _rows(t: torch.Tensor, B, N, V):
+    """(row_stride, seq_stride) in elements of a [B][N][V] tensor with unit inner stride."""
+    if t.dim() != 3 or t.shape[0] != B or t.shape[1] != N or t.shape[2] != V or t.stride(2) != 1:
+        raise ValueError("expected a [B][N][V] tensor with contiguous rows")
+    return t.stride(1), t.stride(0)
+
+
+def build_neighbors(codebook: torch.Tensor, k: int, return_dist=False):
+    """lantern_build_neighbors: [L][k] int32 nearest-neighbour table of an [L][d] codebook."""
+    if not codebook.is_cuda or not codebook.is_contiguous() or codebook.dim() != 2:
+        raise ValueError("codebook must be a contiguous [L][d] CUDA tensor")
+    L, d = codebook.shape
+    idx = torch.empty((L, k), dtype=torch.int32, device=codebook.device)
+    dist = torch.empty((L, k), dtype=torch.float32, device=codebook.device) if return_dist else None
+    dt = _dtype_code(codebook)
+    wbytes = lib.lantern_build_neighbors_workspace(dt, L, d, k)
+    ws = torch.empty(max(wbytes, 256), dtype=torch.uint8, device=codebook.device)
+    with torch.cuda.device(codebook.device):
+        _check(lib.lantern_build_neighbors(_ptr(codebook), dt, L, d, k, _ptr(idx), _ptr(dist), _ptr(ws),
+                                           ws.numel(), _stream()), "lantern_build_neighbors")
+    return (idx, dist) if return_dist else idx
+
+
+def sample_draft_tree(params: Params, tree: Tree, draft_cond, draft_uncond=None, *, tokens=None,
+                      parent_begin=0, parent_end=None, gumbel_uniforms=None, draft_prob=None,
+                      device_status=None):
+    """lantern_sample_draft_tree.  Returns tokens [B][N] int32 (allocated when not given)."""
+    B, N, V = draft_cond.shape[0], tree.n_nodes, params.vocab
+    rs, ss = _rows(draft_cond, B, N, V)
+    if draft_uncond is not None and _rows(draft_uncond, B, N, V) != (rs, ss):
+        raise ValueError("cond and uncond rows must share strides")
+    if tokens is None:
+        tokens = torch.full((B, N), -1, dtype=torch.int32, device=draft_cond.device)
+    if gumbel_uniforms is not None and (not gumbel_uniforms.is_contiguous() or gumbel_uniforms.dtype != torch.float32
+                                        or tuple(gumbel_uniforms.shape) != (B, N, V)):
+        raise ValueError("gumbel_uniforms must be contiguous float32 [B][N][V]")
+    cp = params.c()
+    with torch.cuda.device(draft_cond.device):
+        _check(lib.lantern_sample_draft_tree(
+            ctypes.byref(cp), tree.handle, _ptr(draft_cond), _ptr(draft_uncond), _dtype_code(draft_cond), rs, ss,
+            B, parent_begin, N if parent_end is None else parent_end, _ptr(gumbel_uniforms), _ptr(tokens),
+            _ptr(draft_prob), _ptr(device_status), _stream()), "lantern_sample_draft_tree")
+    return tokens
+
+
+def verify_tree(params: Params, tree: Tree, nbr_idx, target_cond, target_uncond, draft_cond, draft_uncond,
+                tokens, u_accept=None, u_resample=None, *, out=None, debug=False, device_status=None,
+                workspace=None):
+    """lantern_verify_tree.  Returns a dict of tensors: accept_len [B], out_tokens and
+    out_nodes [B][max_depth+1]; with debug=True also node_next, node_token, node_mass,
+    node_thresh [B][N].  `out` may carry preallocated tensors under the same names."""
+    B, N, V = target_cond.shape[0], tree.n_nodes, params.vocab
+    rs, ss = _rows(target_cond, B, N, V)
+    for t in (target_uncond, draft_cond, draft_uncond):
+        if t is not None and _rows(t, B, N, V) != (rs, ss):
+            raise ValueError("all logit tensors must share strides")
+    dev = target_cond.device
+    out = {} if out is None else out
+    D1 = tree.max_depth + 1
+
+    def get(name, shape, dtype):
+        if name not in out:
+            out[name] = torch.empty(shape, dtype=dtype, device=dev)
+        return out[name]
+
+    accept_len = get("accept_len", (B,), torch.int32)
+    out_tokens = get("out_tokens", (B, D1), torch.int32)
+    out_nodes = get("out_nodes", (B, D1), torch.int32)
+    node_next = node_token = node_mass = node_thresh = None
+    if debug:
+        node_next = get("node_next", (B, N), torch.int32)
+        node_token = get("node_token", (B, N), torch.int32)
+        node_mass = get("node_mass", (B, N), torch.float32)
+        node_thresh = get("node_thresh", (B, N), torch.float32)
+    if workspace is None:
+        need = lib.lantern_verify_tree_workspace(tree.handle, B)
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    k_table = 0 if nbr_idx is None else nbr_idx.shape[1]
+    cp = params.c()
+    with torch.cuda.device(dev):
+        _check(lib.lantern_verify_tree(
+            ctypes.byref(cp), tree.handle, _ptr(nbr_idx), k_table, _ptr(target_cond), _ptr(target_uncond),
+            _ptr(draft_cond), _ptr(draft_uncond), _dtype_code(target_cond), rs, ss, B, _ptr(tokens),
+            _ptr(u_accept), _ptr(u_resample), _ptr(accept_len), _ptr(out_tokens), _ptr(out_nodes),
+            _ptr(node_next), _ptr(node_token), _ptr(node_mass), _ptr(node_thresh), _ptr(device_status),
+            _ptr(workspace), workspace.numel(), _stream()), "lantern_verify_tree")
+    return out
+
+
+def philox_raw(seed, first, c1, c2, c3, n, device="cuda"):
+    """lantern_philox_raw: [n][4] raw Philox-4x32-10 words as int64 (values < 2^32)."""
+    out = torch.empty((n, 4), dtype=torch.int32, device=device)
+    with torch.cuda.device(out.device):
+        _check(lib.lantern_philox_raw(seed, first, c1, c2, c3, n, _ptr(out), _stream()), "lantern_philox_raw")
+    return out.to(torch.int64) & 0xFFFFFFFF
+
+
+def set_cluster_size(ctas_per_row: int) -> int:
+    """lantern_set_cluster_size: 0 = automatic; returns the previous value."""
+    return lib.lantern_set_cluster_size(ctas_per_row)

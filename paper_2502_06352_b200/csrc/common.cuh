@@ -1,0 +1,132 @@
+// Shared device helpers: thread-block-cluster primitives, reductions, Philox.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lantern.h"
+
+namespace lantern {
+
+constexpr int kThreads = 256;           // threads per CTA of the row kernels
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxCluster = 16;         // CTAs one logit row may be split over
+
+// Host-side tree handle (the C ABI's opaque lantern_tree).
+struct TreeDev {
+  int32_t n_nodes;
+  int32_t max_depth;
+  int32_t max_children;
+  int32_t n_internal;
+  int32_t* d_first_child;   // [N] first child id, or -1
+  int32_t* d_n_child;       // [N]
+  int32_t* d_order;         // [N] node ids, internal nodes first (launch order)
+  void* d_block;            // the one allocation behind the arrays above
+  int32_t* h_first_child;
+  int32_t* h_n_child;
+};
+
+// ---------------------------------------------------------------- cluster primitives
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+// Barrier over every thread of the cluster; release/acquire at cluster scope.
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;"
+               ::: "memory");
+}
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_saddr, uint32_t rank) {
+  uint32_t d;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(d) : "r"(local_saddr), "r"(rank));
+  return d;
+}
+__device__ __forceinline__ float dsmem_ld_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t dsmem_ld_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+
+// ---------------------------------------------------------------- warp / block reductions
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_incl_scan(float v, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    float t = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += t;
+  }
+  return v;
+}
+
+// Monotone map float -> uint32 (larger float, larger key; -0 < +0).
+__device__ __forceinline__ uint32_t float_key(float f) {
+  uint32_t b = __float_as_uint(f);
+  return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+  uint32_t b = (k >> 31) ? (k ^ 0x80000000u) : ~k;
+  return __uint_as_float(b);
+}
+
+// ---------------------------------------------------------------- Philox-4x32-10
+// Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3" (SC 2011).
+struct Philox4 { uint32_t x, y, z, w; };
+__host__ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2,
+                                                          uint32_t c3, uint32_t k0, uint32_t k1) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint64_t p0 = static_cast<uint64_t>(M0) * c0;
+    uint64_t p1 = static_cast<uint64_t>(M1) * c2;
+    uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ k0;
+    uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ k1;
+    c1 = static_cast<uint32_t>(p1);
+    c3 = static_cast<uint32_t>(p0);
+    c0 = n0;
+    c2 = n2;
+    k0 += W0;
+    k1 += W1;
+  }
+  return Philox4{c0, c1, c2, c3};
+}
+enum { kStreamGumbel = 0, kStreamAccept = 1, kStreamResample = 2 };
+// counter = (block, row, step_lo, step_hi << 2 | stream), key = seed
+__device__ __forceinline__ Philox4 philox_stream(uint64_t seed, uint64_t step, uint32_t row,
+                                                 uint32_t stream, uint32_t block) {
+  return philox4x32_10(block, row, static_cast<uint32_t>(step),
+                       (static_cast<uint32_t>(step >> 32) << 2) | stream,
+                       static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32));
+}
+__device__ __forceinline__ float uniform_halfopen(uint32_t x) {   // [0,1)
+  return static_cast<float>(x >> 8) * 5.9604644775390625e-8f;
+}
+__device__ __forceinline__ float uniform_open(uint32_t x) {       // (0,1), exact in float32
+  return (static_cast<float>(x >> 9) + 0.5f) * 1.1920928955078125e-7f;
+}
+
+}  // namespace lantern

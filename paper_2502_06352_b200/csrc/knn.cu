@@ -1,0 +1,279 @@
+// Latent-neighbour table (Sec. 2.2 / Sec. 4: B_k = k nearest codebook entries; App. A.1:
+// codebook C = {c_1..c_L}, c_i in R^d).  Exact squared-Euclidean k-NN of every row, ordered
+// by (distance, index), self excluded.
+//
+// Exact brute-force kernel.  A CTA owns a tile of QT query rows and streams over all L
+// candidate rows; distances are accumulated in double precision (sum of squared differences,
+// so duplicate rows give distance exactly 0 and equal distances to third rows).  Selection is
+// streaming: per query a float32 threshold tau (the k-th smallest rounded distance seen so
+// far) filters candidates into a shared-memory buffer; when the buffer fills it is sorted and
+// cut back to the entries <= the new tau (rounding to float32 is monotone, so nothing that can
+// belong to the exact top k is ever dropped).  The survivors are re-ranked by their double
+// distances.  If ties at tau overflow the buffer the query falls back to k rounds of an exact
+// arg-min over all candidates.
+#include "common.cuh"
+
+namespace lantern {
+
+constexpr int kKnnThreads = 256;
+constexpr int kDC = 32;             // embedding dims staged per step
+
+struct KnnArgs {
+  const void* cb;
+  int L, d, k, QT, CAP, q_double;
+  int32_t* nbr_idx;
+  float* nbr_dist;
+};
+
+template <typename T> __device__ __forceinline__ float widen(T x);
+template <> __device__ __forceinline__ float widen<float>(float x) { return x; }
+template <> __device__ __forceinline__ float widen<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// in-place ascending bitonic sort of n (power of two) 64-bit keys in shared memory
+__device__ __forceinline__ void bitonic_u64(unsigned long long* a, int n) {
+  for (int size = 2; size <= n; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = threadIdx.x; i < (n >> 1); i += kKnnThreads) {
+        int lo = 2 * i - (i & (stride - 1));
+        int hi = lo + stride;
+        bool up = (lo & size) == 0;
+        unsigned long long x = a[lo], y = a[hi];
+        if ((x > y) == up) { a[lo] = y; a[hi] = x; }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// ascending bitonic sort of n (power of two) (dist, idx) pairs
+__device__ __forceinline__ void bitonic_pair(double* dv, int* iv, int n) {
+  for (int size = 2; size <= n; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = threadIdx.x; i < (n >> 1); i += kKnnThreads) {
+        int lo = 2 * i - (i & (stride - 1));
+        int hi = lo + stride;
+        bool up = (lo & size) == 0;
+        double dx = dv[lo], dy = dv[hi];
+        int ix = iv[lo], iy = iv[hi];
+        bool gt = dx > dy || (dx == dy && ix > iy);
+        if (gt == up) { dv[lo] = dy; dv[hi] = dx; iv[lo] = iy; iv[hi] = ix; }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ double exact_dist(const T* __restrict__ cb, int d, int i, int j) {
+  const T* a = cb + static_cast<long long>(i) * d;
+  const T* b = cb + static_cast<long long>(j) * d;
+  double s = 0.0;
+  for (int t = 0; t < d; ++t) {
+    double diff = static_cast<double>(widen<T>(a[t])) - static_cast<double>(widen<T>(b[t]));
+    s = fma(diff, diff, s);
+  }
+  return s;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kKnnThreads) knn_kernel(const KnnArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int QT = a.QT, CAP = a.CAP, d = a.d, L = a.L, k = a.k;
+  const T* cb = static_cast<const T*>(a.cb);
+  // layout: buf[QT][CAP] u64 | sortd[CAP] f64 | sorti[CAP] i32 | cand[256][kDC+1] f32 | tau[QT] f32 |
+  //         cnt[QT] i32 | ovf[QT] i32 | redd[8] f64 | redi[8] i32 | queries
+  unsigned long long* buf = reinterpret_cast<unsigned long long*>(smem_raw);
+  double* sortd = reinterpret_cast<double*>(buf + static_cast<size_t>(QT) * CAP);
+  double* redd = sortd + CAP;
+  int* sorti = reinterpret_cast<int*>(redd + 8);
+  float* cand = reinterpret_cast<float*>(sorti + CAP);
+  float* tau = cand + kKnnThreads * (kDC + 1);
+  int* cnt = reinterpret_cast<int*>(tau + QT);
+  int* ovf = cnt + QT;
+  int* redi = ovf + QT;
+  unsigned char* qraw = reinterpret_cast<unsigned char*>(redi + 8);
+  qraw += (16 - (reinterpret_cast<uintptr_t>(qraw) & 15)) & 15;
+  double* qd = reinterpret_cast<double*>(qraw);
+  float* qf = reinterpret_cast<float*>(qraw);
+
+  const int tid = threadIdx.x;
+  const int q0 = blockIdx.x * QT;
+  const int nq = min(QT, L - q0);
+
+  for (int i = tid; i < QT * d; i += kKnnThreads) {
+    int q = i / d, t = i - q * d;
+    float v = (q < nq) ? widen<T>(cb[static_cast<long long>(q0 + q) * d + t]) : 0.f;
+    if (a.q_double) qd[i] = static_cast<double>(v); else qf[i] = v;
+  }
+  if (tid < QT) { tau[tid] = INFINITY; cnt[tid] = 0; ovf[tid] = 0; }
+  __syncthreads();
+
+  constexpr int MAXQT = 8;
+  for (int base = 0; base < L; base += kKnnThreads) {
+    double acc[MAXQT];
+#pragma unroll
+    for (int q = 0; q < MAXQT; ++q) acc[q] = 0.0;
+    const int ncand = min(kKnnThreads, L - base);
+    for (int db = 0; db < d; db += kDC) {
+      const int dc = min(kDC, d - db);
+      __syncthreads();
+      for (int i = tid; i < ncand * dc; i += kKnnThreads) {
+        int r = i / dc, t = i - r * dc;
+        cand[r * (kDC + 1) + t] = widen<T>(cb[static_cast<long long>(base + r) * d + db + t]);
+      }
+      __syncthreads();
+      if (tid < ncand) {
+        for (int t = 0; t < dc; ++t) {
+          const double cv = static_cast<double>(cand[tid * (kDC + 1) + t]);
+#pragma unroll
+          for (int q = 0; q < MAXQT; ++q) {
+            if (q < QT) {
+              double qv = a.q_double ? qd[q * d + db + t] : static_cast<double>(qf[q * d + db + t]);
+              double diff = qv - cv;
+              acc[q] = fma(diff, diff, acc[q]);
+            }
+          }
+        }
+      }
+    }
+    // filter into the per-query buffers
+    if (tid < ncand) {
+      const int j = base + tid;
+#pragma unroll
+      for (int q = 0; q < MAXQT; ++q) {
+        if (q < nq && j != q0 + q) {
+          float f = static_cast<float>(acc[q]);
+          if (f <= tau[q]) {
+            int pos = atomicAdd(&cnt[q], 1);
+            if (pos < CAP) buf[static_cast<size_t>(q) * CAP + pos] =
+                (static_cast<unsigned long long>(__float_as_uint(f)) << 32) | static_cast<unsigned>(j);
+          }
+        }
+      }
+    }
+    __syncthreads();
+    // cut back buffers that might overflow during the next tile
+    for (int q = 0; q < nq; ++q) {
+      int n = cnt[q];
+      if (n <= CAP - kKnnThreads || ovf[q]) continue;     // uniform: cnt/ovf are shared
+      unsigned long long* bq = buf + static_cast<size_t>(q) * CAP;
+      for (int i = n + tid; i < CAP; i += kKnnThreads) bq[i] = ~0ull;
+      __syncthreads();
+      bitonic_u64(bq, CAP);
+      // keep everything <= the k-th smallest rounded distance
+      if (tid == 0) {
+        uint32_t tb = static_cast<uint32_t>(bq[k - 1] >> 32);
+        int m = k;
+        while (m < n && static_cast<uint32_t>(bq[m] >> 32) == tb) ++m;
+        tau[q] = __uint_as_float(tb);
+        cnt[q] = m;
+        if (m > CAP - kKnnThreads) ovf[q] = 1;      // ties at tau fill the buffer
+      }
+      __syncthreads();
+    }
+  }
+
+  // final ranking per query
+  for (int q = 0; q < nq; ++q) {
+    const int qi = q0 + q;
+    int32_t* out_i = a.nbr_idx + static_cast<long long>(qi) * k;
+    float* out_d = a.nbr_dist ? a.nbr_dist + static_cast<long long>(qi) * k : nullptr;
+    if (!ovf[q]) {
+      const int n = min(cnt[q], CAP);
+      const unsigned long long* bq = buf + static_cast<size_t>(q) * CAP;
+      for (int i = tid; i < CAP; i += kKnnThreads) {
+        if (i < n) {
+          int j = static_cast<int>(bq[i] & 0xffffffffu);
+          sorti[i] = j;
+          sortd[i] = exact_dist<T>(cb, d, qi, j);
+        } else {
+          sorti[i] = 0x7fffffff;
+          sortd[i] = INFINITY;
+        }
+      }
+      __syncthreads();
+      bitonic_pair(sortd, sorti, CAP);
+      for (int r = tid; r < k; r += kKnnThreads) {
+        out_i[r] = sorti[r];
+        if (out_d) out_d[r] = static_cast<float>(sortd[r]);
+      }
+      __syncthreads();
+    } else {
+      // exact fallback: k rounds of arg-min over (distance, index) greater than the last pick
+      double pd = -1.0;
+      int pj = -1;
+      for (int r = 0; r < k; ++r) {
+        double bd = INFINITY;
+        int bj = 0x7fffffff;
+        for (int j = tid; j < L; j += kKnnThreads) {
+          if (j == qi) continue;
+          double dj = exact_dist<T>(cb, d, qi, j);
+          bool after = dj > pd || (dj == pd && j > pj);
+          if (after && (dj < bd || (dj == bd && j < bj))) { bd = dj; bj = j; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          double od = __shfl_xor_sync(0xffffffffu, bd, o);
+          int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+          if (od < bd || (od == bd && oj < bj)) { bd = od; bj = oj; }
+        }
+        if ((tid & 31) == 0) { redd[tid >> 5] = bd; redi[tid >> 5] = bj; }
+        __syncthreads();
+        bd = redd[0]; bj = redi[0];
+        for (int w = 1; w < kKnnThreads / 32; ++w)
+          if (redd[w] < bd || (redd[w] == bd && redi[w] < bj)) { bd = redd[w]; bj = redi[w]; }
+        __syncthreads();
+        pd = bd; pj = bj;
+        if (tid == 0) {
+          out_i[r] = bj;
+          if (out_d) out_d[r] = static_cast<float>(bd);
+        }
+      }
+    }
+  }
+}
+
+}  // namespace lantern
+
+using namespace lantern;
+
+extern "C" size_t lantern_build_neighbors_workspace(lantern_dtype dt, int32_t L, int32_t d, int32_t k) {
+  (void)dt; (void)L; (void)d; (void)k;
+  return 0;   // the brute-force kernel keeps all of its state on chip
+}
+
+extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_dtype dt, int32_t L, int32_t d,
+                                                  int32_t k, int32_t* nbr_idx, float* nbr_dist, void* workspace,
+                                                  size_t workspace_bytes, void* stream) {
+  (void)workspace; (void)workspace_bytes;
+  if (!codebook || !nbr_idx) return LANTERN_ERR_INVALID_ARG;
+  if (dt != LANTERN_F32 && dt != LANTERN_BF16) return LANTERN_ERR_INVALID_ARG;
+  if (L < 2 || d < 1 || k < 1 || k > L - 1) return LANTERN_ERR_INVALID_ARG;
+  if (k > 1024 || d > 4096) return LANTERN_ERR_UNSUPPORTED;
+  KnnArgs a;
+  a.cb = codebook; a.L = L; a.d = d; a.k = k; a.nbr_idx = nbr_idx; a.nbr_dist = nbr_dist;
+  int cap = 512;
+  while (cap < k + 2 * kKnnThreads) cap *= 2;
+  a.CAP = cap;
+  a.QT = cap <= 1024 ? 8 : 4;
+  auto smem_for = [&](int qt, int qdouble) {
+    return static_cast<size_t>(qt) * cap * 8 + static_cast<size_t>(cap) * 12 + 8 * 12 +
+           static_cast<size_t>(kKnnThreads) * (kDC + 1) * 4 + static_cast<size_t>(qt) * 12 + 16 +
+           static_cast<size_t>(qt) * d * (qdouble ? 8 : 4);
+  };
+  a.q_double = smem_for(a.QT, 1) <= 160 * 1024 ? 1 : 0;
+  while (a.QT > 1 && smem_for(a.QT, a.q_double) > 220 * 1024) a.QT /= 2;
+  size_t smem = smem_for(a.QT, a.q_double);
+  if (smem > 227 * 1024) return LANTERN_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int grid = (L + a.QT - 1) / a.QT;
+  cudaError_t e;
+  if (dt == LANTERN_F32) {
+    e = cudaFuncSetAttribute(knn_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e == cudaSuccess) { knn_kernel<float><<<grid, kKnnThreads, smem, st>>>(a); e = cudaGetLastError(); }
+  } else {
+    e = cudaFuncSetAttribute(knn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e == cudaSuccess) { knn_kernel<__nv_bfloat16><<<grid, kKnnThreads, smem, st>>>(a); e = cudaGetLastError(); }
+  }
+  return e == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
+}

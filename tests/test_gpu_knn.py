@@ -1,0 +1,73 @@
+"""Parity of lantern_build_neighbors with the oracle's brute force (Sec. 2.2 / Sec. 4: B_k)."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from parity_util import compare_neighbors
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def L():
+    import paper_2502_06352_b200 as lib
+    return lib
+
+
+def _check(L, cb, k, rows=None):
+    idx, dist = L.build_neighbors(cb.cuda(), k, return_dist=True)
+    torch.cuda.synchronize()
+    idx, dist = idx.cpu().numpy(), dist.cpu().numpy()
+    cb64 = cb.to(torch.float64).numpy()
+    n = cb.shape[0]
+    rows = list(range(n)) if rows is None else rows
+    ties = compare_neighbors(idx, dist, cb64, rows, k)
+    assert ties == 0 or ties <= len(rows) // 1000
+    return idx, dist
+
+
+@pytest.mark.parametrize("n,d,k,dt", [(2, 1, 1, "f32"), (17, 3, 16, "f32"), (300, 8, 10, "f32"),
+                                      (1000, 8, 50, "bf16"), (777, 64, 33, "bf16"), (600, 256, 200, "bf16"),
+                                      (1500, 40, 700, "f32")])
+def test_small_codebooks_all_rows(L, n, d, k, dt):
+    cb = W.make_codebook(n, d, dt, seed=n + d, dup_frac=0.05 if n > 50 else 0.0)
+    _check(L, cb, k)
+
+
+def test_duplicates_tie_by_index_and_zero_distance(L):
+    cb = W.make_codebook(64, 8, "bf16", seed=1)
+    cb[10] = cb[3]
+    cb[40] = cb[3]
+    idx, dist = _check(L, cb, 5)
+    assert list(idx[3][:2]) == [10, 40] and list(dist[3][:2]) == [0, 0]
+    assert list(idx[10][:2]) == [3, 40] and list(idx[40][:2]) == [3, 10]
+
+
+def test_massive_ties_take_the_exact_fallback(L):
+    # every row equal: all distances are 0, neighbours are the lowest indices
+    cb = torch.ones((700, 4), dtype=torch.float32)
+    idx, dist = _check(L, cb, 20)
+    assert list(idx[0]) == list(range(1, 21)) and list(idx[5][:6]) == [0, 1, 2, 3, 4, 6]
+    # integer line: closed-form neighbours
+    cb = torch.arange(900, dtype=torch.float32)[:, None].contiguous()
+    idx, _ = _check(L, cb, 4, rows=[0, 450, 899])
+    assert list(idx[450]) == [449, 451, 448, 452]
+
+
+@pytest.mark.parametrize("n,d,k,dt", [(16384, 8, 100, "f32"), (8192, 256, 200, "bf16")])
+def test_config_codebooks_sampled_rows(L, n, d, k, dt):
+    cb = W.make_codebook(n, d, dt, seed=5, dup_frac=0.05)
+    rows = [0, 1, 2, n // 2, n - 1] + list(np.random.default_rng(0).integers(0, n, 20))
+    idx, _ = _check(L, cb, k, rows=rows)
+    # properties on every row: no self, distinct, in range
+    assert not np.any(idx == np.arange(n)[:, None])
+    s = np.sort(idx, axis=1)
+    assert np.all(s[:, 1:] != s[:, :-1]) and idx.min() >= 0 and idx.max() < n
+
+
+def test_sweep_largest_shape_sampled_rows(L):
+    n, d, k = 65536, 64, 50
+    cb = W.make_codebook(n, d, "bf16", seed=6, dup_frac=0.05)
+    rows = [0, n - 1] + list(np.random.default_rng(1).integers(0, n, 10))
+    _check(L, cb, k, rows=rows)

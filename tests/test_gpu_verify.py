@@ -1,0 +1,175 @@
+"""Parity of lantern_verify_tree with the oracle (Sec. 4; App. A.2 Eq. 1-2; Sec. 2.1)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as W
+from gpu_cases import Case, small_config
+from parity_util import check_walk, compare_verify
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def L():
+    import paper_2502_06352_b200 as lib
+    return lib
+
+
+def _run(L, case, **kw):
+    res = case.gpu_verify(L, **kw)
+    assert res["status"] == 0
+    orc = case.oracle_verify()
+    ua = case.u_accept.numpy()
+    stats = compare_verify(res, orc, case.parent, ua, case.seqs)
+    check_walk(res, case.tokens, res["max_depth"], orc, stats["dirty_sequences"], case.seqs)
+    assert stats["tie_accept"] + stats["tie_cut"] + stats["tie_resample"] <= max(1, stats["nodes"] // 500)
+    return res, stats
+
+
+@pytest.mark.parametrize("cs", [0, 1, 2, 4, 8, 16])
+def test_small_vocab_all_cluster_sizes(L, cs):
+    # V = 1003 with a padded row stride: ragged tail in the last slice, several slices
+    case = Case(small_config(vocab=1003, codebook_size=1003, k=8, lam=3.0), seed=1, pad=5)
+    old = L.set_cluster_size(cs)
+    try:
+        _run(L, case)
+    finally:
+        L.set_cluster_size(old)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(cfg_scale=None),                                   # no guidance rows
+    dict(top_k=50),                                         # truncation on both sides
+    dict(k=0),                                              # standard speculative sampling
+    dict(lam=1.0),                                          # bound 1: A = {x}
+    dict(lam=20.0, k=50),                                   # wide relaxation
+    dict(dtype="bf16", cfg_scale=None),
+    dict(dtype="bf16", top_k=30),
+    dict(temperature=0.7, top_k=100),
+    dict(codebook_size=300, code_offset=200, k=10),         # codes are a sub-range of the vocabulary
+    dict(n_nodes=60, batch=3),
+])
+def test_parameter_variants(L, kw):
+    case = Case(small_config(**kw), seed=2)
+    _run(L, case)
+
+
+def test_allowed_range_and_topk_counts_only_allowed(L):
+    case = Case(small_config(vocab=2048, codebook_size=512, code_offset=256, k=6, top_k=40), seed=3,
+                allowed=(256, 768))
+    res, _ = _run(L, case)
+    tok = res["node_token"]
+    assert np.all((tok == -1) | ((tok >= 256) & (tok < 768)))
+
+
+def test_unrelaxed_equals_textbook_thresholds(L):
+    """k = 0: thr = min(1, q/p) on the rows as torch computes them."""
+    case = Case(small_config(k=0, cfg_scale=None, batch=1), seed=4)
+    res, _ = _run(L, case)
+    q = torch.softmax(case.logits["target_cond"][0].double(), -1).numpy()
+    p = torch.softmax(case.logits["draft_cond"][0].double(), -1).numpy()
+    kids = oracle.tree_children(case.parent)
+    for n in range(case.N):
+        if kids[n]:
+            c = kids[n][0]          # the first child sees the unmodified rows
+            x = case.tokens[0, c]
+            assert abs(res["node_thresh"][0, c] - min(1.0, q[n, x] / p[n, x])) < 1e-5
+            assert abs(res["node_mass"][0, c] - q[n, x]) < 1e-6
+
+
+def test_identical_models_accept_first_chain(L):
+    cfg = small_config(draft_mix=1.0, draft_noise=0.0, batch=2)
+    case = Case(cfg, seed=5)
+    res, _ = _run(L, case)
+    depth = 0
+    n = 0
+    kids = oracle.tree_children(case.parent)
+    while kids[n]:
+        n = kids[n][0]
+        depth += 1
+    assert list(res["accept_len"]) == [depth, depth]
+
+
+def test_missing_drafts_and_single_node_tree(L):
+    case = Case(small_config(batch=2), seed=6)
+    case.tokens[0, 1] = -1           # first child of the root has no draft
+    case.tokens[1, 2:5] = -1
+    _run(L, case)
+    leaf = Case(small_config(batch=3), parent=[-1], seed=7)
+    res, _ = _run(L, leaf)
+    assert list(res["accept_len"]) == [0, 0, 0] and res["out_tokens"].shape == (3, 1)
+
+
+def test_philox_uniforms_match_oracle_stream(L):
+    case = Case(small_config(batch=2), seed=8)
+    seed, step = 0x1A27E2, (3 << 32) | 41
+    for b in range(case.B):
+        for n in range(case.N):
+            case.u_accept[b, n] = float(oracle.stream_uniforms(seed, step, b * case.N + n, 1))
+            case.u_resample[b, n] = float(oracle.stream_uniforms(seed, step, b * case.N + n, 2))
+    _run(L, case, use_philox=(seed, step))
+
+
+def test_bitwise_repeatable(L):
+    case = Case(small_config(top_k=64), seed=9)
+    a = case.gpu_verify(L)
+    b = case.gpu_verify(L)
+    for k in ("node_next", "node_token", "node_mass", "node_thresh", "accept_len", "out_tokens"):
+        assert a[k].tobytes() == b[k].tobytes()
+
+
+def test_bulk_copy_and_plain_table_paths_agree(L):
+    # k_table = 8 rows are 16-byte aligned (bulk async copy); k_table = 7 uses plain loads
+    a = Case(small_config(k=7), seed=10, k_table=8)
+    b = Case(small_config(k=7), seed=10, k_table=7)
+    ra, _ = _run(L, a)
+    rb, _ = _run(L, b)
+    assert np.array_equal(ra["node_next"], rb["node_next"]) and np.array_equal(ra["node_mass"], rb["node_mass"])
+
+
+def test_bad_table_index_is_flagged_not_faulted(L):
+    case = Case(small_config(batch=1, k=4), seed=11)
+    case.nbr = case.nbr.copy()
+    case.nbr[:, 1] = 10 ** 6          # outside the vocabulary
+    res = case.gpu_verify(L)
+    assert res["status"] & 1
+
+
+def test_invalid_arguments_are_rejected(L):
+    case = Case(small_config(batch=1), seed=12)
+    g, par, nbr, tok = case.gpu_inputs(L)
+    tree = L.Tree(case.parent)
+    par.lam = 0.5
+    with pytest.raises(L.LanternError) as e:
+        L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"], tok)
+    assert e.value.status == 1
+    par.lam = 2.0
+    par.k = 100                       # larger than the table
+    with pytest.raises(L.LanternError):
+        L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"], tok)
+    par.k = 4
+    bad = g["target_cond"][:, :, 1:]  # rows no longer 16-byte aligned
+    with pytest.raises((L.LanternError, ValueError)):
+        L.verify_tree(par, tree, nbr, bad, None, bad, None, tok)
+
+
+@pytest.mark.parametrize("name", ["c1_tiny", "c2_llamagen512"])
+def test_named_configs_full_size(L, name):
+    case = Case(W.CONFIGS[name], seed=0)
+    res, stats = _run(L, case)
+    print(name, {k: v for k, v in stats.items() if k != "dirty_sequences"})
+
+
+@pytest.mark.parametrize("name,seqs", [("c3_lumina", [0, 3]), ("c4_batch64", [0, 37, 63])])
+def test_large_vocab_configs_sampled_sequences(L, name, seqs):
+    case = Case(W.CONFIGS[name], seed=0, oracle_seqs=seqs)
+    res, stats = _run(L, case)
+    # properties that hold for every sequence
+    tok = res["node_token"]
+    nxt = res["node_next"]
+    assert np.all((nxt >= 0) != (tok >= 0))
+    thr = res["node_thresh"]
+    assert np.all((thr == -1) | ((thr >= 0) & (thr <= 1)))
+    print(name, {k: v for k, v in stats.items() if k != "dirty_sequences"})

@@ -31,7 +31,7 @@ def test_reduces_to_speculative_sampling():
                 tokens = [0, x]
                 u = [0.0, 1.0]      # force rejection to see the residual
                 nxt, q_cur, tested = oracle.sibling_loop(q, p, [1], tokens, u, nbr, k, lam, 0, V)
-                m, thr = tested[1]
+                m, thr = tested[1][:2]
                 assert m == q[x]
                 assert thr == min(1.0, q[x] / p[x])
                 res = np.maximum(q - p, 0)
@@ -73,7 +73,7 @@ def test_bound_on_accept_probability_and_monotonicity():
             row = []
             for kk in (0, 1, 2, 5, 10):
                 _, _, tested = oracle.sibling_loop(q, p, [1], [0, x], [0, 1.0], nbr, kk, lam, 0, V)
-                m, thr = tested[1]
+                m, thr = tested[1][:2]
                 assert thr <= lam * min(1.0, q[x] / p[x]) * (1 + 1e-12)
                 row.append((m, thr))
             ms = [r[0] for r in row]
@@ -180,7 +180,7 @@ def test_full_neighbourhood_unbounded_lambda_always_accepts():
     q, p = _dists(rng, V)
     for x in range(V):
         _, _, tested = oracle.sibling_loop(q, p, [1], [0, x], [0, 0.999999], nbr, V - 1, 1e30, 0, V)
-        m, thr = tested[1]
+        m, thr = tested[1][:2]
         assert abs(m - 1) < 1e-12 and thr == 1.0 or p[x] > m
 
 

@@ -14,4 +14,5 @@ from .generators import (  # noqa: F401
     make_uniforms,
     make_gumbel_uniforms,
     random_sibling_tokens,
+    random_neighbor_table,
 )

@@ -92,3 +92,30 @@ def random_sibling_tokens(parent, B, lo, hi, seed, device="cpu"):
                 new = torch.randint(lo, hi, (B,), generator=g, device=device, dtype=torch.int32)
                 tok[:, ch[a]] = torch.where(clash, new, tok[:, ch[a]])
     return tok
+
+
+def random_neighbor_table(L, k, seed, device="cpu"):
+    """[L][k] int32 table of k distinct indices != row per row, uniformly random.  A stand-in
+    for a real neighbour table where only its shape matters (the synthetic logits carry no
+    relation to codebook geometry)."""
+    g = _gen(seed, device)
+    # k distinct values of [0, L-1) per row via random keys, then skip over the row's own index
+    keys = torch.rand((L, L - 1) if L <= 2048 else (L, min(L - 1, 8 * k)), generator=g, device=device)
+    if keys.shape[1] == L - 1:
+        idx = keys.argsort(dim=1)[:, :k]
+    else:
+        # large L: draw with replacement from a wide range and keep the first k distinct values
+        cand = torch.randint(0, L - 1, (L, 8 * k), generator=g, device=device)
+        idx = torch.empty((L, k), dtype=torch.int64, device=device)
+        srt, order = cand.sort(dim=1, stable=True)
+        first = torch.ones_like(srt, dtype=torch.bool)
+        first[:, 1:] = srt[:, 1:] != srt[:, :-1]
+        keep = torch.zeros_like(first)
+        keep.scatter_(1, order, first)          # keep[r, c] = cand[r, c] is a first occurrence
+        rank = keep.cumsum(dim=1) - 1
+        sel = keep & (rank < k)
+        assert bool((sel.sum(dim=1) == k).all())
+        idx = cand[sel].view(L, k)
+    rows = torch.arange(L, device=device).unsqueeze(1)
+    idx = idx + (idx >= rows).to(idx.dtype)
+    return idx.to(torch.int32).contiguous()
