@@ -1,0 +1,364 @@
+"""Benchmark of the relaxed tree-verification hot path.
+
+One step = one pass of the path over one batch of synthetic input: the draft sampler over
+every internal node, the relaxed verification of every node and the walk (three kernel
+launches).  The neighbour table is built once per codebook and is timed separately.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints one JSON line (rank 0).  Under torchrun every rank verifies its own batch of
+sequences (no data-path collective); the value is all ranks' nodes over the slowest rank's
+device time.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verified tree nodes/sec"
+UNIT = "nodes/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="c2_llamagen512")
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--ring", type=int, default=0, help="input buffer sets cycled through (0 = enough to exceed L2)")
+    ap.add_argument("--e2e-steps", type=int, default=100)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def algorithmic_bytes(cfg, parent, batch):
+    """Bytes one verify launch must move: every target row and every internal node's drafter
+    row once, the neighbour rows of the draft tokens, and the per-node outputs."""
+    N = len(parent)
+    I = len(set(parent[1:]))
+    c = 2 if cfg.cfg_scale is not None else 1
+    e = 4 if cfg.dtype == "f32" else 2
+    rows = batch * (N + I) * c * cfg.vocab * e
+    table = batch * (N - 1) * cfg.k * 4
+    outs = batch * N * (4 + 4 + 4 + 4 + 4)      # tokens, two uniforms in; next, token out
+    return rows + table + outs, batch * I * c * cfg.vocab * e
+
+
+def peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples of one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        sm.sort()
+        # the busy half of the samples (the tool also samples before and after the region)
+        busy = sm[len(sm) // 2:] if sm else []
+        return {"sm_mhz": busy[len(busy) // 2] if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_step_inputs(cfg, parent, logits_cpu, seqs, seed):
+    import workloads as W
+    N, V = len(parent), cfg.vocab
+    gum = W.make_gumbel_uniforms(len(seqs), N, V, seed).numpy()
+    ua, ur = W.make_uniforms(len(seqs), N, seed + 1)
+    nbr = W.random_neighbor_table(cfg.codebook_size, cfg.k, seed + 2).numpy()
+    return gum, ua.numpy(), ur.numpy(), nbr
+
+
+def oracle_run_nodes(cfg, parent, lg, b, gum, ua, ur, nbr, n_nodes):
+    """Oracle sampler + verifier on the first n_nodes nodes of sequence b (bounded sample)."""
+    import numpy as np
+    import oracle
+    f = lambda t: None if t is None else t[b].float().numpy()
+    kw = dict(cfg_scale=cfg.cfg_scale if cfg.cfg_scale is not None else 1.0, temperature=cfg.temperature)
+    tc, tu, dc, du = f(lg["target_cond"]), f(lg["target_uncond"]), f(lg["draft_cond"]), f(lg["draft_uncond"])
+    children = oracle.tree_children(parent)
+    tokens, _ = oracle.sample_draft_tree(parent, dc, du, gum, top_k_draft=cfg.top_k, **kw)
+    tokens[0] = 0
+    done = 0
+    for n in range(min(n_nodes, len(parent))):
+        q, _ = oracle.postprocess_row(tc[n], None if tu is None else tu[n], kw["cfg_scale"], cfg.temperature, cfg.top_k)
+        p = None
+        if children[n]:
+            p, _ = oracle.postprocess_row(dc[n], None if du is None else du[n], kw["cfg_scale"], cfg.temperature, cfg.top_k)
+        oracle.verify_node(q, p, children[n], tokens, ua, ur[n], nbr, cfg.k, cfg.lam, cfg.code_offset, cfg.codebook_size)
+        done += 1
+    return done
+
+
+def cpu_baseline(cfg, parent, lg_cpu, budget_s=15.0):
+    """The oracle, as it stands, on whole sequences of the workload until about budget_s."""
+    N = len(parent)
+    B = lg_cpu["target_cond"].shape[0]
+    gum, ua, ur, nbr = oracle_step_inputs(cfg, parent, lg_cpu, list(range(B)), 4242)
+    t0 = time.perf_counter()
+    nodes = 0
+    seqs = 0
+    while True:
+        b = seqs % B
+        nodes += oracle_run_nodes(cfg, parent, lg_cpu, b, gum[b], ua[b], ur[b], nbr, N)
+        seqs += 1
+        if time.perf_counter() - t0 > budget_s or seqs >= 4 * B:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": nodes / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "%d whole sequences (%d nodes: draft sampling + relaxed verification of every node) of %s, %.1f s"
+                      % (seqs, nodes, cfg.name, dt)}
+
+
+def run_reference(args, cfg, parent):
+    """--impl reference: the CPU oracle on bounded samples of the same workload."""
+    import workloads as W
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    N = len(parent)
+    lg = W.make_logits(cfg, step=0, device="cpu", batch=1)
+    gum, ua, ur, nbr = oracle_step_inputs(cfg, parent, lg, [0], 4242)
+    t0 = time.perf_counter()
+    oracle_run_nodes(cfg, parent, lg, 0, gum[0], ua[0], ur[0], nbr, 4)
+    t_node = (time.perf_counter() - t0) / 4
+    per_step = int(max(1, min(N, 120.0 / (max(1, args.steps + args.warmup) * t_node))))
+    for _ in range(args.warmup):
+        oracle_run_nodes(cfg, parent, lg, 0, gum[0], ua[0], ur[0], nbr, per_step)
+    t0 = time.perf_counter()
+    nodes = 0
+    for _ in range(args.steps):
+        nodes += oracle_run_nodes(cfg, parent, lg, 0, gum[0], ua[0], ur[0], nbr, per_step)
+    dt = time.perf_counter() - t0
+    val = nodes / dt
+    sample = "each step: draft sampling of one sequence + relaxed verification of its first %d of %d nodes" % (per_step, N)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(1, args.steps), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": 1, "tree_nodes": N, "vocab": cfg.vocab, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    args = parse_args()
+    import workloads as W
+    cfg = W.CONFIGS[args.workload]
+    parent = W.static_tree(cfg.n_nodes)
+    if args.impl == "reference":
+        run_reference(args, cfg, parent)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2502_06352_b200 as L
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    N, B, V = len(parent), cfg.batch, cfg.vocab
+    tree = L.Tree(parent)
+    alg_bytes, sampler_bytes = algorithmic_bytes(cfg, parent, B)
+    set_bytes = sum(B * N * V * (4 if cfg.dtype == "f32" else 2) for _ in range(4 if cfg.cfg_scale is not None else 2))
+    ring = args.ring if args.ring > 0 else max(2, -(-3 * 126 * 2 ** 20 // set_bytes))
+    ring = min(ring, max(2, int(60e9 // set_bytes)))
+
+    # ---- neighbour table: built once per codebook by the library (timed on its own)
+    codebook = W.make_codebook(cfg.codebook_size, cfg.codebook_dim, cfg.codebook_dtype, seed=cfg.index, device=dev)
+    nbr = L.build_neighbors(codebook, cfg.k)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    tb = []
+    for _ in range(3):
+        ev0.record()
+        nbr = L.build_neighbors(codebook, cfg.k)
+        ev1.record()
+        torch.cuda.synchronize()
+        tb.append(ev0.elapsed_time(ev1))
+    table_ms = min(tb)
+
+    # ---- inputs: a ring of independent step buffers, together larger than L2
+    bufs = [W.make_logits(cfg, step=1000 * rank + s, device=dev) for s in range(ring)]
+    params = L.Params(vocab=V, cfg_scale=cfg.cfg_scale if cfg.cfg_scale is not None else 1.0,
+                      temperature=cfg.temperature, top_k_target=cfg.top_k, top_k_draft=cfg.top_k, lam=cfg.lam,
+                      k=cfg.k, code_offset=cfg.code_offset, n_codes=cfg.codebook_size, seed=0x1A27E2 + rank)
+    tokens = torch.zeros((B, N), dtype=torch.int32, device=dev)
+    out = {}
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    need = L.lib.lantern_verify_tree_workspace(tree.handle, B)
+    workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+
+    def step(i, lg):
+        params.step = i
+        L.sample_draft_tree(params, tree, lg["draft_cond"], lg["draft_uncond"], tokens=tokens, device_status=status)
+        L.verify_tree(params, tree, nbr, lg["target_cond"], lg["target_uncond"], lg["draft_cond"], lg["draft_uncond"],
+                      tokens, None, None, out=out, device_status=status, workspace=workspace)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        step(i, bufs[i % ring])
+    sync_all()
+
+    # ---- timed region: exactly K steps, device-resident inputs
+    K = args.steps
+    kernel_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(min(K, 256))]
+    clocks = ClockSampler(local)
+    time.sleep(0.3)
+    sync_all()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    emitted = torch.zeros((), dtype=torch.int64, device=dev)
+    for i in range(K):
+        lg = bufs[i % ring]
+        params.step = 100000 + i
+        L.sample_draft_tree(params, tree, lg["draft_cond"], lg["draft_uncond"], tokens=tokens, device_status=status)
+        if i < len(kernel_ev):
+            kernel_ev[i][0].record()
+        L.verify_tree(params, tree, nbr, lg["target_cond"], lg["target_uncond"], lg["draft_cond"], lg["draft_uncond"],
+                      tokens, None, None, out=out, device_status=status, workspace=workspace)
+        if i < len(kernel_ev):
+            kernel_ev[i][1].record()
+    t_end.record()
+    sync_all()
+    elapsed_ms = t_start.elapsed_time(t_end)
+    clk = clocks.stop()
+    verify_ms = sorted(a.elapsed_time(b) for a, b in kernel_ev)
+    verify_avg_ms = sum(verify_ms) / len(verify_ms)
+    accept_mean = float(out["accept_len"].float().mean().item())
+    dev_status = int(status.item())
+
+    if world > 1:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    total_nodes = world * B * N * K
+    value = total_nodes / (elapsed_ms * 1e-3)
+
+    # ---- end to end: per step, inputs come from pinned host memory and results go back
+    KE = max(1, min(args.e2e_steps, K))
+    host = {k: (None if v is None else torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v))
+            for k, v in bufs[0].items()}
+    stage = {k: (None if v is None else torch.empty_like(v)) for k, v in bufs[0].items()}
+    h_len = torch.empty((B,), dtype=torch.int32, pin_memory=True)
+    h_tok = torch.empty((B, tree.max_depth + 1), dtype=torch.int32, pin_memory=True)
+    h2d = sum(v.numel() * v.element_size() for v in host.values() if v is not None)
+    d2h = h_len.numel() * 4 + h_tok.numel() * 4
+
+    def e2e_step(i):
+        for k_, v in host.items():
+            if v is not None:
+                stage[k_].copy_(v, non_blocking=True)
+        step(200000 + i, stage)
+        h_len.copy_(out["accept_len"], non_blocking=True)
+        h_tok.copy_(out["out_tokens"], non_blocking=True)
+        torch.cuda.synchronize()
+
+    for i in range(3):
+        e2e_step(i)
+    sync_all()
+    w0 = time.perf_counter()
+    t_start.record()
+    for i in range(KE):
+        e2e_step(i)
+    t_end.record()
+    sync_all()
+    e2e_ms = max(t_start.elapsed_time(t_end), 1e3 * (time.perf_counter() - w0))
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * B * N * KE / (e2e_ms * 1e-3)
+
+    if rank == 0:
+        peak, peak_kind = peak_hbm()
+        achieved = alg_bytes / (verify_avg_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
+            "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "batch_per_gpu": B, "tree_nodes": N, "vocab": V, "logits": cfg.dtype,
+                       "cfg_scale": cfg.cfg_scale, "top_k": cfg.top_k, "neighbours_k": cfg.k, "lambda": cfg.lam,
+                       "codebook": [cfg.codebook_size, cfg.codebook_dim], "parallelism": "dp%d" % world,
+                       "l2_policy": "ring of %d input sets, %.0f MB in total (> 126 MB L2)" % (ring, ring * set_bytes / 1e6),
+                       "step": "sample_draft_tree + verify_tree (+ walk)"},
+            "roofline": {"bound": "hbm", "kernel": "verify_nodes_kernel (+ walk_kernel)", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                         "algorithmic_bytes": alg_bytes, "launch_ms_avg": verify_avg_ms,
+                         "launch_ms_median": verify_ms[len(verify_ms) // 2],
+                         "step_bytes_incl_sampler": alg_bytes + sampler_bytes,
+                         "step_gbs": (alg_bytes + sampler_bytes) / (elapsed_ms / K * 1e-3) / 1e9},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": KE},
+            "gpu_launches": 3 * K,
+            "clocks": clk,
+            "table_build": {"ms": table_ms, "L": cfg.codebook_size, "d": cfg.codebook_dim, "k": cfg.k,
+                            "dtype": cfg.codebook_dtype},
+            "stats": {"mean_accept_len": accept_mean, "tokens_per_step": accept_mean + 1.0, "device_status": dev_status},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            lg_cpu = {k: (None if v is None else v.cpu()) for k, v in bufs[0].items()}
+            line["cpu_baseline"] = cpu_baseline(cfg, parent, lg_cpu)
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

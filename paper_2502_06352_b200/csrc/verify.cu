@@ -280,24 +280,27 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
       P[x - lo] = 0.f;
     }
     __syncthreads();
-    float zsum[1] = {0.f};
+    // one sweep: residual of Eq. 2 in place, its mass, and the drafter mass left without x
+    // (summing what is left avoids the cancellation in 1 - p_cur(x) when p_cur(x) is near 1)
+    float zs[2] = {0.f, 0.f};
     for (int j = tid; j < len; j += kThreads) {
-      float pj = (lo + j == x) ? px : P[j] * ps;        // p_cur before x was dropped
+      const float pr = P[j];
+      float pj = (lo + j == x) ? px : pr * ps;          // p_cur before x was dropped
       float r = fmaxf(Q[j] * qs - pj, 0.f);
       Q[j] = r;
-      zsum[0] += r;
+      zs[0] += r;
+      zs[1] += pr;
     }
-    cluster_reduce<1, false>(c, zsum);
-    if (zsum[0] > 0.f) {
-      qs = 1.f / zsum[0];
+    cluster_reduce<2, false>(c, zs);
+    if (zs[0] > 0.f) {
+      qs = 1.f / zs[0];
     } else {
       // q~ <= p_cur everywhere: both sum to one, so q~ equals p_cur; keep it as the target
       for (int j = tid; j < len; j += kThreads) Q[j] = (lo + j == x) ? px : P[j] * ps;
       qs = 1.f;
       cluster_sync();
     }
-    const float w = 1.f - px;
-    if (w > 0.f) ps = ps / w;
+    ps = zs[1] > 0.f ? 1.f / zs[1] : 0.f;
   }
 
   // ---- no child accepted (or leaf): draw node_token from q_cur by inverse CDF in token order

@@ -54,7 +54,8 @@ def _compare(case, gum, gtok, gprob):
                 ties += 1
                 continue
             assert np.allclose(gprob[b, kids[n]], wp, atol=1e-5)
-            assert len(set(got)) == len(got)
+            real = [t for t in got if t >= 0]
+            assert len(set(real)) == len(real)
     return ties
 
 
