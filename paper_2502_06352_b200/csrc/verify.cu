@@ -8,7 +8,7 @@
 //
 // Distributions are stored unnormalised: q_cur[j] = Q[j] * qs, p_cur[j] = P[j] * ps with the
 // scalars qs, ps held in registers, so a renormalisation never rewrites a row.
-#include "rowops.cuh"
+#include "rowregs.cuh"
 
 namespace lantern {
 
@@ -30,9 +30,11 @@ struct VerifyArgs {
 };
 
 constexpr int kMiscInts = 16;
+constexpr int kCandInts = 40;
 // fixed part of the dynamic shared memory behind the two row slices
-constexpr int kFixedSmemBytes = 2 * 2 * 256 * 4 + kWarps * 4 * 4 + 8 * 4 + kMaxCluster * 4 * 4 + 4 * 4 +
-                                kMiscInts * 4 + 16;
+constexpr int kTopkBytes = 2 * 256 * 4 + 2 * kCandLocal * 4 + 2 * kCandTotal * 4;
+constexpr int kFixedSmemBytes = kTopkBytes + kWarps * 4 * 4 + 8 * 4 + kMaxCluster * 4 * 4 + 4 * 4 +
+                                kCandInts * 4 + kMiscInts * 4 + 16;
 
 __device__ __forceinline__ void flag(int32_t* status, int bit) {
   if (status) atomicOr(status, bit);
@@ -52,18 +54,27 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t phase)
   return false;
 }
 
-template <typename T, bool CFG>
-__global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs a) {
+// E = row entries per thread; the CTA's slice holds SL = 256 * E entries.
+template <typename T, bool CFG, int E>
+__global__ void __launch_bounds__(kThreads, (E >= 16) ? 2 : 3) verify_nodes_kernel(const VerifyArgs a) {
+  constexpr int VN = Vec<T>::N;
+  constexpr int SL = kThreads * E;
+  constexpr int NV4 = E / 4;                 // float4 per thread in a shared-memory sweep
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* Q = reinterpret_cast<float*>(smem_raw);
-  float* P = Q + a.SL;
+  float* P = Q + SL;
+  TopkSmem tk;
+  tk.bins = reinterpret_cast<uint32_t*>(P + SL);
+  tk.candl = reinterpret_cast<float*>(tk.bins + 2 * 256);
+  tk.all = tk.candl + 2 * kCandLocal;
   ClusterCtx c;
-  c.hist = reinterpret_cast<uint32_t*>(P + a.SL);
-  c.red = reinterpret_cast<float*>(c.hist + 2 * 2 * 256);
+  c.hist = reinterpret_cast<uint32_t*>(tk.all);          // radix fallback only
+  c.red = tk.all + 2 * kCandTotal;
   c.xch = c.red + kWarps * 4;
   c.gath = c.xch + 8;
   c.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
-  int* misc = c.sel + 4;
+  tk.candn = c.sel + 4;
+  int* misc = tk.candn + kCandInts;
   uint64_t* mbar = reinterpret_cast<uint64_t*>(misc + kMiscInts);
   int* nbr_s = reinterpret_cast<int*>(mbar + 2);
   c.rank = cluster_ctarank();
@@ -76,10 +87,8 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
   const int b = idx % a.B;
   const int n = a.order[idx / a.B];
   const int fc = a.first_child[n], nc = a.n_child[n];
-  const int SL = a.SL;
   const int lo = c.rank * SL;
   const int len = max(0, min(a.V - lo, SL));
-  const int len4 = (len + 3) & ~3;
   const long long row_off = static_cast<long long>(b) * a.seq_stride + static_cast<long long>(n) * a.row_stride;
   const int32_t* tok_b = a.tokens + static_cast<long long>(b) * a.N;
   const long long out_b = static_cast<long long>(b) * a.N;
@@ -93,7 +102,6 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
     if (tid == 0) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar_a) : "memory");
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       uint32_t bytes = 0;
       const uint32_t row_bytes = static_cast<uint32_t>(((a.k + 3) & ~3) * 4);
       for (int ci = 0; ci < nc; ++ci) {
@@ -122,53 +130,60 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
     }
   }
 
-  // ---- read the rows once: z_q -> Q, z_p -> P
-  float mx[2];
-  mx[0] = load_slice<T, CFG>(static_cast<const T*>(a.tc) + row_off,
-                             CFG ? static_cast<const T*>(a.tu) + row_off : nullptr, a.g, a.inv_tau, lo,
-                             len, a.allow_lo, a.allow_hi, Q);
-  mx[1] = -INFINITY;
-  if (nc > 0)
-    mx[1] = load_slice<T, CFG>(static_cast<const T*>(a.dc) + row_off,
-                               CFG ? static_cast<const T*>(a.du) + row_off : nullptr, a.g, a.inv_tau, lo,
-                               len, a.allow_lo, a.allow_hi, P);
+  // ---- read the rows once into registers: z_q, z_p
+  float zq[E], zp[E];
+  load_row_regs<T, CFG, E>(static_cast<const T*>(a.tc) + row_off,
+                           CFG ? static_cast<const T*>(a.tu) + row_off : nullptr, a.g, a.inv_tau, lo, len, zq);
+  if (nc > 0) {
+    load_row_regs<T, CFG, E>(static_cast<const T*>(a.dc) + row_off,
+                             CFG ? static_cast<const T*>(a.du) + row_off : nullptr, a.g, a.inv_tau, lo, len, zp);
+  } else {
+#pragma unroll
+    for (int e = 0; e < E; ++e) zp[e] = -INFINITY;
+  }
+  if (a.allow_lo > 0 || a.allow_hi < a.V) {
+    mask_regs<E, VN>(zq, lo, a.allow_lo, a.allow_hi);
+    mask_regs<E, VN>(zp, lo, a.allow_lo, a.allow_hi);
+  }
+  float mx[2] = {max_regs<E>(zq), max_regs<E>(zp)};
   cluster_reduce<2, true>(c, mx);
   if (mx[0] == -INFINITY || (nc > 0 && mx[1] == -INFINITY)) {
     if (tid == 0 && c.rank == 0) flag(a.status, LANTERN_DEV_EMPTY_ROW);
     if (mx[0] == -INFINITY) mx[0] = 0.f;
-    if (mx[1] == -INFINITY) mx[1] = 0.f;
   }
+  if (mx[1] == -INFINITY) mx[1] = 0.f;
 
   // ---- top-k truncation thresholds (exact)
   float theta[2] = {-INFINITY, -INFINITY};
-  {
-    int kth[2] = {(a.topk_t > 0 && a.topk_t < a.V) ? a.topk_t : 0,
-                  (nc > 0 && a.topk_d > 0 && a.topk_d < a.V) ? a.topk_d : 0};
-    if (kth[0] > 0 || kth[1] > 0) {
+  const int kth[2] = {(a.topk_t > 0 && a.topk_t < a.V) ? a.topk_t : 0,
+                      (nc > 0 && a.topk_d > 0 && a.topk_d < a.V) ? a.topk_d : 0};
+  const bool has_topk = kth[0] > 0 || kth[1] > 0;
+  if (has_topk) {
+    if (!topk_regs<E>(c, tk, zq, zp, mx, kth, theta)) {
+      // too many entries tie around the k-th one: radix select over shared-memory copies
+      store_regs<E, VN>(zq, Q);
+      store_regs<E, VN>(zp, P);
+      __syncthreads();
       float* const rows[2] = {Q, P};
-      cluster_topk_threshold<2>(c, rows, len, kth, theta);
+      int kk[2] = {kth[0], kth[1]};
+      cluster_topk_threshold<2>(c, rows, len, kk, theta);
+      __syncthreads();
     }
   }
 
-  // ---- softmax numerators in place, row sums
-  float sm[2] = {0.f, 0.f};
-  for (int j = tid; j < len4; j += kThreads) {
-    float z = Q[j];
-    float e = (z >= theta[0]) ? expf(z - mx[0]) : 0.f;
-    Q[j] = e;
-    sm[0] += e;
-  }
-  if (nc > 0) {
-    for (int j = tid; j < len4; j += kThreads) {
-      float z = P[j];
-      float e = (z >= theta[1]) ? expf(z - mx[1]) : 0.f;
-      P[j] = e;
-      sm[1] += e;
-    }
+  // ---- softmax numerators -> shared memory, row sums
+  float sm[2];
+  if (has_topk) {
+    sm[0] = exp_store_regs<E, VN, true>(zq, mx[0], theta[0], Q);
+    sm[1] = exp_store_regs<E, VN, true>(zp, mx[1], theta[1], P);
+  } else {
+    sm[0] = exp_store_regs<E, VN, false>(zq, mx[0], 0.f, Q);
+    sm[1] = nc > 0 ? exp_store_regs<E, VN, false>(zp, mx[1], 0.f, P) : 0.f;
   }
   cluster_reduce<2, false>(c, sm);     // its cluster barrier also publishes Q and P
-  float qs = sm[0] > 0.f ? 1.f / sm[0] : 0.f;     // q_cur[j] = Q[j] * qs
-  float ps = sm[1] > 0.f ? 1.f / sm[1] : 0.f;     // p_cur[j] = P[j] * ps
+  // q_cur[j] = Q[j] * qs,  p_cur[j] = P[j] / psum
+  float qs = sm[0] > 0.f ? 1.f / sm[0] : 0.f;
+  float psum = sm[1];
 
   // ---- neighbour rows must have landed
   if (bulk_issued) {
@@ -207,11 +222,13 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
     const int code = x - a.code_offset;
     const bool has_code = a.k > 0 && code >= 0 && code < a.n_codes;
     const int* nrow = nbr_s + ci * a.kpad;
+    const float ps = psum > 0.f ? 1.f / psum : 0.f;
     if (warp == 0) {
       // every CTA evaluates the relaxed mass redundantly (same values, same order, same result)
       const uint32_t xr = static_cast<uint32_t>(x) / SL, xo = static_cast<uint32_t>(x) - xr * SL;
       const float qx = dsmem_ld_f32(dsmem_addr(q_base + xo * 4, xr)) * qs;
-      const float px = dsmem_ld_f32(dsmem_addr(p_base + xo * 4, xr)) * ps;
+      const float pxraw = dsmem_ld_f32(dsmem_addr(p_base + xo * 4, xr));
+      const float px = pxraw * ps;
       const float bound = a.lambda * qx;
       float cum = qx;
       int nA = 0;
@@ -252,7 +269,7 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
         misc[0] = (u < thr) ? 1 : 0;
         misc[1] = nA;
         reinterpret_cast<float*>(misc)[2] = m;
-        reinterpret_cast<float*>(misc)[3] = px;
+        reinterpret_cast<float*>(misc)[3] = pxraw;
         if (c.rank == 0) {
           if (a.node_mass) a.node_mass[out_b + child] = m;
           if (a.node_thresh) a.node_thresh[out_b + child] = thr;
@@ -263,7 +280,7 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
     const int acc = misc[0];
     const int nA = misc[1];
     const float m = reinterpret_cast<float*>(misc)[2];
-    const float px = reinterpret_cast<float*>(misc)[3];
+    const float pxraw = reinterpret_cast<float*>(misc)[3];
     if (acc) {
       accepted = child;
       __syncthreads();       // misc is rewritten by the next tested child
@@ -275,36 +292,62 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
       const int t = a.code_offset + nrow[r] - lo;
       if (t >= 0 && t < len) Q[t] = 0.f;
     }
-    if (tid == 0 && x >= lo && x < lo + len) {
-      Q[x - lo] = qs > 0.f ? m / qs : 0.f;
-      P[x - lo] = 0.f;
-    }
+    const int xl = x - lo;                                   // position of x in this slice, if any
+    if (tid == 0 && xl >= 0 && xl < len) Q[xl] = qs > 0.f ? m / qs : 0.f;
     __syncthreads();
-    // one sweep: residual of Eq. 2 in place, its mass, and the drafter mass left without x
-    // (summing what is left avoids the cancellation in 1 - p_cur(x) when p_cur(x) is near 1)
+    // One sweep: Q <- [Q * rho - P]_+ with rho = qs * psum, i.e. the residual of Eq. 2 in the
+    // (unnormalised) units of P; its sum gives the new scale.  The drafter mass left without
+    // x is psum - P[x] unless that cancels badly, in which case it is summed in the sweep.
+    const bool resum = pxraw > 0.5f * psum;
+    const float rho = psum > 0.f ? qs * psum : qs;
+    const int xj4 = (xl >= 0 && xl < len) ? (xl & ~3) : -1;
     float zs[2] = {0.f, 0.f};
-    for (int j = tid; j < len; j += kThreads) {
-      const float pr = P[j];
-      float pj = (lo + j == x) ? px : pr * ps;          // p_cur before x was dropped
-      float r = fmaxf(Q[j] * qs - pj, 0.f);
-      Q[j] = r;
-      zs[0] += r;
-      zs[1] += pr;
+#pragma unroll
+    for (int v = 0; v < NV4; ++v) {
+      const int j = warp * 32 * E + v * 128 + lane * 4;
+      float4 q4 = *reinterpret_cast<const float4*>(Q + j);
+      float4 p4 = *reinterpret_cast<const float4*>(P + j);
+      q4.x = fmaxf(fmaf(q4.x, rho, -p4.x), 0.f);
+      q4.y = fmaxf(fmaf(q4.y, rho, -p4.y), 0.f);
+      q4.z = fmaxf(fmaf(q4.z, rho, -p4.z), 0.f);
+      q4.w = fmaxf(fmaf(q4.w, rho, -p4.w), 0.f);
+      *reinterpret_cast<float4*>(Q + j) = q4;
+      zs[0] += (q4.x + q4.y) + (q4.z + q4.w);
+      if (j == xj4) {                                        // drop x from the drafter
+        P[xl] = 0.f;
+        const int e = xl & 3;
+        if (e == 0) p4.x = 0.f; else if (e == 1) p4.y = 0.f; else if (e == 2) p4.z = 0.f; else p4.w = 0.f;
+      }
+      if (resum) zs[1] += (p4.x + p4.y) + (p4.z + p4.w);
     }
     cluster_reduce<2, false>(c, zs);
+    const float ps_old = ps;
+    psum = resum ? zs[1] : psum - pxraw;
     if (zs[0] > 0.f) {
       qs = 1.f / zs[0];
     } else {
-      // q~ <= p_cur everywhere: both sum to one, so q~ equals p_cur; keep it as the target
-      for (int j = tid; j < len; j += kThreads) Q[j] = (lo + j == x) ? px : P[j] * ps;
-      qs = 1.f;
-      cluster_sync();
+      // q~ <= p_cur everywhere: both sum to one, so q~ equals p_cur (before x was dropped);
+      // keep it as the target
+      float s2[2] = {0.f, 0.f};
+#pragma unroll
+      for (int v = 0; v < NV4; ++v) {
+        const int j = warp * 32 * E + v * 128 + lane * 4;
+        float4 p4 = *reinterpret_cast<const float4*>(P + j);
+        if (j == xj4) {
+          const int e = xl & 3;
+          if (e == 0) p4.x = pxraw; else if (e == 1) p4.y = pxraw; else if (e == 2) p4.z = pxraw; else p4.w = pxraw;
+        }
+        *reinterpret_cast<float4*>(Q + j) = p4;
+        s2[0] += (p4.x + p4.y) + (p4.z + p4.w);
+      }
+      cluster_reduce<2, false>(c, s2);       // leaves the per-warp and per-rank sums of Q in place
+      qs = ps_old;
     }
-    ps = zs[1] > 0.f ? 1.f / zs[1] : 0.f;
   }
 
-  // ---- no child accepted (or leaf): draw node_token from q_cur by inverse CDF in token order
-  int32_t result_token = -1;
+  // ---- no child accepted (or leaf): draw node_token from q_cur by inverse CDF in token order.
+  // The last reduction left the per-warp sums of Q in c.red[w*2] and the per-rank sums in
+  // c.gath[r*2]; the slice and the warp segment that hold the draw follow from those.
   if (accepted < 0) {
     float u;
     if (a.u_res) {
@@ -312,39 +355,16 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
     } else {
       u = uniform_halfopen(philox_stream(a.seed, a.step, static_cast<uint32_t>(out_b + n), kStreamResample, 0).x);
     }
-    // warp w owns [w*wseg, (w+1)*wseg) of the slice, swept 128 elements at a time
-    const int wseg = (((SL + kWarps - 1) / kWarps) + 127) & ~127;
-    const int wlo = warp * wseg, whi = min(len4, wlo + wseg);
-    float run = 0.f;
-    for (int base = wlo; base < whi; base += 128) {
-      const int j = base + lane * 4;
-      float4 v = (j < whi) ? *reinterpret_cast<const float4*>(Q + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-      float s4 = ((v.x + v.y) + v.z) + v.w;
-      float incl = warp_incl_scan(s4, lane);
-      run += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    if (lane == 0) c.red[warp] = run;
-    __syncthreads();
-    if (tid == 0) {
-      float t = 0.f;
-      for (int w = 0; w < kWarps; ++w) t += c.red[w];
-      c.xch[c.parity * 4] = t;
-    }
-    cluster_sync();
-    if (tid < static_cast<int>(c.nrank)) c.gath[tid] = dsmem_ld_f32(dsmem_addr(smem_u32(&c.xch[c.parity * 4]), tid));
-    __syncthreads();
-    c.parity ^= 1;
     float total = 0.f;
-    for (uint32_t r = 0; r < c.nrank; ++r) total += c.gath[r];
+    for (uint32_t r = 0; r < c.nrank; ++r) total += c.gath[r * 2];
     const float target = u * total;
-    // owner CTA: first slice whose cumulative mass exceeds the target
     int owner = -1, last_pos = -1;
-    float E = 0.f, E_owner = 0.f;
+    float Erun = 0.f, E_owner = 0.f;
     for (uint32_t r = 0; r < c.nrank; ++r) {
-      float t = c.gath[r];
+      const float t = c.gath[r * 2];
       if (t > 0.f) last_pos = r;
-      if (owner < 0 && E + t > target) { owner = r; E_owner = E; }
-      E += t;
+      if (owner < 0 && Erun + t > target) { owner = r; E_owner = Erun; }
+      Erun += t;
     }
     bool fallback = false;
     if (owner < 0) { owner = last_pos; fallback = true; }     // rounding pushed the target past the end
@@ -352,7 +372,7 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
       int ow = -1, lastw = -1;
       float Ew = E_owner, Ew_owner = 0.f;
       for (int w = 0; w < kWarps; ++w) {
-        float t = c.red[w];
+        const float t = c.red[w * 2];
         if (t > 0.f) lastw = w;
         if (!fallback && ow < 0 && Ew + t > target) { ow = w; Ew_owner = Ew; }
         Ew += t;
@@ -361,26 +381,27 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
       if (ow < 0) { ow = lastw; wfallback = true; }
       if (warp == ow) {
         int found = -1;
+        const int wlo = warp * 32 * E;
         if (!wfallback) {
           float runw = Ew_owner;
-          for (int base = wlo; base < whi && found < 0; base += 128) {
-            const int j = base + lane * 4;
-            float4 v = (j < whi) ? *reinterpret_cast<const float4*>(Q + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-            float s4 = ((v.x + v.y) + v.z) + v.w;
-            float incl = warp_incl_scan(s4, lane);
+          for (int v = 0; v < NV4 && found < 0; ++v) {
+            const int j = wlo + v * 128 + lane * 4;
+            const float4 q4 = *reinterpret_cast<const float4*>(Q + j);
+            const float s4 = (q4.x + q4.y) + (q4.z + q4.w);
+            const float incl = warp_incl_scan(s4, lane);
             const uint32_t ballot = __ballot_sync(0xffffffffu, runw + incl > target);
             if (ballot) {
               const int src = __ffs(ballot) - 1;
               int cand = -1;
               if (lane == src) {
                 float cc = runw + (incl - s4);
-                const float e[4] = {v.x, v.y, v.z, v.w};
+                const float ev[4] = {q4.x, q4.y, q4.z, q4.w};
                 int lastp = -1;
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                  cc += e[t];
-                  if (e[t] > 0.f) lastp = t;
-                  if (cand < 0 && e[t] > 0.f && cc > target) cand = t;
+                  cc += ev[t];
+                  if (ev[t] > 0.f) lastp = t;
+                  if (cand < 0 && ev[t] > 0.f && cc > target) cand = t;
                 }
                 if (cand < 0) cand = lastp;
                 cand = (cand >= 0) ? j + cand : -1;
@@ -394,14 +415,13 @@ __global__ void __launch_bounds__(kThreads) verify_nodes_kernel(const VerifyArgs
         if (found < 0) {
           // last positive entry of this warp's segment
           int best = -1;
-          for (int j = wlo + lane; j < whi; j += 32)
+          for (int j = wlo + lane; j < wlo + 32 * E; j += 32)
             if (Q[j] > 0.f) best = j;
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
           found = best;
         }
-        if (lane == 0) result_token = found >= 0 ? lo + found : -1;
-        if (lane == 0) a.node_token[out_b + n] = result_token;
+        if (lane == 0) a.node_token[out_b + n] = found >= 0 ? lo + found : -1;
       }
     } else if (owner < 0 && c.rank == 0 && tid == 0) {
       a.node_token[out_b + n] = -1;      // empty distribution
@@ -443,38 +463,42 @@ __global__ void walk_kernel(const int32_t* __restrict__ node_next, const int32_t
 
 static int g_cluster_override = 0;
 
-struct LaunchShape { int cs, sl; size_t smem; };
+struct LaunchShape { int cs, e; size_t smem; };
 
-// Choose how many CTAs share a row: slices of about 4096 entries, more CTAs per row when the
-// launch is too small to fill the GPU.
-static bool choose_shape(int V, int rows, int max_children, int kpad, LaunchShape* out) {
-  auto smem_for = [&](int sl) {
-    return static_cast<size_t>(2) * sl * 4 + kFixedSmemBytes + static_cast<size_t>(max_children) * kpad * 4;
+// Choose E (row entries per thread, slice = 256*E) and the cluster size (CTAs per row).
+// `min_e` is 4 for float32 rows and 8 for bfloat16 rows (one 16-byte vector per thread).
+static bool choose_shape(int V, int rows, int max_children, int kpad, int min_e, LaunchShape* out) {
+  auto smem_for = [&](int e) {
+    return static_cast<size_t>(2) * kThreads * e * 4 + kFixedSmemBytes + static_cast<size_t>(max_children) * kpad * 4;
   };
-  int cs = 1;
+  auto cs_for = [&](int e) { int cs = (V + kThreads * e - 1) / (kThreads * e); return cs > 8 ? (cs > 16 ? 0 : 16) : cs; };
+  int e = 0;
   if (g_cluster_override > 0) {
-    cs = g_cluster_override;
+    for (int cand = min_e; cand <= 16; cand *= 2)
+      if (static_cast<long long>(kThreads) * cand * g_cluster_override >= V) { e = cand; break; }
+    if (e == 0) return false;
+    out->cs = g_cluster_override;
   } else {
-    while (cs < kMaxCluster && (V + cs - 1) / cs > 4096) cs *= 2;
-    while (cs < 8 && rows * cs < 296 && (V + cs - 1) / cs > 1024) cs *= 2;
-  }
-  int sl = (((V + cs - 1) / cs) + 7) & ~7;
-  if (smem_for(sl) > 227 * 1024) {
-    while (cs < kMaxCluster && smem_for(sl) > 227 * 1024) {
-      cs *= 2;
-      sl = (((V + cs - 1) / cs) + 7) & ~7;
+    // largest slice first; smaller slices (more CTAs) when the launch would not fill the GPU
+    for (int cand = 16; cand >= min_e; cand /= 2) {
+      int cs = cs_for(cand);
+      if (cs == 0) continue;
+      e = cand;
+      if (static_cast<long long>(rows) * cs >= 2 * 148 || cand == min_e) break;
+      int cs_next = cs_for(cand / 2);
+      if (cs_next == 0) break;
     }
-    if (smem_for(sl) > 227 * 1024) return false;
+    if (e == 0) return false;
+    out->cs = cs_for(e);
   }
-  out->cs = cs;
-  out->sl = sl;
-  out->smem = smem_for(sl);
-  return true;
+  out->e = e;
+  out->smem = smem_for(e);
+  return out->smem <= 227 * 1024;
 }
 
-template <typename T, bool CFG>
-static cudaError_t launch_verify(const VerifyArgs& a, const LaunchShape& sh, cudaStream_t st) {
-  auto kern = verify_nodes_kernel<T, CFG>;
+template <typename T, bool CFG, int E>
+static cudaError_t launch_verify_e(const VerifyArgs& a, const LaunchShape& sh, cudaStream_t st) {
+  auto kern = verify_nodes_kernel<T, CFG, E>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sh.smem));
   if (e != cudaSuccess) return e;
   if (sh.cs > 8) {
@@ -494,6 +518,16 @@ static cudaError_t launch_verify(const VerifyArgs& a, const LaunchShape& sh, cud
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+template <typename T, bool CFG>
+static cudaError_t launch_verify(const VerifyArgs& a, const LaunchShape& sh, cudaStream_t st) {
+  if (sh.e == 16) return launch_verify_e<T, CFG, 16>(a, sh, st);
+  if (sh.e == 8) return launch_verify_e<T, CFG, 8>(a, sh, st);
+  if constexpr (Vec<T>::N <= 4) {
+    if (sh.e == 4) return launch_verify_e<T, CFG, 4>(a, sh, st);
+  }
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace lantern
@@ -569,8 +603,8 @@ extern "C" lantern_status lantern_verify_tree(
   a.node_next = node_next; a.node_token = node_token; a.node_mass = node_mass; a.node_thresh = node_thresh;
   a.status = device_status;
   LaunchShape sh;
-  if (!choose_shape(V, batch * t->n_nodes, t->max_children, a.kpad, &sh)) return LANTERN_ERR_UNSUPPORTED;
-  a.SL = sh.sl;
+  if (!choose_shape(V, batch * t->n_nodes, t->max_children, a.kpad, dt == LANTERN_F32 ? 4 : 8, &sh)) return LANTERN_ERR_UNSUPPORTED;
+  a.SL = kThreads * sh.e;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = target_uncond != nullptr;
   cudaError_t e;
