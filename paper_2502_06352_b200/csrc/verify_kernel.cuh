@@ -1,0 +1,786 @@
+// Device code of the relaxed tree-verification kernel (Sec. 4; App. A.2 Eq. 1-2; Sec. 2.1).
+//
+// One CTA of 1024 threads owns a slice of SL = 1024*E row entries; a row wider than one slice
+// is split over the CTAs of a thread-block cluster (CTA `rank` owns [rank*SL, rank*SL+SL)).
+// With V <= 16384 a node is one CTA and every reduction is a block reduction; only wider
+// rows pay for cluster barriers and distributed-shared-memory reads.
+//
+// The node's target row (and, if it has children, its drafter row) is read from HBM once with
+// 128-bit streaming loads and post-processed (guidance, temperature, top-k, softmax); the
+// unnormalised distributions stay in shared memory: q_cur[j] = Q[j]*qs, p_cur[j] = P[j]/psum.
+// The sibling loop, the residual updates and the inverse-CDF draw run on chip.
+#pragma once
+
+#include "rowops.cuh"
+
+namespace lantern {
+
+constexpr int VT = 1024;          // threads per CTA
+constexpr int VW = VT / 32;       // warps per CTA
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kBins = 512;        // histogram bins of the top-k locator
+constexpr int kBinBase = (127 - 9) << 5;   // 32 bins per binade of d = max - z, d in [2^-9, 2^7)
+constexpr int kCandLocal = 512;   // top-k candidates one CTA may contribute per row
+constexpr int kCandTotal = 1024;  // and the whole cluster
+
+struct VerifyArgs {
+  const void *tc, *tu, *dc, *du;
+  long long row_stride, seq_stride;
+  const int32_t* tokens;
+  const float *u_acc, *u_res;
+  const int32_t* nbr;
+  int k_table, use_bulk;
+  const int32_t *first_child, *n_child, *order;
+  int B, N, V, kpad;
+  float g, inv_tau, lambda;
+  int topk_t, topk_d, k, code_offset, n_codes, allow_lo, allow_hi;
+  unsigned long long seed, step;
+  int32_t *node_next, *node_token;
+  float *node_mass, *node_thresh;
+  int32_t* status;
+};
+
+constexpr int kMiscInts = 16;
+constexpr int kCntInts = 2 + 2 * kMaxCluster + 2;
+// fixed part of the dynamic shared memory behind the two row slices
+constexpr int kVerifyFixedSmem = 2 * kBins * 4 + 2 * kCandLocal * 4 + 2 * kCandTotal * 4   // top-k
+                                 + 2 * VW * 4 * 4      // red (two buffers)
+                                 + 2 * 4 * 4           // xch
+                                 + kMaxCluster * 4 * 4 // gath
+                                 + 8 * 4 + kCntInts * 4 + kMiscInts * 4 + 16;
+
+struct VCtx {
+  uint32_t rank, nrank;
+  int parity;
+  float* red;      // [2][VW*4]
+  float* xch;      // [2][4]
+  float* gath;     // [kMaxCluster*4] per-rank values of the last reduction
+  float* last_red; // red buffer of the last reduction (per-warp values)
+};
+
+__device__ __forceinline__ void vflag(int32_t* status, int bit) {
+  if (status) atomicOr(status, bit);
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ void csync(const VCtx& c) {       // whole row: block or cluster
+  if (c.nrank > 1) cluster_sync(); else __syncthreads();
+}
+
+// Row-wide sum or max of NV values per thread.  Every thread of the row's CTAs gets the same
+// result (fixed combination order).  The per-warp partials stay in c.last_red[w*NV+i] and the
+// per-rank partials in c.gath[r*NV+i] until the next call.
+template <int NV, bool IS_MAX>
+__device__ __forceinline__ void row_reduce(VCtx& c, float (&v)[NV]) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float* red = c.red + c.parity * (VW * 4);
+#pragma unroll
+  for (int i = 0; i < NV; ++i) v[i] = IS_MAX ? warp_max(v[i]) : warp_sum(v[i]);
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < NV; ++i) red[warp * NV + i] = v[i];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    float t = red[lane * NV + i];               // VW == 32: one partial per lane
+    v[i] = IS_MAX ? warp_max(t) : warp_sum(t);
+  }
+  if (c.nrank > 1) {
+    if (threadIdx.x < NV) c.xch[c.parity * 4 + threadIdx.x] = v[threadIdx.x];
+    cluster_sync();
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      float t = IS_MAX ? -INFINITY : 0.f;
+      if (lane < static_cast<int>(c.nrank)) t = dsmem_ld_f32(dsmem_addr(smem_u32(&c.xch[c.parity * 4 + i]), lane));
+      if (warp == 0 && lane < static_cast<int>(c.nrank)) c.gath[lane * NV + i] = t;
+      v[i] = IS_MAX ? warp_max(t) : warp_sum(t);
+    }
+  } else if (threadIdx.x < NV) {
+    c.gath[threadIdx.x] = v[threadIdx.x];
+  }
+  c.last_red = red;
+  c.parity ^= 1;
+}
+
+// Pre-softmax values of one row slice -> shared memory (entries beyond the row end and
+// outside the allowed token range become -inf).  Returns this thread's maximum.
+template <typename T, bool CFG, int E>
+__device__ __forceinline__ float load_row(const T* __restrict__ cond, const T* __restrict__ uncond, float g,
+                                          float inv_tau, int lo, int len, int allow_lo, int allow_hi,
+                                          bool masked, float* __restrict__ dst) {
+  using VTT = Vec<T>;
+  constexpr int VN = VTT::N, NV = E / VN;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int wb = warp * 32 * E + lane * VN;
+  typename VTT::V cr[NV], ur[NV];
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    const int j = wb + v * 32 * VN;
+    if (j + VN <= len) {
+      cr[v] = __ldcs(reinterpret_cast<const typename VTT::V*>(cond + lo + j));
+      if (CFG) ur[v] = __ldcs(reinterpret_cast<const typename VTT::V*>(uncond + lo + j));
+    }
+  }
+  float mx = -INFINITY;
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    const int j = wb + v * 32 * VN;
+    float zf[VN];
+    if (j + VN <= len) {
+      float cf[VN], uf[VN];
+      VTT::unpack(cr[v], cf);
+      if (CFG) VTT::unpack(ur[v], uf);
+#pragma unroll
+      for (int e = 0; e < VN; ++e) zf[e] = combine<CFG>(cf[e], CFG ? uf[e] : 0.f, g, inv_tau);
+    } else {
+#pragma unroll
+      for (int e = 0; e < VN; ++e) {
+        float val = -INFINITY;
+        if (j + e < len) {
+          const float cc = VTT::widen(cond[lo + j + e]);
+          const float uu = CFG ? VTT::widen(uncond[lo + j + e]) : 0.f;
+          val = combine<CFG>(cc, uu, g, inv_tau);
+        }
+        zf[e] = val;
+      }
+    }
+    if (masked) {
+#pragma unroll
+      for (int e = 0; e < VN; ++e)
+        if (lo + j + e < allow_lo || lo + j + e >= allow_hi) zf[e] = -INFINITY;
+    }
+#pragma unroll
+    for (int e = 0; e < VN; ++e) mx = fmaxf(mx, zf[e]);
+    float4* d4 = reinterpret_cast<float4*>(dst + j);
+#pragma unroll
+    for (int e = 0; e < VN; e += 4) d4[e / 4] = make_float4(zf[e], zf[e + 1], zf[e + 2], zf[e + 3]);
+  }
+  return mx;
+}
+
+// Coarse position of an entry below the row maximum: a monotone function of z.
+__device__ __forceinline__ int dist_bin(float mx, float z) {
+  const float d = mx - z;
+  const int b = static_cast<int>(__float_as_uint(d) >> 18) - kBinBase;
+  return min(max(b, 0), kBins - 1);
+}
+
+struct TopkSmem {
+  uint32_t* bins;   // [2][kBins]
+  float* candl;     // [2][kCandLocal]   (first used as staging of the cluster-wide bins)
+  float* all;       // [2][kCandTotal]
+  int* sel;         // [8]
+  int* cnts;        // [2] local counts, then [2][kMaxCluster] counts of every rank
+};
+
+// Exact top-k thresholds of up to two rows whose pre-softmax values sit in shared memory
+// (row r active iff kth[r] > 0): theta[r] = the kth[r]-th largest entry of the whole row.
+// A histogram over dist_bin locates the bin of the k-th entry; the entries of that bin are
+// gathered from all CTAs of the row and ranked exactly.  If they do not fit, the bin is
+// refined by a radix select on the raw keys restricted to it.
+template <int E>
+__device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, const float* __restrict__ z0,
+                                                const float* __restrict__ z1, const float (&mx)[2],
+                                                const int (&kth)[2], float (&theta)[2]) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NV4 = E / 4;
+  for (int i = tid; i < 2 * kBins; i += VT) s.bins[i] = 0;
+  if (tid < 2) s.cnts[tid] = 0;
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (kth[r] <= 0) continue;
+    const float* z = r ? z1 : z0;
+#pragma unroll
+    for (int v = 0; v < NV4; ++v) {
+      const float4 q = *reinterpret_cast<const float4*>(z + warp * 32 * E + v * 128 + lane * 4);
+      atomicAdd(&s.bins[r * kBins + dist_bin(mx[r], q.x)], 1u);
+      atomicAdd(&s.bins[r * kBins + dist_bin(mx[r], q.y)], 1u);
+      atomicAdd(&s.bins[r * kBins + dist_bin(mx[r], q.z)], 1u);
+      atomicAdd(&s.bins[r * kBins + dist_bin(mx[r], q.w)], 1u);
+    }
+  }
+  csync(c);
+  uint32_t* gb = reinterpret_cast<uint32_t*>(s.candl);     // [2][kBins] bins of the whole row
+  if (c.nrank > 1) {
+    for (int i = tid; i < 2 * kBins; i += VT) {
+      uint32_t g = 0;
+      if (kth[i / kBins] > 0) {
+        const uint32_t addr = smem_u32(&s.bins[i]);
+        for (uint32_t q = 0; q < c.nrank; ++q) g += dsmem_ld_u32(dsmem_addr(addr, q));
+      }
+      gb[i] = g;
+    }
+    __syncthreads();
+  } else {
+    gb = s.bins;
+  }
+  if (warp < 2 && kth[warp & 1] > 0) {
+    // smallest bin whose cumulative count reaches k: lane l covers bins 16l .. 16l+15
+    const int r = warp;
+    constexpr int PER = kBins / 32;
+    uint32_t sum = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) sum += gb[r * kBins + PER * lane + i];
+    uint32_t incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    const uint32_t excl = incl - sum, need = static_cast<uint32_t>(kth[r]);
+    if (excl < need && need <= incl) {
+      uint32_t run = excl;
+      for (int i = 0; i < PER; ++i) {
+        const uint32_t cnt = gb[r * kBins + PER * lane + i];
+        if (run < need && need <= run + cnt) {
+          s.sel[r * 2 + 0] = PER * lane + i;
+          s.sel[r * 2 + 1] = static_cast<int>(need - run);
+        }
+        run += cnt;
+      }
+    }
+  }
+  __syncthreads();           // also: the staged bins have been consumed, candl may be overwritten
+  int bstar[2], krem[2];
+#pragma unroll
+  for (int r = 0; r < 2; ++r) { bstar[r] = kth[r] > 0 ? s.sel[r * 2] : -1; krem[r] = kth[r] > 0 ? s.sel[r * 2 + 1] : 0; }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (kth[r] <= 0) continue;
+    const float* z = r ? z1 : z0;
+#pragma unroll
+    for (int v = 0; v < NV4; ++v) {
+      const float4 q = *reinterpret_cast<const float4*>(z + warp * 32 * E + v * 128 + lane * 4);
+      const float ev[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (dist_bin(mx[r], ev[e]) == bstar[r]) {
+          const int pos = atomicAdd(&s.cnts[r], 1);
+          if (pos < kCandLocal) s.candl[r * kCandLocal + pos] = ev[e];
+        }
+    }
+  }
+  csync(c);
+  // candidate counts of every rank
+  int* rc = s.cnts + 2;
+  if (tid < 2 * static_cast<int>(c.nrank)) {
+    const int r = tid / c.nrank, q = tid % c.nrank;
+    rc[r * kMaxCluster + q] = static_cast<int>(dsmem_ld_u32(dsmem_addr(smem_u32(&s.cnts[r]), q)));
+  }
+  __syncthreads();
+  int total[2] = {0, 0};
+  bool fits[2] = {true, true};
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (kth[r] <= 0) continue;
+    for (uint32_t q = 0; q < c.nrank; ++q) {
+      const int n = rc[r * kMaxCluster + q];
+      if (n > kCandLocal) fits[r] = false;
+      total[r] += n;
+    }
+    if (total[r] > kCandTotal) fits[r] = false;
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (kth[r] <= 0 || !fits[r]) continue;
+    int off = 0;
+    for (uint32_t q = 0; q < c.nrank; ++q) {
+      const int n = rc[r * kMaxCluster + q];
+      const uint32_t base = dsmem_addr(smem_u32(&s.candl[r * kCandLocal]), q);
+      for (int i = tid; i < n; i += VT) s.all[r * kCandTotal + off + i] = dsmem_ld_f32(base + 4u * i);
+      off += n;
+    }
+  }
+  __syncthreads();
+  // exact rank by counting: theta = v with  #(> v) < k' <= #(>= v)
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (kth[r] <= 0 || !fits[r]) continue;
+    const float* al = s.all + r * kCandTotal;
+    for (int i = tid; i < total[r]; i += VT) {
+      const float v = al[i];
+      int gt = 0, ge = 0;
+      for (int t = 0; t < total[r]; ++t) {
+        const float w = al[t];
+        gt += (w > v);
+        ge += (w >= v);
+      }
+      if (gt < krem[r] && krem[r] <= ge) reinterpret_cast<float*>(s.sel)[4 + r] = v;
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 2; ++r) theta[r] = (kth[r] > 0 && fits[r]) ? reinterpret_cast<float*>(s.sel)[4 + r] : -INFINITY;
+  // ---- refinement when a bin holds too many entries: radix select (4 x 8 bits) on the
+  // monotone key, restricted to that bin, rank krem within it
+  for (int r = 0; r < 2; ++r) {
+    if (kth[r] <= 0 || fits[r]) continue;        // same decision in every CTA of the row
+    const float* z = r ? z1 : z0;
+    uint32_t prefix = 0;
+    int remaining = krem[r];
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      __syncthreads();
+      if (tid < 256) s.bins[tid] = 0;
+      __syncthreads();
+      for (int v = 0; v < NV4; ++v) {
+        const float4 q = *reinterpret_cast<const float4*>(z + warp * 32 * E + v * 128 + lane * 4);
+        const float ev[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (dist_bin(mx[r], ev[e]) != bstar[r]) continue;
+          const uint32_t key = float_key(ev[e]);
+          if (pass == 0 || (key >> (shift + 8)) == prefix) atomicAdd(&s.bins[(key >> shift) & 255u], 1u);
+        }
+      }
+      csync(c);
+      uint32_t g = 0;
+      if (tid < 256) {
+        const uint32_t addr = smem_u32(&s.bins[tid]);
+        for (uint32_t q = 0; q < c.nrank; ++q) g += dsmem_ld_u32(dsmem_addr(addr, q));
+      }
+      csync(c);               // every CTA has read the bins before anyone clears them again
+      if (tid < 256) s.bins[256 + tid] = g;
+      __syncthreads();
+      if (tid == 0) {
+        uint32_t run = 0;
+        for (int dgt = 255; dgt >= 0; --dgt) {
+          const uint32_t cnt = s.bins[256 + dgt];
+          if (run < static_cast<uint32_t>(remaining) && static_cast<uint32_t>(remaining) <= run + cnt) {
+            s.sel[6] = dgt;
+            s.sel[7] = remaining - static_cast<int>(run);
+            break;
+          }
+          run += cnt;
+        }
+      }
+      __syncthreads();
+      prefix = (prefix << 8) | static_cast<uint32_t>(s.sel[6]);
+      remaining = s.sel[7];
+    }
+    theta[r] = key_float(prefix);
+  }
+  __syncthreads();
+}
+
+
+// ---- bounded wait on an mbarrier phase; false when the limit was reached
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t phase) {
+  for (int it = 0; it < (1 << 22); ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(mbar), "r"(phase) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+// E = row entries per thread; the CTA's slice holds SL = 1024 * E entries.
+template <typename T, bool CFG, int E>
+__global__ void __launch_bounds__(VT, 1) verify_nodes_kernel(const VerifyArgs a) {
+  constexpr int SL = VT * E;
+  constexpr int NV4 = E / 4;                 // float4 per thread in a shared-memory sweep
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* Q = reinterpret_cast<float*>(smem_raw);
+  float* P = Q + SL;
+  TopkSmem tk;
+  tk.bins = reinterpret_cast<uint32_t*>(P + SL);
+  tk.candl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
+  tk.all = tk.candl + 2 * kCandLocal;
+  VCtx c;
+  c.red = tk.all + 2 * kCandTotal;
+  c.xch = c.red + 2 * VW * 4;
+  c.gath = c.xch + 8;
+  tk.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
+  tk.cnts = tk.sel + 8;
+  int* misc = tk.cnts + kCntInts;
+  uint64_t* mbar = reinterpret_cast<uint64_t*>(misc + kMiscInts);
+  int* nbr_s = reinterpret_cast<int*>(mbar + 2);
+  c.rank = cluster_ctarank();
+  c.nrank = cluster_nctarank();
+  c.parity = 0;
+  c.last_red = c.red;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int idx = blockIdx.x / c.nrank;
+  const int b = idx % a.B;
+  const int n = a.order[idx / a.B];
+  const int fc = a.first_child[n], nc = a.n_child[n];
+  const int lo = c.rank * SL;
+  const int len = max(0, min(a.V - lo, SL));
+  const long long row_off = static_cast<long long>(b) * a.seq_stride + static_cast<long long>(n) * a.row_stride;
+  const int32_t* tok_b = a.tokens + static_cast<long long>(b) * a.N;
+  const long long out_b = static_cast<long long>(b) * a.N;
+  const uint32_t q_base = smem_u32(Q), p_base = smem_u32(P);
+  const bool single = c.nrank == 1;
+
+  // ---- stage the children's neighbour rows (bulk async copy when rows are 16-byte aligned)
+  const bool want_nbr = nc > 0 && a.k > 0;
+  const uint32_t mbar_a = smem_u32(mbar);
+  bool bulk_issued = false;
+  if (want_nbr && a.use_bulk) {
+    if (tid == 0) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar_a) : "memory");
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      uint32_t bytes = 0;
+      const uint32_t row_bytes = static_cast<uint32_t>(((a.k + 3) & ~3) * 4);
+      for (int ci = 0; ci < nc; ++ci) {
+        int code = tok_b[fc + ci] - a.code_offset;
+        if (code >= 0 && code < a.n_codes) bytes += row_bytes;
+      }
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar_a), "r"(bytes) : "memory");
+      for (int ci = 0; ci < nc; ++ci) {
+        int code = tok_b[fc + ci] - a.code_offset;
+        if (code >= 0 && code < a.n_codes) {
+          const int32_t* src = a.nbr + static_cast<long long>(code) * a.k_table;
+          uint32_t dst = smem_u32(nbr_s + ci * a.kpad);
+          asm volatile(
+              "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+              ::"r"(dst), "l"(src), "r"(row_bytes), "r"(mbar_a) : "memory");
+        }
+      }
+    }
+    bulk_issued = true;
+  } else if (want_nbr) {
+    for (int ci = 0; ci < nc; ++ci) {
+      int code = tok_b[fc + ci] - a.code_offset;
+      if (code >= 0 && code < a.n_codes)
+        for (int r = tid; r < a.k; r += VT)
+          nbr_s[ci * a.kpad + r] = a.nbr[static_cast<long long>(code) * a.k_table + r];
+    }
+  }
+
+  // ---- read the rows once: z_q -> Q, z_p -> P
+  const bool masked = a.allow_lo > 0 || a.allow_hi < a.V;
+  float mx[2];
+  mx[0] = load_row<T, CFG, E>(static_cast<const T*>(a.tc) + row_off,
+                              CFG ? static_cast<const T*>(a.tu) + row_off : nullptr, a.g, a.inv_tau, lo, len,
+                              a.allow_lo, a.allow_hi, masked, Q);
+  mx[1] = -INFINITY;
+  if (nc > 0)
+    mx[1] = load_row<T, CFG, E>(static_cast<const T*>(a.dc) + row_off,
+                                CFG ? static_cast<const T*>(a.du) + row_off : nullptr, a.g, a.inv_tau, lo, len,
+                                a.allow_lo, a.allow_hi, masked, P);
+  row_reduce<2, true>(c, mx);
+  if (mx[0] == -INFINITY || (nc > 0 && mx[1] == -INFINITY)) {
+    if (tid == 0 && c.rank == 0) vflag(a.status, LANTERN_DEV_EMPTY_ROW);
+    if (mx[0] == -INFINITY) mx[0] = 0.f;
+  }
+  if (mx[1] == -INFINITY) mx[1] = 0.f;
+
+  // ---- top-k truncation thresholds (exact)
+  float theta[2] = {-INFINITY, -INFINITY};
+  const int kth[2] = {(a.topk_t > 0 && a.topk_t < a.V) ? a.topk_t : 0,
+                      (nc > 0 && a.topk_d > 0 && a.topk_d < a.V) ? a.topk_d : 0};
+  const bool has_topk = kth[0] > 0 || kth[1] > 0;
+  if (has_topk) topk_thresholds<E>(c, tk, Q, P, mx, kth, theta);
+
+  // ---- softmax numerators 2^((z - max) log2 e) in place, row sums
+  float sm[2] = {0.f, 0.f};
+  {
+    const float c0 = -mx[0] * kLog2e, c1 = -mx[1] * kLog2e;
+#pragma unroll
+    for (int v = 0; v < NV4; ++v) {
+      const int j = warp * 32 * E + v * 128 + lane * 4;
+      float4 q4 = *reinterpret_cast<const float4*>(Q + j);
+      float ev[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float x = ex2_approx(fmaf(ev[e], kLog2e, c0));
+        if (has_topk) x = (ev[e] >= theta[0]) ? x : 0.f;
+        ev[e] = x;
+      }
+      *reinterpret_cast<float4*>(Q + j) = make_float4(ev[0], ev[1], ev[2], ev[3]);
+      sm[0] += (ev[0] + ev[1]) + (ev[2] + ev[3]);
+    }
+    if (nc > 0) {
+#pragma unroll
+      for (int v = 0; v < NV4; ++v) {
+        const int j = warp * 32 * E + v * 128 + lane * 4;
+        float4 p4 = *reinterpret_cast<const float4*>(P + j);
+        float ev[4] = {p4.x, p4.y, p4.z, p4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float x = ex2_approx(fmaf(ev[e], kLog2e, c1));
+          if (has_topk) x = (ev[e] >= theta[1]) ? x : 0.f;
+          ev[e] = x;
+        }
+        *reinterpret_cast<float4*>(P + j) = make_float4(ev[0], ev[1], ev[2], ev[3]);
+        sm[1] += (ev[0] + ev[1]) + (ev[2] + ev[3]);
+      }
+    }
+  }
+  row_reduce<2, false>(c, sm);     // its barrier also publishes Q and P
+  float qs = sm[0] > 0.f ? 1.f / sm[0] : 0.f;
+  float psum = sm[1];
+
+  // ---- neighbour rows must have landed
+  if (bulk_issued) {
+    bool ok = mbar_wait_bounded(mbar_a, 0);
+    if (!__syncthreads_and(ok)) {
+      if (tid == 0) vflag(a.status, LANTERN_DEV_TIMEOUT);
+      for (int ci = 0; ci < nc; ++ci) {
+        int code = tok_b[fc + ci] - a.code_offset;
+        if (code >= 0 && code < a.n_codes)
+          for (int r = tid; r < a.k; r += VT)
+            nbr_s[ci * a.kpad + r] = a.nbr[static_cast<long long>(code) * a.k_table + r];
+      }
+    }
+  }
+  __syncthreads();
+
+  if (n == 0 && c.rank == 0 && tid == 0) {
+    if (a.node_mass) a.node_mass[out_b] = -1.f;
+    if (a.node_thresh) a.node_thresh[out_b] = -1.f;
+  }
+
+  // value of Q / P at a token of the row, wherever its slice lives
+  auto row_at = [&](const float* loc, uint32_t base, int t) -> float {
+    if (single) return loc[t];
+    const uint32_t tr = static_cast<uint32_t>(t) / SL, to = static_cast<uint32_t>(t) - tr * SL;
+    return dsmem_ld_f32(dsmem_addr(base + to * 4, tr));
+  };
+
+  // ---- sibling loop (Sec. 4; Eq. 1-2)
+  int accepted = -1;
+  for (int ci = 0; ci < nc; ++ci) {
+    const int child = fc + ci;
+    const int x = tok_b[child];
+    bool skip = accepted >= 0 || x < 0 || x >= a.V;
+    if (skip) {
+      if (accepted < 0 && x >= a.V && tid == 0 && c.rank == 0) vflag(a.status, LANTERN_DEV_BAD_INDEX);
+      if (c.rank == 0 && tid == 0) {
+        if (a.node_mass) a.node_mass[out_b + child] = -1.f;
+        if (a.node_thresh) a.node_thresh[out_b + child] = -1.f;
+      }
+      continue;
+    }
+    const int code = x - a.code_offset;
+    const bool has_code = a.k > 0 && code >= 0 && code < a.n_codes;
+    const int* nrow = nbr_s + ci * a.kpad;
+    const float ps = psum > 0.f ? 1.f / psum : 0.f;
+    if (warp == 0) {
+      // every CTA evaluates the relaxed mass redundantly (same values, same order, same result)
+      const float qx = row_at(Q, q_base, x) * qs;
+      const float pxraw = row_at(P, p_base, x);
+      const float px = pxraw * ps;
+      const float bound = a.lambda * qx;
+      float cum = qx;
+      int nA = 0;
+      bool bad = false, open = has_code;
+      for (int base8 = 0; base8 < a.k && open; base8 += 256) {
+        float qa[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {           // all loads of this lane first, then the scans
+          const int r = base8 + i * 32 + lane;
+          qa[i] = 0.f;
+          if (r < a.k) {
+            const int t = a.code_offset + nrow[r];
+            if (t >= 0 && t < a.V) qa[i] = row_at(Q, q_base, t) * qs; else bad = true;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (!open) break;
+          const int r = base8 + i * 32 + lane;
+          if (base8 + i * 32 >= a.k) { open = false; break; }
+          const float incl = warp_incl_scan(qa[i], lane);
+          const bool ok = r < a.k && (cum + incl < bound);
+          const uint32_t ballot = __ballot_sync(0xffffffffu, ok);
+          const int ntake = __ffs(~ballot) - 1;          // leading accepted entries; -1 when all 32
+          const int take = ntake < 0 ? 32 : ntake;
+          if (take > 0) cum += __shfl_sync(0xffffffffu, incl, take - 1);
+          nA += take;
+          if (take < 32) open = false;
+        }
+      }
+      if (__any_sync(0xffffffffu, bad) && lane == 0 && c.rank == 0) vflag(a.status, LANTERN_DEV_BAD_INDEX);
+      const float m = cum;
+      const float thr = px > 0.f ? fminf(1.f, m / px) : (m > 0.f ? 1.f : 0.f);
+      float u;
+      if (a.u_acc) {
+        u = a.u_acc[out_b + child];
+      } else {
+        u = uniform_halfopen(philox_stream(a.seed, a.step, static_cast<uint32_t>(out_b + child), kStreamAccept, 0).x);
+      }
+      if (lane == 0) {
+        misc[0] = (u < thr) ? 1 : 0;
+        misc[1] = nA;
+        reinterpret_cast<float*>(misc)[2] = m;
+        reinterpret_cast<float*>(misc)[3] = pxraw;
+        if (c.rank == 0) {
+          if (a.node_mass) a.node_mass[out_b + child] = m;
+          if (a.node_thresh) a.node_thresh[out_b + child] = thr;
+        }
+      }
+    }
+    __syncthreads();
+    const int acc = misc[0];
+    const int nA = misc[1];
+    const float m = reinterpret_cast<float*>(misc)[2];
+    const float pxraw = reinterpret_cast<float*>(misc)[3];
+    if (acc) {
+      accepted = child;
+      __syncthreads();       // misc is rewritten by the next tested child
+      continue;
+    }
+    // ---- rejection: q~ (mass of A moved onto x), residual, drafter without x
+    if (!single) cluster_sync();     // every CTA has finished reading q_cur / p_cur of this round
+    for (int r = tid; r < nA; r += VT) {
+      const int t = a.code_offset + nrow[r] - lo;
+      if (t >= 0 && t < len) Q[t] = 0.f;
+    }
+    const int xl = x - lo;                                   // position of x in this slice, if any
+    if (tid == 0 && xl >= 0 && xl < len) Q[xl] = qs > 0.f ? m / qs : 0.f;
+    __syncthreads();
+    // One sweep: Q <- [Q * rho - P]_+ with rho = qs * psum, i.e. the residual of Eq. 2 in the
+    // (unnormalised) units of P; its sum gives the new scale.  The drafter mass left without
+    // x is psum - P[x] unless that cancels badly, in which case it is summed in the sweep.
+    const bool resum = pxraw > 0.5f * psum;
+    const float rho = psum > 0.f ? qs * psum : qs;
+    const int xj4 = (xl >= 0 && xl < len) ? (xl & ~3) : -1;
+    float zs[2] = {0.f, 0.f};
+#pragma unroll
+    for (int v = 0; v < NV4; ++v) {
+      const int j = warp * 32 * E + v * 128 + lane * 4;
+      float4 q4 = *reinterpret_cast<const float4*>(Q + j);
+      float4 p4 = *reinterpret_cast<const float4*>(P + j);
+      q4.x = fmaxf(fmaf(q4.x, rho, -p4.x), 0.f);
+      q4.y = fmaxf(fmaf(q4.y, rho, -p4.y), 0.f);
+      q4.z = fmaxf(fmaf(q4.z, rho, -p4.z), 0.f);
+      q4.w = fmaxf(fmaf(q4.w, rho, -p4.w), 0.f);
+      *reinterpret_cast<float4*>(Q + j) = q4;
+      zs[0] += (q4.x + q4.y) + (q4.z + q4.w);
+      if (j == xj4) {                                        // drop x from the drafter
+        P[xl] = 0.f;
+        const int e = xl & 3;
+        if (e == 0) p4.x = 0.f; else if (e == 1) p4.y = 0.f; else if (e == 2) p4.z = 0.f; else p4.w = 0.f;
+      }
+      if (resum) zs[1] += (p4.x + p4.y) + (p4.z + p4.w);
+    }
+    row_reduce<2, false>(c, zs);
+    const float ps_old = ps;
+    psum = resum ? zs[1] : psum - pxraw;
+    if (zs[0] > 0.f) {
+      qs = 1.f / zs[0];
+    } else {
+      // q~ <= p_cur everywhere: both sum to one, so q~ equals p_cur (before x was dropped);
+      // keep it as the target
+      float s2[2] = {0.f, 0.f};
+#pragma unroll
+      for (int v = 0; v < NV4; ++v) {
+        const int j = warp * 32 * E + v * 128 + lane * 4;
+        float4 p4 = *reinterpret_cast<const float4*>(P + j);
+        if (j == xj4) {
+          const int e = xl & 3;
+          if (e == 0) p4.x = pxraw; else if (e == 1) p4.y = pxraw; else if (e == 2) p4.z = pxraw; else p4.w = pxraw;
+        }
+        *reinterpret_cast<float4*>(Q + j) = p4;
+        s2[0] += (p4.x + p4.y) + (p4.z + p4.w);
+      }
+      row_reduce<2, false>(c, s2);       // leaves the per-warp and per-rank sums of Q in place
+      qs = ps_old;
+    }
+  }
+
+  // ---- no child accepted (or leaf): draw node_token from q_cur by inverse CDF in token order.
+  // The last reduction left the per-warp sums of Q in c.last_red[w*2] and the per-rank sums in
+  // c.gath[r*2]; the slice and the warp segment that hold the draw follow from those.
+  if (accepted < 0) {
+    float u;
+    if (a.u_res) {
+      u = a.u_res[out_b + n];
+    } else {
+      u = uniform_halfopen(philox_stream(a.seed, a.step, static_cast<uint32_t>(out_b + n), kStreamResample, 0).x);
+    }
+    __syncthreads();                      // c.gath was written by warp 0
+    float total = 0.f;
+    for (uint32_t r = 0; r < c.nrank; ++r) total += c.gath[r * 2];
+    const float target = u * total;
+    int owner = -1, last_pos = -1;
+    float Erun = 0.f, E_owner = 0.f;
+    for (uint32_t r = 0; r < c.nrank; ++r) {
+      const float t = c.gath[r * 2];
+      if (t > 0.f) last_pos = r;
+      if (owner < 0 && Erun + t > target) { owner = r; E_owner = Erun; }
+      Erun += t;
+    }
+    bool fallback = false;
+    if (owner < 0) { owner = last_pos; fallback = true; }     // rounding pushed the target past the end
+    if (owner == static_cast<int>(c.rank)) {
+      int ow = -1, lastw = -1;
+      float Ew = E_owner, Ew_owner = 0.f;
+      for (int w = 0; w < VW; ++w) {
+        const float t = c.last_red[w * 2];
+        if (t > 0.f) lastw = w;
+        if (!fallback && ow < 0 && Ew + t > target) { ow = w; Ew_owner = Ew; }
+        Ew += t;
+      }
+      bool wfallback = fallback;
+      if (ow < 0) { ow = lastw; wfallback = true; }
+      if (warp == ow) {
+        int found = -1;
+        const int wlo = warp * 32 * E;
+        if (!wfallback) {
+          float runw = Ew_owner;
+          for (int v = 0; v < NV4 && found < 0; ++v) {
+            const int j = wlo + v * 128 + lane * 4;
+            const float4 q4 = *reinterpret_cast<const float4*>(Q + j);
+            const float s4 = (q4.x + q4.y) + (q4.z + q4.w);
+            const float incl = warp_incl_scan(s4, lane);
+            const uint32_t ballot = __ballot_sync(0xffffffffu, runw + incl > target);
+            if (ballot) {
+              const int src = __ffs(ballot) - 1;
+              int cand = -1;
+              if (lane == src) {
+                float cc = runw + (incl - s4);
+                const float ev[4] = {q4.x, q4.y, q4.z, q4.w};
+                int lastp = -1;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                  cc += ev[t];
+                  if (ev[t] > 0.f) lastp = t;
+                  if (cand < 0 && ev[t] > 0.f && cc > target) cand = t;
+                }
+                if (cand < 0) cand = lastp;
+                cand = (cand >= 0) ? j + cand : -1;
+              }
+              found = __shfl_sync(0xffffffffu, cand, src);
+              if (found < 0) found = -2;       // numerically empty quad: use the fallback below
+            }
+            runw += __shfl_sync(0xffffffffu, incl, 31);
+          }
+        }
+        if (found < 0) {
+          // last positive entry of this warp's segment
+          int best = -1;
+          for (int j = wlo + lane; j < wlo + 32 * E; j += 32)
+            if (Q[j] > 0.f) best = j;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+          found = best;
+        }
+        if (lane == 0) a.node_token[out_b + n] = found >= 0 ? lo + found : -1;
+      }
+    } else if (owner < 0 && c.rank == 0 && tid == 0) {
+      a.node_token[out_b + n] = -1;      // empty distribution
+      vflag(a.status, LANTERN_DEV_EMPTY_ROW);
+    }
+  } else if (c.rank == 0 && tid == 0) {
+    a.node_token[out_b + n] = -1;
+  }
+  if (c.rank == 0 && tid == 0) a.node_next[out_b + n] = accepted;
+  if (!single) cluster_sync();    // peers may still be reading this CTA's shared memory
+}
+
+}  // namespace lantern
