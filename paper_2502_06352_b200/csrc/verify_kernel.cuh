@@ -18,7 +18,7 @@ namespace lantern {
 constexpr int VT = 1024;          // threads per CTA
 constexpr int VW = VT / 32;       // warps per CTA
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kBins = 512;        // histogram bins of the top-k locator
+constexpr int kBins = 512;        // histogram bins of the top-k locator (2 * kBins == VT)
 constexpr int kBinBase = (127 - 9) << 5;   // 32 bins per binade of d = max - z, d in [2^-9, 2^7)
 constexpr int kCandLocal = 512;   // top-k candidates one CTA may contribute per row
 constexpr int kCandTotal = 1024;  // and the whole cluster
@@ -43,7 +43,7 @@ struct VerifyArgs {
 constexpr int kMiscInts = 16;
 constexpr int kCntInts = 2 + 2 * kMaxCluster + 2;
 // fixed part of the dynamic shared memory behind the two row slices
-constexpr int kVerifyFixedSmem = 2 * kBins * 4 + 2 * kCandLocal * 4 + 2 * kCandTotal * 4   // top-k
+constexpr int kVerifyFixedSmem = 2 * kBins * 4 + 4 * kCandLocal * 4 + 2 * kCandTotal * 4 + 2 * VW * 4   // top-k
                                  + 2 * VW * 4 * 4      // red (two buffers)
                                  + 2 * 4 * 4           // xch
                                  + kMaxCluster * 4 * 4 // gath
@@ -173,8 +173,10 @@ __device__ __forceinline__ int dist_bin(float mx, float z) {
 
 struct TopkSmem {
   uint32_t* bins;   // [2][kBins]
-  float* candl;     // [2][kCandLocal]   (first used as staging of the cluster-wide bins)
+  float* wl;        // [2][VW][kCandLocal/VW] per-warp candidate lists
+  float* comp;      // [2][kCandLocal]   compacted candidates (first: staging of the row-wide bins)
   float* all;       // [2][kCandTotal]
+  int* wcnt;        // [2][VW]
   int* sel;         // [8]
   int* cnts;        // [2] local counts, then [2][kMaxCluster] counts of every rank
 };
@@ -191,7 +193,6 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int NV4 = E / 4;
   for (int i = tid; i < 2 * kBins; i += VT) s.bins[i] = 0;
-  if (tid < 2) s.cnts[tid] = 0;
   __syncthreads();
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
@@ -207,7 +208,7 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
     }
   }
   csync(c);
-  uint32_t* gb = reinterpret_cast<uint32_t*>(s.candl);     // [2][kBins] bins of the whole row
+  uint32_t* gb = reinterpret_cast<uint32_t*>(s.comp);      // [2][kBins] bins of the whole row
   if (c.nrank > 1) {
     for (int i = tid; i < 2 * kBins; i += VT) {
       uint32_t g = 0;
@@ -221,58 +222,66 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
   } else {
     gb = s.bins;
   }
-  if (warp < 2 && kth[warp & 1] > 0) {
-    // smallest bin whose cumulative count reaches k: lane l covers bins 16l .. 16l+15
-    const int r = warp;
-    constexpr int PER = kBins / 32;
-    uint32_t sum = 0;
-#pragma unroll
-    for (int i = 0; i < PER; ++i) sum += gb[r * kBins + PER * lane + i];
-    uint32_t incl = sum;
+  {
+    // smallest bin whose cumulative count reaches k.  Two-level scan over the 2 x 512 bins:
+    // thread t holds bin t % 512 of row t / 512 (VT == 2 * kBins).
+    const int r = tid / kBins, bin = tid % kBins;
+    const uint32_t cnt = kth[r] > 0 ? gb[tid] : 0u;
+    uint32_t incl = cnt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += t;
     }
-    const uint32_t excl = incl - sum, need = static_cast<uint32_t>(kth[r]);
-    if (excl < need && need <= incl) {
-      uint32_t run = excl;
-      for (int i = 0; i < PER; ++i) {
-        const uint32_t cnt = gb[r * kBins + PER * lane + i];
-        if (run < need && need <= run + cnt) {
-          s.sel[r * 2 + 0] = PER * lane + i;
-          s.sel[r * 2 + 1] = static_cast<int>(need - run);
-        }
-        run += cnt;
-      }
+    uint32_t* wtot = reinterpret_cast<uint32_t*>(s.all);      // [VW] inclusive totals per warp
+    if (lane == 31) wtot[warp] = incl;
+    __syncthreads();
+    uint32_t before = 0;
+    for (int w = r * (kBins / 32); w < warp; ++w) before += wtot[w];
+    const uint32_t need = static_cast<uint32_t>(kth[r] > 0 ? kth[r] : 0);
+    const uint32_t hi = before + incl, lo_ = hi - cnt;
+    if (kth[r] > 0 && lo_ < need && need <= hi) {
+      s.sel[r * 2 + 0] = bin;
+      s.sel[r * 2 + 1] = static_cast<int>(need - lo_);
     }
   }
   __syncthreads();           // also: the staged bins have been consumed, candl may be overwritten
   int bstar[2], krem[2];
 #pragma unroll
   for (int r = 0; r < 2; ++r) { bstar[r] = kth[r] > 0 ? s.sel[r * 2] : -1; krem[r] = kth[r] > 0 ? s.sel[r * 2 + 1] : 0; }
+  // Entries of the located bin -> per-warp lists (ballot-compacted, no atomics): warp w keeps
+  // up to kWarpCand entries of row r in wl[(r*VW + w)*kWarpCand ..] and their count in wcnt.
+  constexpr int kWarpCand = kCandLocal / VW;
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
     if (kth[r] <= 0) continue;
     const float* z = r ? z1 : z0;
+    float* wl = s.wl + (r * VW + warp) * kWarpCand;
+    // dist_bin(z) == bstar  <=>  bits(max - z) - lo_bits < span  (unsigned); the clamped end
+    // bins take everything below / above
+    const uint32_t lo_bits = bstar[r] == 0 ? 0u : static_cast<uint32_t>(bstar[r] + kBinBase) << 18;
+    const uint32_t hi_bits = bstar[r] == kBins - 1 ? 0xffffffffu : (static_cast<uint32_t>(bstar[r] + kBinBase + 1) << 18) - 1u;
+    const uint32_t span = hi_bits - lo_bits;
+    const float mxr = mx[r];
+    int run = 0;
 #pragma unroll
     for (int v = 0; v < NV4; ++v) {
       const float4 q = *reinterpret_cast<const float4*>(z + warp * 32 * E + v * 128 + lane * 4);
       const float ev[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-      for (int e = 0; e < 4; ++e)
-        if (dist_bin(mx[r], ev[e]) == bstar[r]) {
-          const int pos = atomicAdd(&s.cnts[r], 1);
-          if (pos < kCandLocal) s.candl[r * kCandLocal + pos] = ev[e];
+      for (int e = 0; e < 4; ++e) {
+        const bool match = (__float_as_uint(mxr - ev[e]) - lo_bits) <= span;
+        const uint32_t m = __ballot_sync(0xffffffffu, match);
+        if (m) {                                   // rare: a few entries per warp
+          if (match) {
+            const int pos = run + __popc(m & ((1u << lane) - 1u));
+            if (pos < kWarpCand) wl[pos] = ev[e];
+          }
+          run += __popc(m);
         }
+      }
     }
-  }
-  csync(c);
-  // candidate counts of every rank
-  int* rc = s.cnts + 2;
-  if (tid < 2 * static_cast<int>(c.nrank)) {
-    const int r = tid / c.nrank, q = tid % c.nrank;
-    rc[r * kMaxCluster + q] = static_cast<int>(dsmem_ld_u32(dsmem_addr(smem_u32(&s.cnts[r]), q)));
+    if (lane == 0) s.wcnt[r * VW + warp] = run;
   }
   __syncthreads();
   int total[2] = {0, 0};
@@ -280,39 +289,85 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
     if (kth[r] <= 0) continue;
-    for (uint32_t q = 0; q < c.nrank; ++q) {
-      const int n = rc[r * kMaxCluster + q];
-      if (n > kCandLocal) fits[r] = false;
-      total[r] += n;
-    }
-    if (total[r] > kCandTotal) fits[r] = false;
+    const int n = s.wcnt[r * VW + lane];                    // VW == 32
+    total[r] = __reduce_add_sync(0xffffffffu, n);
+    if (__any_sync(0xffffffffu, n > kWarpCand)) fits[r] = false;
   }
+  // compact the per-warp lists: every warp places its own entries behind those of the
+  // warps before it
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (kth[r] <= 0) continue;
+    const int n = min(s.wcnt[r * VW + lane], kWarpCand);
+    int incl = n;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    const int my_off = __shfl_sync(0xffffffffu, incl - n, warp);
+    const int my_n = __shfl_sync(0xffffffffu, n, warp);
+    if (lane < my_n) s.comp[r * kCandLocal + my_off + lane] = s.wl[(r * VW + warp) * kWarpCand + lane];
+    if (warp == 0 && lane == 31) s.cnts[r] = fits[r] ? incl : kCandLocal + 1;
+  }
+  csync(c);
+  const float* cand_base = s.comp;             // [2][cand_stride] candidates of the whole row
+  int cand_stride = kCandLocal;
+  if (c.nrank > 1) {
+    int* rc = s.cnts + 2;
+    if (tid < 2 * static_cast<int>(c.nrank)) {
+      const int r = tid / c.nrank, q = tid % c.nrank;
+      rc[r * kMaxCluster + q] = static_cast<int>(dsmem_ld_u32(dsmem_addr(smem_u32(&s.cnts[r]), q)));
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      total[r] = 0;
+      fits[r] = true;
+      if (kth[r] <= 0) continue;
+      for (uint32_t q = 0; q < c.nrank; ++q) {
+        const int n = rc[r * kMaxCluster + q];
+        if (n > kCandLocal) fits[r] = false;
+        total[r] += n;
+      }
+      if (total[r] > kCandTotal) fits[r] = false;
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      if (kth[r] <= 0 || !fits[r]) continue;
+      int off = 0;
+      for (uint32_t q = 0; q < c.nrank; ++q) {
+        const int n = rc[r * kMaxCluster + q];
+        const uint32_t base = dsmem_addr(smem_u32(&s.comp[r * kCandLocal]), q);
+        for (int i = tid; i < n; i += VT) s.all[r * kCandTotal + off + i] = dsmem_ld_f32(base + 4u * i);
+        off += n;
+      }
+    }
+    __syncthreads();
+    cand_base = s.all;
+    cand_stride = kCandTotal;
+  }
+  // exact rank by counting: theta = v with #(> v) < k' <= #(>= v); eight lanes share the
+  // comparisons of one candidate
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
     if (kth[r] <= 0 || !fits[r]) continue;
-    int off = 0;
-    for (uint32_t q = 0; q < c.nrank; ++q) {
-      const int n = rc[r * kMaxCluster + q];
-      const uint32_t base = dsmem_addr(smem_u32(&s.candl[r * kCandLocal]), q);
-      for (int i = tid; i < n; i += VT) s.all[r * kCandTotal + off + i] = dsmem_ld_f32(base + 4u * i);
-      off += n;
-    }
-  }
-  __syncthreads();
-  // exact rank by counting: theta = v with  #(> v) < k' <= #(>= v)
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    if (kth[r] <= 0 || !fits[r]) continue;
-    const float* al = s.all + r * kCandTotal;
-    for (int i = tid; i < total[r]; i += VT) {
-      const float v = al[i];
+    const float* al = cand_base + r * cand_stride;
+    const int nc8 = (total[r] + (VT / 8) - 1) / (VT / 8) * (VT / 8);
+    for (int i = tid >> 3; i < nc8; i += VT / 8) {
+      const float v = i < total[r] ? al[i] : 0.f;
       int gt = 0, ge = 0;
-      for (int t = 0; t < total[r]; ++t) {
+      for (int t = tid & 7; t < total[r]; t += 8) {
         const float w = al[t];
         gt += (w > v);
         ge += (w >= v);
       }
-      if (gt < krem[r] && krem[r] <= ge) reinterpret_cast<float*>(s.sel)[4 + r] = v;
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) {
+        gt += __shfl_xor_sync(0xffffffffu, gt, o);
+        ge += __shfl_xor_sync(0xffffffffu, ge, o);
+      }
+      if (i < total[r] && (tid & 7) == 0 && gt < krem[r] && krem[r] <= ge) reinterpret_cast<float*>(s.sel)[4 + r] = v;
     }
   }
   __syncthreads();
@@ -395,10 +450,12 @@ __global__ void __launch_bounds__(VT, 1) verify_nodes_kernel(const VerifyArgs a)
   float* P = Q + SL;
   TopkSmem tk;
   tk.bins = reinterpret_cast<uint32_t*>(P + SL);
-  tk.candl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
-  tk.all = tk.candl + 2 * kCandLocal;
+  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
+  tk.comp = tk.wl + 2 * kCandLocal;
+  tk.all = tk.comp + 2 * kCandLocal;
   VCtx c;
-  c.red = tk.all + 2 * kCandTotal;
+  tk.wcnt = reinterpret_cast<int*>(tk.all + 2 * kCandTotal);
+  c.red = reinterpret_cast<float*>(tk.wcnt + 2 * VW);
   c.xch = c.red + 2 * VW * 4;
   c.gath = c.xch + 8;
   tk.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
@@ -458,6 +515,26 @@ __global__ void __launch_bounds__(VT, 1) verify_nodes_kernel(const VerifyArgs a)
         for (int r = tid; r < a.k; r += VT)
           nbr_s[ci * a.kpad + r] = a.nbr[static_cast<long long>(code) * a.k_table + r];
     }
+  }
+
+  // ---- uniforms of this node (fetched early: off the critical path later)
+  if (tid == 32) {
+    float u;
+    if (a.u_res) {
+      u = a.u_res[out_b + n];
+    } else {
+      u = uniform_halfopen(philox_stream(a.seed, a.step, static_cast<uint32_t>(out_b + n), kStreamResample, 0).x);
+    }
+    reinterpret_cast<float*>(misc)[7] = u;
+  }
+  if (tid < nc) {
+    float u;
+    if (a.u_acc) {
+      u = a.u_acc[out_b + fc + tid];
+    } else {
+      u = uniform_halfopen(philox_stream(a.seed, a.step, static_cast<uint32_t>(out_b + fc + tid), kStreamAccept, 0).x);
+    }
+    reinterpret_cast<float*>(misc)[8 + tid] = u;
   }
 
   // ---- read the rows once: z_q -> Q, z_p -> P
@@ -607,12 +684,7 @@ __global__ void __launch_bounds__(VT, 1) verify_nodes_kernel(const VerifyArgs a)
       if (__any_sync(0xffffffffu, bad) && lane == 0 && c.rank == 0) vflag(a.status, LANTERN_DEV_BAD_INDEX);
       const float m = cum;
       const float thr = px > 0.f ? fminf(1.f, m / px) : (m > 0.f ? 1.f : 0.f);
-      float u;
-      if (a.u_acc) {
-        u = a.u_acc[out_b + child];
-      } else {
-        u = uniform_halfopen(philox_stream(a.seed, a.step, static_cast<uint32_t>(out_b + child), kStreamAccept, 0).x);
-      }
+      const float u = reinterpret_cast<const float*>(misc)[8 + ci];
       if (lane == 0) {
         misc[0] = (u < thr) ? 1 : 0;
         misc[1] = nA;
@@ -697,13 +769,8 @@ __global__ void __launch_bounds__(VT, 1) verify_nodes_kernel(const VerifyArgs a)
   // The last reduction left the per-warp sums of Q in c.last_red[w*2] and the per-rank sums in
   // c.gath[r*2]; the slice and the warp segment that hold the draw follow from those.
   if (accepted < 0) {
-    float u;
-    if (a.u_res) {
-      u = a.u_res[out_b + n];
-    } else {
-      u = uniform_halfopen(philox_stream(a.seed, a.step, static_cast<uint32_t>(out_b + n), kStreamResample, 0).x);
-    }
     __syncthreads();                      // c.gath was written by warp 0
+    const float u = reinterpret_cast<const float*>(misc)[7];
     float total = 0.f;
     for (uint32_t r = 0; r < c.nrank; ++r) total += c.gath[r * 2];
     const float target = u * total;
@@ -718,16 +785,15 @@ __global__ void __launch_bounds__(VT, 1) verify_nodes_kernel(const VerifyArgs a)
     bool fallback = false;
     if (owner < 0) { owner = last_pos; fallback = true; }     // rounding pushed the target past the end
     if (owner == static_cast<int>(c.rank)) {
-      int ow = -1, lastw = -1;
-      float Ew = E_owner, Ew_owner = 0.f;
-      for (int w = 0; w < VW; ++w) {
-        const float t = c.last_red[w * 2];
-        if (t > 0.f) lastw = w;
-        if (!fallback && ow < 0 && Ew + t > target) { ow = w; Ew_owner = Ew; }
-        Ew += t;
-      }
+      // every warp finds the owner warp: lane w holds the sum of warp w's segment
+      const float wt = c.last_red[lane * 2];
+      const float wincl = warp_incl_scan(wt, lane);
+      const uint32_t hit = fallback ? 0u : __ballot_sync(0xffffffffu, E_owner + wincl > target);
+      const uint32_t pos = __ballot_sync(0xffffffffu, wt > 0.f);
+      int ow = hit ? __ffs(hit) - 1 : -1;
       bool wfallback = fallback;
-      if (ow < 0) { ow = lastw; wfallback = true; }
+      if (ow < 0) { ow = pos ? 31 - __clz(pos) : 0; wfallback = true; }
+      const float Ew_owner = E_owner + __shfl_sync(0xffffffffu, wincl - wt, ow);
       if (warp == ow) {
         int found = -1;
         const int wlo = warp * 32 * E;
