@@ -160,6 +160,38 @@ lantern_status lantern_verify_tree(const lantern_params* params, const lantern_t
                                    int32_t* device_status, void* workspace, size_t workspace_bytes,
                                    void* stream);
 
+/* ---- relaxed verification without any allocation ---------------------------------------------
+ * The paper has no counterpart to this entry point; it exists for callers that must not, or
+ * cannot, allocate device memory around the call: code running inside a memory pool that is
+ * already fully handed out, a serving loop that forbids cudaMalloc because it synchronises the
+ * device, or a host that only passes buffers it was given.  It is lantern_verify_tree with the
+ * per-node scratch (accepted child and drawn token of every node, 8 bytes per node) taken from a
+ * fixed array inside the library instead of a caller workspace.  The array holds
+ * lantern_verify_tree_static_max_nodes() = 65536 nodes (512 KB), so batch * n_nodes must not
+ * exceed that: larger calls return LANTERN_ERR_UNSUPPORTED and launch nothing.  Every GPU that
+ * loads the library keeps the array until the process exits.
+ *  - Nothing is allocated or freed, by this call or by anything it calls.
+ *  - The first call on a device looks up the array's device address (a one-time query with that
+ *    device current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array and it keeps the previous call's contents.  The
+ *    kernel writes every entry it later reads, so nothing needs clearing, but two calls that
+ *    overlap on the GPU (different streams, no ordering between them) race on it and give
+ *    wrong results.  Order such calls, or give the overlapping ones a workspace through
+ *    lantern_verify_tree.
+ * Arguments and results are those of lantern_verify_tree; node_next / node_token are not
+ * returned.                                                                                      */
+int32_t lantern_verify_tree_static_max_nodes(void);
+lantern_status lantern_verify_tree_static(const lantern_params* params, const lantern_tree* tree,
+                                          const int32_t* nbr_idx, int32_t k_table,
+                                          const void* target_cond, const void* target_uncond,
+                                          const void* draft_cond, const void* draft_uncond,
+                                          lantern_dtype dt, int64_t row_stride, int64_t seq_stride,
+                                          int32_t batch, const int32_t* tokens,
+                                          const float* u_accept, const float* u_resample,
+                                          int32_t* accept_len, int32_t* out_tokens, int32_t* out_nodes,
+                                          float* node_mass, float* node_thresh,
+                                          int32_t* device_status, void* stream);
+
 /* Raw Philox-4x32-10 words (Salmon et al., SC 2011) for counters (first + i, c1, c2, c3), i in
  * [0, n): out[i][0..3].  Exists so that the generator can be checked against other
  * implementations.  out is a device pointer to n*4 uint32.                                      */

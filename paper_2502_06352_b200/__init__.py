@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     build_neighbors,
     sample_draft_tree,
     verify_tree,
+    verify_tree_static,
     philox_raw,
     set_cluster_size,
     lib,

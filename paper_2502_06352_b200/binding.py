@@ -83,6 +83,11 @@ def _load():
     L.lantern_verify_tree.restype = ctypes.c_int
     L.lantern_verify_tree.argtypes = [ctypes.POINTER(_CParams), vp, vp, i32, vp, vp, vp, vp, ctypes.c_int,
                                       i64, i64, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.lantern_verify_tree_static.restype = ctypes.c_int
+    L.lantern_verify_tree_static.argtypes = [ctypes.POINTER(_CParams), vp, vp, i32, vp, vp, vp, vp, ctypes.c_int,
+                                             i64, i64, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.lantern_verify_tree_static_max_nodes.restype = i32
+    L.lantern_verify_tree_static_max_nodes.argtypes = []
     L.lantern_philox_raw.restype = ctypes.c_int
     L.lantern_philox_raw.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
                                      ctypes.c_uint32, i32, vp, vp]
@@ -220,6 +225,31 @@ def verify_tree(params: Params, tree: Tree, nbr_idx, target_cond, target_uncond,
             _ptr(u_accept), _ptr(u_resample), _ptr(accept_len), _ptr(out_tokens), _ptr(out_nodes),
             _ptr(node_next), _ptr(node_token), _ptr(node_mass), _ptr(node_thresh), _ptr(device_status),
             _ptr(workspace), workspace.numel(), _stream()), "lantern_verify_tree")
+    return out
+
+
+def verify_tree_static(params: Params, tree: Tree, nbr_idx, target_cond, target_uncond, draft_cond, draft_uncond,
+                       tokens, u_accept=None, u_resample=None, *, out, device_status=None):
+    """lantern_verify_tree_static: verification for callers that cannot allocate.
+
+    The library call allocates nothing; to keep this wrapper allocation-free as well, `out`
+    must already hold accept_len [B], out_tokens and out_nodes [B][max_depth+1] (int32, on the
+    logits' device).  batch * n_nodes may not exceed lantern_verify_tree_static_max_nodes().
+    Calls share one built-in scratch array per GPU: do not let two of them overlap."""
+    B, N, V = target_cond.shape[0], tree.n_nodes, params.vocab
+    rs, ss = _rows(target_cond, B, N, V)
+    for t in (target_uncond, draft_cond, draft_uncond):
+        if t is not None and _rows(t, B, N, V) != (rs, ss):
+            raise ValueError("all logit tensors must share strides")
+    k_table = 0 if nbr_idx is None else nbr_idx.shape[1]
+    cp = params.c()
+    with torch.cuda.device(target_cond.device):
+        _check(lib.lantern_verify_tree_static(
+            ctypes.byref(cp), tree.handle, _ptr(nbr_idx), k_table, _ptr(target_cond), _ptr(target_uncond),
+            _ptr(draft_cond), _ptr(draft_uncond), _dtype_code(target_cond), rs, ss, B, _ptr(tokens),
+            _ptr(u_accept), _ptr(u_resample), _ptr(out["accept_len"]), _ptr(out["out_tokens"]),
+            _ptr(out["out_nodes"]), _ptr(out.get("node_mass")), _ptr(out.get("node_thresh")),
+            _ptr(device_status), _stream()), "lantern_verify_tree_static")
     return out
 
 

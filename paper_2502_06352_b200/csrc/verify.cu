@@ -184,3 +184,50 @@ extern "C" lantern_status lantern_verify_tree(
   if (cudaGetLastError() != cudaSuccess) return LANTERN_ERR_CUDA;
   return LANTERN_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Variant of lantern_verify_tree for callers that cannot allocate device memory.
+// Its per-node scratch (accepted child and drawn token of every node) lives in a fixed array
+// that is part of the library image; every GPU that loads the library holds it until exit.
+namespace {
+constexpr int kStaticMaxNodes = 1 << 16;       // batch * tree nodes the built-in scratch can hold
+static __device__ __align__(256) int32_t g_static_scratch[2 * kStaticMaxNodes];
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_ptr[kMaxDevices] = {};  // device address of the array, per device
+
+// The array's name is only a handle on the host; the kernels need its device address, which is
+// looked up once per device (with that device current).
+lantern_status static_scratch_for_current_device(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LANTERN_ERR_CUDA;
+  if (!g_static_scratch_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return LANTERN_ERR_CUDA;
+    g_static_scratch_ptr[dev] = p;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return LANTERN_OK;
+}
+}  // namespace
+
+extern "C" int32_t lantern_verify_tree_static_max_nodes(void) { return kStaticMaxNodes; }
+
+extern "C" lantern_status lantern_verify_tree_static(
+    const lantern_params* p, const lantern_tree* tree, const int32_t* nbr_idx, int32_t k_table,
+    const void* target_cond, const void* target_uncond, const void* draft_cond, const void* draft_uncond,
+    lantern_dtype dt, int64_t row_stride, int64_t seq_stride, int32_t batch, const int32_t* tokens,
+    const float* u_accept, const float* u_resample, int32_t* accept_len, int32_t* out_tokens,
+    int32_t* out_nodes, float* node_mass, float* node_thresh, int32_t* device_status, void* stream) {
+  if (!tree || batch <= 0) return LANTERN_ERR_INVALID_ARG;
+  const TreeDev* t = reinterpret_cast<const TreeDev*>(tree);
+  if (static_cast<int64_t>(batch) * t->n_nodes > kStaticMaxNodes) return LANTERN_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  lantern_status st = static_scratch_for_current_device(&scratch);
+  if (st != LANTERN_OK) return st;
+  // Every scratch entry of the nodes in use is written by the kernel before the walk reads it,
+  // so nothing has to be cleared between calls.
+  return lantern_verify_tree(p, tree, nbr_idx, k_table, target_cond, target_uncond, draft_cond, draft_uncond, dt,
+                             row_stride, seq_stride, batch, tokens, u_accept, u_resample, accept_len, out_tokens,
+                             out_nodes, nullptr, nullptr, node_mass, node_thresh, device_status, scratch,
+                             sizeof(int32_t) * 2 * kStaticMaxNodes, stream);
+}
