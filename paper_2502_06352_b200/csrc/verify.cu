@@ -33,6 +33,7 @@ __global__ void walk_kernel(const int32_t* __restrict__ node_next, const int32_t
 static int g_cluster_override = 0;
 
 struct LaunchShape { int cs, e; size_t smem; };
+constexpr int kMaxE = 16384 / VT;      // a CTA's slice holds at most 16384 row entries
 
 // Choose E (row entries per thread; a CTA's slice is 1024*E entries) and the cluster size.
 // `min_e` is 4 for float32 rows and 8 for bfloat16 rows (one 16-byte vector per thread).
@@ -43,15 +44,15 @@ static bool choose_shape(int V, int rows, int max_children, int kpad, int min_e,
   auto cs_for = [&](int e) { int cs = (V + VT * e - 1) / (VT * e); return cs > 8 ? (cs > 16 ? 0 : 16) : cs; };
   int e = 0;
   if (g_cluster_override > 0) {
-    for (int cand = min_e; cand <= 16; cand *= 2)
+    for (int cand = min_e; cand <= kMaxE; cand *= 2)
       if (static_cast<long long>(VT) * cand * g_cluster_override >= V) { e = cand; break; }
     if (e == 0) return false;
     out->cs = g_cluster_override;
   } else {
     // the smallest slice that holds the row in one CTA, else the largest slice
-    for (int cand = min_e; cand <= 16; cand *= 2)
+    for (int cand = min_e; cand <= kMaxE; cand *= 2)
       if (VT * cand >= V) { e = cand; break; }
-    if (e == 0) e = 16;
+    if (e == 0) e = kMaxE;
     if (cs_for(e) == 0) return false;
     // few rows: split each over more CTAs so that more SMs stream
     while (e > min_e && static_cast<long long>(rows) * cs_for(e) < 74 && cs_for(e / 2) != 0 && cs_for(e / 2) <= 8) e /= 2;
@@ -88,6 +89,9 @@ static cudaError_t launch_verify_e(const VerifyArgs& a, const LaunchShape& sh, c
 
 template <typename T, bool CFG>
 static cudaError_t launch_verify(const VerifyArgs& a, const LaunchShape& sh, cudaStream_t st) {
+  if constexpr (kMaxE >= 32) {
+    if (sh.e == 32) return launch_verify_e<T, CFG, 32>(a, sh, st);
+  }
   if (sh.e == 16) return launch_verify_e<T, CFG, 16>(a, sh, st);
   if (sh.e == 8) return launch_verify_e<T, CFG, 8>(a, sh, st);
   if constexpr (Vec<T>::N <= 4) {

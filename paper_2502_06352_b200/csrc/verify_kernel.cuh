@@ -15,11 +15,17 @@
 
 namespace lantern {
 
-constexpr int VT = 1024;          // threads per CTA
+#ifndef LANTERN_VT
+#define LANTERN_VT 1024
+#endif
+constexpr int VT = LANTERN_VT;    // threads per CTA (1024 or 512)
 constexpr int VW = VT / 32;       // warps per CTA
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kBins = 512;        // histogram bins of the top-k locator (2 * kBins == VT)
-constexpr int kBinBase = (127 - 9) << 5;   // 32 bins per binade of d = max - z, d in [2^-9, 2^7)
+constexpr int kBins = 512;        // histogram bins of the top-k locator
+constexpr int kBinLog = 5;        // log2 of the bins per binade of d = max - z
+constexpr int kBinShift = 23 - kBinLog;
+constexpr int kBinBase = (127 - 9) << kBinLog;        // 16 binades: d in [2^-9, 2^7)
+static_assert(VT == 1024 || VT == 512, "thread count");
 constexpr int kCandLocal = 512;   // top-k candidates one CTA may contribute per row
 constexpr int kCandTotal = 1024;  // and the whole cluster
 
@@ -88,7 +94,7 @@ __device__ __forceinline__ void row_reduce(VCtx& c, float (&v)[NV]) {
   __syncthreads();
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
-    float t = red[lane * NV + i];               // VW == 32: one partial per lane
+    float t = lane < VW ? red[lane * NV + i] : (IS_MAX ? -INFINITY : 0.f);   // one partial per lane
     v[i] = IS_MAX ? warp_max(t) : warp_sum(t);
   }
   if (c.nrank > 1) {
@@ -167,7 +173,7 @@ __device__ __forceinline__ float load_row(const T* __restrict__ cond, const T* _
 // Coarse position of an entry below the row maximum: a monotone function of z.
 __device__ __forceinline__ int dist_bin(float mx, float z) {
   const float d = mx - z;
-  const int b = static_cast<int>(__float_as_uint(d) >> 18) - kBinBase;
+  const int b = static_cast<int>(__float_as_uint(d) >> kBinShift) - kBinBase;
   return min(max(b, 0), kBins - 1);
 }
 
@@ -223,26 +229,36 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
     gb = s.bins;
   }
   {
-    // smallest bin whose cumulative count reaches k.  Two-level scan over the 2 x 512 bins:
-    // thread t holds bin t % 512 of row t / 512 (VT == 2 * kBins).
-    const int r = tid / kBins, bin = tid % kBins;
-    const uint32_t cnt = kth[r] > 0 ? gb[tid] : 0u;
-    uint32_t incl = cnt;
+    // smallest bin whose cumulative count reaches k.  Two-level scan over the 2 x kBins bins:
+    // in round `it` thread t holds entry it*VT + t of the [row][bin] array.
+    constexpr int RPT = 2 * kBins / VT;
+    constexpr int WPR = kBins / 32;                            // warps' worth of bins per row
+    uint32_t cnt[RPT], incl[RPT];
+    uint32_t* wtot = reinterpret_cast<uint32_t*>(s.all);       // [2 * WPR] inclusive totals
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += t;
+    for (int it = 0; it < RPT; ++it) {
+      const int g = it * VT + tid, r = g / kBins;
+      cnt[it] = kth[r] > 0 ? gb[g] : 0u;
+      incl[it] = cnt[it];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl[it], o);
+        if (lane >= o) incl[it] += t;
+      }
+      if (lane == 31) wtot[it * VW + warp] = incl[it];
     }
-    uint32_t* wtot = reinterpret_cast<uint32_t*>(s.all);      // [VW] inclusive totals per warp
-    if (lane == 31) wtot[warp] = incl;
     __syncthreads();
-    uint32_t before = 0;
-    for (int w = r * (kBins / 32); w < warp; ++w) before += wtot[w];
-    const uint32_t need = static_cast<uint32_t>(kth[r] > 0 ? kth[r] : 0);
-    const uint32_t hi = before + incl, lo_ = hi - cnt;
-    if (kth[r] > 0 && lo_ < need && need <= hi) {
-      s.sel[r * 2 + 0] = bin;
-      s.sel[r * 2 + 1] = static_cast<int>(need - lo_);
+#pragma unroll
+    for (int it = 0; it < RPT; ++it) {
+      const int g = it * VT + tid, r = g / kBins, bin = g % kBins, gw = it * VW + warp;
+      uint32_t before = 0;
+      for (int w = r * WPR; w < gw; ++w) before += wtot[w];
+      const uint32_t need = static_cast<uint32_t>(kth[r] > 0 ? kth[r] : 0);
+      const uint32_t hi = before + incl[it], lo_ = hi - cnt[it];
+      if (kth[r] > 0 && lo_ < need && need <= hi) {
+        s.sel[r * 2 + 0] = bin;
+        s.sel[r * 2 + 1] = static_cast<int>(need - lo_);
+      }
     }
   }
   __syncthreads();           // also: the staged bins have been consumed, candl may be overwritten
@@ -259,8 +275,8 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
     float* wl = s.wl + (r * VW + warp) * kWarpCand;
     // dist_bin(z) == bstar  <=>  bits(max - z) - lo_bits < span  (unsigned); the clamped end
     // bins take everything below / above
-    const uint32_t lo_bits = bstar[r] == 0 ? 0u : static_cast<uint32_t>(bstar[r] + kBinBase) << 18;
-    const uint32_t hi_bits = bstar[r] == kBins - 1 ? 0xffffffffu : (static_cast<uint32_t>(bstar[r] + kBinBase + 1) << 18) - 1u;
+    const uint32_t lo_bits = bstar[r] == 0 ? 0u : static_cast<uint32_t>(bstar[r] + kBinBase) << kBinShift;
+    const uint32_t hi_bits = bstar[r] == kBins - 1 ? 0xffffffffu : (static_cast<uint32_t>(bstar[r] + kBinBase + 1) << kBinShift) - 1u;
     const uint32_t span = hi_bits - lo_bits;
     const float mxr = mx[r];
     int run = 0;
@@ -289,7 +305,7 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
     if (kth[r] <= 0) continue;
-    const int n = s.wcnt[r * VW + lane];                    // VW == 32
+    const int n = lane < VW ? s.wcnt[r * VW + lane] : 0;
     total[r] = __reduce_add_sync(0xffffffffu, n);
     if (__any_sync(0xffffffffu, n > kWarpCand)) fits[r] = false;
   }
@@ -298,7 +314,7 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
     if (kth[r] <= 0) continue;
-    const int n = min(s.wcnt[r * VW + lane], kWarpCand);
+    const int n = lane < VW ? min(s.wcnt[r * VW + lane], kWarpCand) : 0;
     int incl = n;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -786,7 +802,7 @@ __global__ void __launch_bounds__(VT, 1) verify_nodes_kernel(const VerifyArgs a)
     if (owner < 0) { owner = last_pos; fallback = true; }     // rounding pushed the target past the end
     if (owner == static_cast<int>(c.rank)) {
       // every warp finds the owner warp: lane w holds the sum of warp w's segment
-      const float wt = c.last_red[lane * 2];
+      const float wt = lane < VW ? c.last_red[lane * 2] : 0.f;
       const float wincl = warp_incl_scan(wt, lane);
       const uint32_t hit = fallback ? 0u : __ballot_sync(0xffffffffu, E_owner + wincl > target);
       const uint32_t pos = __ballot_sync(0xffffffffu, wt > 0.f);
