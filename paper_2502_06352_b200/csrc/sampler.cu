@@ -2,10 +2,12 @@
 // distribution p without replacement.  Gumbel-top-s: key_j = log p_j - log(-log U_j); since
 // log p_j = z_j - const over the row, ranking z_j + G_j gives the same children.
 //
-// One thread-block cluster per expanded parent; the drafter row is read once, its
-// post-processed logits stay in shared memory (slice per CTA), the s winners are found by s
-// rounds of a cluster-wide arg-max.
-#include "rowops.cuh"
+// Same row machinery as the verify kernel: one CTA (a cluster for rows wider than 16384) per
+// expanded parent, the drafter row read once into shared memory, exact top-k threshold, then
+// one sweep that forms the keys (Philox-4x32-10, four uniforms per counter) and the softmax
+// denominator.  Every thread keeps the best key of its own entries in registers; a round picks
+// the row-wide best (ties: lower token id) and only the winner's owner rescans its entries.
+#include "verify_kernel.cuh"
 
 namespace lantern {
 
@@ -15,7 +17,7 @@ struct SampleArgs {
   const float* gumbel;
   const int32_t *first_child, *n_child, *order;
   int order_begin;
-  int B, N, V, SL;
+  int B, N, V;
   float g, inv_tau;
   int topk_d, allow_lo, allow_hi;
   unsigned long long seed, step;
@@ -24,155 +26,193 @@ struct SampleArgs {
   int32_t* status;
 };
 
-constexpr int kSamplerFixedSmem = 2 * 2 * 256 * 4 + kWarps * 4 * 4 + 8 * 4 + kMaxCluster * 4 * 4 + 4 * 4 + 16;
-
 __device__ __forceinline__ bool better(float ka, int ia, float kb, int ib) {   // a beats b
   return ka > kb || (ka == kb && ia < ib);
 }
 
-template <typename T, bool CFG>
-__global__ void __launch_bounds__(kThreads) sample_children_kernel(const SampleArgs a) {
+__device__ __forceinline__ void warp_argbest(float& k, int& i) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ok = __shfl_xor_sync(0xffffffffu, k, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+    if (better(ok, oi, k, i)) { k = ok; i = oi; }
+  }
+}
+
+// best key among this thread's entries of the key slice
+template <int E>
+__device__ __forceinline__ void thread_best(const float* __restrict__ K, int lo, float& bk, int& bi) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  bk = -INFINITY;
+  bi = 0x7fffffff;
+#pragma unroll
+  for (int v = 0; v < E / 4; ++v) {
+    const int j = warp * 32 * E + v * 128 + lane * 4;
+    const float4 k4 = *reinterpret_cast<const float4*>(K + j);
+    const float kv[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (kv[e] > bk) { bk = kv[e]; bi = lo + j + e; }     // ascending ids: strict > keeps the lower id
+  }
+}
+
+template <typename T, bool CFG, int E>
+__global__ void __launch_bounds__(VT, 1) sample_children_kernel(const SampleArgs a) {
+  constexpr int SL = VT * E;
+  constexpr int NV4 = E / 4;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* Z = reinterpret_cast<float*>(smem_raw);
-  float* K = Z + a.SL;
-  ClusterCtx c;
-  c.hist = reinterpret_cast<uint32_t*>(K + a.SL);
-  c.red = reinterpret_cast<float*>(c.hist + 2 * 2 * 256);
-  c.xch = c.red + kWarps * 4;
+  float* K = Z + SL;
+  TopkSmem tk;
+  tk.bins = reinterpret_cast<uint32_t*>(K + SL);
+  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
+  tk.comp = tk.wl + 2 * kCandLocal;
+  tk.all = tk.comp + 2 * kCandLocal;
+  VCtx c;
+  tk.wcnt = reinterpret_cast<int*>(tk.all + 2 * kCandTotal);
+  c.red = reinterpret_cast<float*>(tk.wcnt + 2 * VW);
+  c.xch = c.red + 2 * VW * 4;
   c.gath = c.xch + 8;
-  c.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
+  tk.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
+  tk.cnts = tk.sel + 8;
   c.rank = cluster_ctarank();
   c.nrank = cluster_nctarank();
   c.parity = 0;
-  c.hist_parity = 0;
+  c.last_red = c.red;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int idx = blockIdx.x / c.nrank;
   const int b = idx % a.B;
   const int n = a.order[a.order_begin + idx / a.B];
   const int fc = a.first_child[n], nc = a.n_child[n];
-  const int SL = a.SL;
   const int lo = c.rank * SL;
   const int len = max(0, min(a.V - lo, SL));
   const long long row_off = static_cast<long long>(b) * a.seq_stride + static_cast<long long>(n) * a.row_stride;
   const long long out_b = static_cast<long long>(b) * a.N;
+  const bool single = c.nrank == 1;
 
-  float mx[1];
-  mx[0] = load_slice<T, CFG>(static_cast<const T*>(a.dc) + row_off,
-                             CFG ? static_cast<const T*>(a.du) + row_off : nullptr, a.g, a.inv_tau, lo,
-                             len, a.allow_lo, a.allow_hi, Z);
-  cluster_reduce<1, true>(c, mx);
+  const bool masked = a.allow_lo > 0 || a.allow_hi < a.V;
+  float mx[2];
+  mx[0] = load_row<T, CFG, E>(static_cast<const T*>(a.dc) + row_off,
+                              CFG ? static_cast<const T*>(a.du) + row_off : nullptr, a.g, a.inv_tau, lo, len,
+                              a.allow_lo, a.allow_hi, masked, Z);
+  mx[1] = -INFINITY;
+  row_reduce<2, true>(c, mx);
   if (mx[0] == -INFINITY) {
-    if (tid == 0 && c.rank == 0 && a.status) atomicOr(a.status, LANTERN_DEV_EMPTY_ROW);
+    if (tid == 0 && c.rank == 0) vflag(a.status, LANTERN_DEV_EMPTY_ROW);
     mx[0] = 0.f;
   }
-  float theta[1] = {-INFINITY};
-  if (a.topk_d > 0 && a.topk_d < a.V) {
-    float* const rows[1] = {Z};
-    const int kth[1] = {a.topk_d};
-    cluster_topk_threshold<1>(c, rows, len, kth, theta);
-  }
+  mx[1] = 0.f;
+  float theta[2] = {-INFINITY, -INFINITY};
+  const int kth[2] = {(a.topk_d > 0 && a.topk_d < a.V) ? a.topk_d : 0, 0};
+  const bool has_topk = kth[0] > 0;
+  if (has_topk) topk_thresholds<E>(c, tk, Z, Z, mx, kth, theta);
 
-  // keys and the softmax denominator in one sweep
+  // ---- keys z + G, G = -log(-log U), and the softmax denominator, in one sweep
   const uint32_t row_id = static_cast<uint32_t>(out_b + n);
   const float* gum = a.gumbel ? a.gumbel + (static_cast<long long>(row_id) * a.V + lo) : nullptr;
-  float sm[1] = {0.f};
-  for (int i = tid; i * 4 < len; i += kThreads) {
-    const int j = i * 4;
+  const float c0 = -mx[0] * kLog2e;
+  float sm[2] = {0.f, 0.f};
+  float bk = -INFINITY;
+  int bi = 0x7fffffff;
+#pragma unroll 2
+  for (int v = 0; v < NV4; ++v) {
+    const int j = warp * 32 * E + v * 128 + lane * 4;
+    const float4 z4 = *reinterpret_cast<const float4*>(Z + j);
+    const float zv[4] = {z4.x, z4.y, z4.z, z4.w};
     float u4[4];
     if (gum) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) u4[e] = (j + e < len) ? __ldcs(gum + j + e) : 0.5f;
     } else {
-      Philox4 r = philox_stream(a.seed, a.step, row_id, kStreamGumbel, static_cast<uint32_t>((lo + j) >> 2));
+      const Philox4 r = philox_stream(a.seed, a.step, row_id, kStreamGumbel, static_cast<uint32_t>((lo + j) >> 2));
       u4[0] = uniform_open(r.x); u4[1] = uniform_open(r.y); u4[2] = uniform_open(r.z); u4[3] = uniform_open(r.w);
     }
+    float kv[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      if (j + e < len) {
-        const float z = Z[j + e];
-        const bool keep = z >= theta[0] && z != -INFINITY;
-        K[j + e] = keep ? z - logf(-logf(u4[e])) : -INFINITY;
-        if (keep) sm[0] += expf(z - mx[0]);
-      }
+      const bool keep = zv[e] >= theta[0] && zv[e] != -INFINITY;
+      kv[e] = keep ? zv[e] - __logf(-logf(u4[e])) : -INFINITY;
+      if (keep) sm[0] += ex2_approx(fmaf(zv[e], kLog2e, c0));
+      if (kv[e] > bk) { bk = kv[e]; bi = lo + j + e; }
     }
+    *reinterpret_cast<float4*>(K + j) = make_float4(kv[0], kv[1], kv[2], kv[3]);
   }
-  cluster_reduce<1, false>(c, sm);
+  row_reduce<2, false>(c, sm);
   const float inv_sum = sm[0] > 0.f ? 1.f / sm[0] : 0.f;
 
+  // ---- s rounds: row-wide best key; the owner of the winner retires it and rescans
+  float* pk = c.red + 2 * VW * 4 - 2 * VW;     // [VW] keys and [VW] ids of the warps' best (tail of red[1])
   for (int round = 0; round < nc; ++round) {
-    float bk = -INFINITY;
-    int bi = 0x7fffffff;
-    for (int j = tid; j < len; j += kThreads) {
-      const float kj = K[j];
-      if (better(kj, lo + j, bk, bi)) { bk = kj; bi = lo + j; }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ok = __shfl_xor_sync(0xffffffffu, bk, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (better(ok, oi, bk, bi)) { bk = ok; bi = oi; }
-    }
-    if (lane == 0) { c.red[warp * 2] = bk; c.red[warp * 2 + 1] = __int_as_float(bi); }
+    float wk = bk;
+    int wi = bi;
+    warp_argbest(wk, wi);
+    __syncthreads();                            // pk of the previous round has been consumed
+    if (lane == 0) { pk[warp] = wk; pk[VW + warp] = __int_as_float(wi); }
     __syncthreads();
-    if (tid == 0) {
-      for (int w = 1; w < kWarps; ++w) {
-        const float ok = c.red[w * 2];
-        const int oi = __float_as_int(c.red[w * 2 + 1]);
-        if (better(ok, oi, bk, bi)) { bk = ok; bi = oi; }
+    float ck = lane < VW ? pk[lane] : -INFINITY;
+    int ci = lane < VW ? __float_as_int(pk[VW + lane]) : 0x7fffffff;
+    warp_argbest(ck, ci);
+    if (!single) {
+      if (tid == 0) { c.xch[c.parity * 4] = ck; c.xch[c.parity * 4 + 1] = __int_as_float(ci); }
+      cluster_sync();
+      float rk = -INFINITY;
+      int ri = 0x7fffffff;
+      if (lane < static_cast<int>(c.nrank)) {
+        rk = dsmem_ld_f32(dsmem_addr(smem_u32(&c.xch[c.parity * 4]), lane));
+        ri = __float_as_int(dsmem_ld_f32(dsmem_addr(smem_u32(&c.xch[c.parity * 4 + 1]), lane)));
       }
-      c.xch[c.parity * 4] = bk;
-      c.xch[c.parity * 4 + 1] = __int_as_float(bi);
+      warp_argbest(rk, ri);
+      ck = rk;
+      ci = ri;
+      c.parity ^= 1;
     }
-    cluster_sync();
-    if (tid < static_cast<int>(c.nrank) * 2)
-      c.gath[tid] = dsmem_ld_f32(dsmem_addr(smem_u32(&c.xch[c.parity * 4 + (tid & 1)]), tid >> 1));
-    __syncthreads();
-    c.parity ^= 1;
-    bk = c.gath[0];
-    bi = __float_as_int(c.gath[1]);
-    for (uint32_t r = 1; r < c.nrank; ++r) {
-      const float ok = c.gath[r * 2];
-      const int oi = __float_as_int(c.gath[r * 2 + 1]);
-      if (better(ok, oi, bk, bi)) { bk = ok; bi = oi; }
-    }
-    const bool valid = bk != -INFINITY;
-    if (valid && bi >= lo && bi < lo + len && tid == 0) {
-      K[bi - lo] = -INFINITY;
-      a.tokens[out_b + fc + round] = bi;
-      if (a.draft_prob) a.draft_prob[out_b + fc + round] = expf(Z[bi - lo] - mx[0]) * inv_sum;
+    const bool valid = ck != -INFINITY;
+    if (valid && ci == bi) {                    // exactly one thread of the row owns the winner
+      const int jl = ci - lo;
+      K[jl] = -INFINITY;
+      a.tokens[out_b + fc + round] = ci;
+      if (a.draft_prob) a.draft_prob[out_b + fc + round] = ex2_approx(fmaf(Z[jl], kLog2e, c0)) * inv_sum;
+      thread_best<E>(K, lo, bk, bi);           // this thread's own writes are visible to it
     }
     if (!valid && c.rank == 0 && tid == 0) {
       a.tokens[out_b + fc + round] = -1;
       if (a.draft_prob) a.draft_prob[out_b + fc + round] = 0.f;
     }
-    __syncthreads();
   }
-  cluster_sync();
+  if (!single) cluster_sync();
 }
 
-static bool sampler_shape(int V, int rows, int* cs_out, int* sl_out, size_t* smem_out, int override_cs) {
-  auto smem_for = [&](int sl) { return static_cast<size_t>(2) * sl * 4 + kSamplerFixedSmem; };
-  int cs = 1;
+}  // namespace lantern
+
+namespace lantern {
+
+// Choose E (row entries per thread; a CTA's slice is VT*E entries) and the cluster size.
+static bool sampler_shape(int V, int rows, int min_e, int override_cs, int* cs_out, int* e_out, size_t* smem_out) {
+  constexpr int kMaxE = 16384 / VT;
+  auto cs_for = [&](int e) { int cs = (V + VT * e - 1) / (VT * e); return cs > 8 ? (cs > 16 ? 0 : 16) : cs; };
+  int e = 0;
   if (override_cs > 0) {
-    cs = override_cs;
+    for (int cand = min_e; cand <= kMaxE; cand *= 2)
+      if (static_cast<long long>(VT) * cand * override_cs >= V) { e = cand; break; }
+    if (e == 0) return false;
+    *cs_out = override_cs;
   } else {
-    while (cs < kMaxCluster && (V + cs - 1) / cs > 4096) cs *= 2;
-    while (cs < 8 && rows * cs < 296 && (V + cs - 1) / cs > 1024) cs *= 2;
+    for (int cand = min_e; cand <= kMaxE; cand *= 2)
+      if (VT * cand >= V) { e = cand; break; }
+    if (e == 0) e = kMaxE;
+    if (cs_for(e) == 0) return false;
+    while (e > min_e && static_cast<long long>(rows) * cs_for(e) < 74 && cs_for(e / 2) != 0 && cs_for(e / 2) <= 8) e /= 2;
+    *cs_out = cs_for(e);
   }
-  int sl = (((V + cs - 1) / cs) + 7) & ~7;
-  while (cs < kMaxCluster && smem_for(sl) > 227 * 1024) {
-    cs *= 2;
-    sl = (((V + cs - 1) / cs) + 7) & ~7;
-  }
-  if (smem_for(sl) > 227 * 1024) return false;
-  *cs_out = cs; *sl_out = sl; *smem_out = smem_for(sl);
-  return true;
+  *e_out = e;
+  *smem_out = static_cast<size_t>(2) * VT * e * 4 + kVerifyFixedSmem;
+  return *smem_out <= 227 * 1024;
 }
 
-template <typename T, bool CFG>
-static cudaError_t launch_sampler(const SampleArgs& a, int n_parents, int cs, size_t smem, cudaStream_t st) {
-  auto kern = sample_children_kernel<T, CFG>;
+template <typename T, bool CFG, int E>
+static cudaError_t launch_sampler_e(const SampleArgs& a, int n_parents, int cs, size_t smem, cudaStream_t st) {
+  auto kern = sample_children_kernel<T, CFG, E>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
   if (cs > 8) {
@@ -181,7 +221,7 @@ static cudaError_t launch_sampler(const SampleArgs& a, int n_parents, int cs, si
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(a.B) * n_parents * cs, 1, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.blockDim = dim3(VT, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -192,6 +232,19 @@ static cudaError_t launch_sampler(const SampleArgs& a, int n_parents, int cs, si
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+template <typename T, bool CFG>
+static cudaError_t launch_sampler(const SampleArgs& a, int n_parents, int cs, int e, size_t smem, cudaStream_t st) {
+  if constexpr (16384 / VT >= 32) {
+    if (e == 32) return launch_sampler_e<T, CFG, 32>(a, n_parents, cs, smem, st);
+  }
+  if (e == 16) return launch_sampler_e<T, CFG, 16>(a, n_parents, cs, smem, st);
+  if (e == 8) return launch_sampler_e<T, CFG, 8>(a, n_parents, cs, smem, st);
+  if constexpr (Vec<T>::N <= 4) {
+    if (e == 4) return launch_sampler_e<T, CFG, 4>(a, n_parents, cs, smem, st);
+  }
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace lantern
@@ -238,18 +291,17 @@ extern "C" lantern_status lantern_sample_draft_tree(
   a.topk_d = p->top_k_draft; a.allow_lo = allow_lo; a.allow_hi = allow_hi;
   a.seed = p->seed; a.step = p->step;
   a.tokens = tokens; a.draft_prob = draft_prob; a.status = device_status;
-  int cs, sl;
+  int cs, e;
   size_t smem;
-  int ov = lantern_set_cluster_size(-1);     // -1 is not a valid size: reads the current value
-  if (!sampler_shape(V, batch * (i1 - i0), &cs, &sl, &smem, ov)) return LANTERN_ERR_UNSUPPORTED;
-  a.SL = sl;
+  const int ov = lantern_set_cluster_size(-1);     // -1 is not a valid size: reads the current value
+  if (!sampler_shape(V, batch * (i1 - i0), dt == LANTERN_F32 ? 4 : 8, ov, &cs, &e, &smem)) return LANTERN_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = draft_uncond != nullptr;
-  cudaError_t e;
+  cudaError_t err;
   if (dt == LANTERN_F32)
-    e = cfg ? launch_sampler<float, true>(a, i1 - i0, cs, smem, st) : launch_sampler<float, false>(a, i1 - i0, cs, smem, st);
+    err = cfg ? launch_sampler<float, true>(a, i1 - i0, cs, e, smem, st) : launch_sampler<float, false>(a, i1 - i0, cs, e, smem, st);
   else
-    e = cfg ? launch_sampler<__nv_bfloat16, true>(a, i1 - i0, cs, smem, st)
-            : launch_sampler<__nv_bfloat16, false>(a, i1 - i0, cs, smem, st);
-  return e == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
+    err = cfg ? launch_sampler<__nv_bfloat16, true>(a, i1 - i0, cs, e, smem, st)
+              : launch_sampler<__nv_bfloat16, false>(a, i1 - i0, cs, e, smem, st);
+  return err == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
 }
