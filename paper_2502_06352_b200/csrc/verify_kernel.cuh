@@ -457,8 +457,11 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t phase)
 }
 
 // E = row entries per thread; the CTA's slice holds SL = 1024 * E entries.
+#ifndef LANTERN_MINB
+#define LANTERN_MINB 1
+#endif
 template <typename T, bool CFG, int E>
-__global__ void __launch_bounds__(VT, 1) verify_nodes_kernel(const VerifyArgs a) {
+__global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const VerifyArgs a) {
   constexpr int SL = VT * E;
   constexpr int NV4 = E / 4;                 // float4 per thread in a shared-memory sweep
   extern __shared__ __align__(16) unsigned char smem_raw[];
