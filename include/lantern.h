@@ -94,6 +94,10 @@ typedef struct {
  *   codebook  [L][d] row-major, dt = F32 or BF16            nbr_idx  [L][k] int32
  *   nbr_dist  [L][k] float32 squared distances, or NULL
  *   workspace device scratch of at least lantern_build_neighbors_workspace() bytes, 256-B aligned
+ *             (row norms for the tensor-core path; 0 bytes when that path is not taken)
+ * bfloat16 codebooks with d a multiple of 16 in [32, 256] and k <= 320 take a tensor-core path:
+ * approximate distances from bf16 MMAs select a superset of the neighbours (with a proven error
+ * margin), which is then ranked exactly.  Everything else takes an exact brute-force kernel.
  * Requires 1 <= k <= min(L-1, 1024), 1 <= d <= 4096.                                            */
 size_t lantern_build_neighbors_workspace(lantern_dtype dt, int32_t L, int32_t d, int32_t k);
 lantern_status lantern_build_neighbors(const void* codebook, lantern_dtype dt, int32_t L, int32_t d,

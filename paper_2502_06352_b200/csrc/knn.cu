@@ -75,6 +75,68 @@ __device__ __forceinline__ double exact_dist(const T* __restrict__ cb, int d, in
   return s;
 }
 
+// Exact ranking of one query's surviving candidates (keys carry the candidate index in their
+// low 32 bits): distances re-evaluated in double, sorted by (distance, index), first k written.
+// With `overflow` the buffer is ignored and k rounds of an exact arg-min over all rows are run.
+template <typename T>
+__device__ __forceinline__ void rank_query(const T* __restrict__ cb, int L, int d, int k, int qi,
+                                           const unsigned long long* bq, int n_in, bool overflow, int CAP,
+                                           double* sortd, int* sorti, double* redd, int* redi,
+                                           int32_t* out_i, float* out_d) {
+  const int tid = threadIdx.x;
+    if (!overflow) {
+    const int n = min(n_in, CAP);
+          for (int i = tid; i < CAP; i += kKnnThreads) {
+      if (i < n) {
+        int j = static_cast<int>(bq[i] & 0xffffffffu);
+        sorti[i] = j;
+        sortd[i] = exact_dist<T>(cb, d, qi, j);
+      } else {
+        sorti[i] = 0x7fffffff;
+        sortd[i] = INFINITY;
+      }
+    }
+    __syncthreads();
+    bitonic_pair(sortd, sorti, CAP);
+    for (int r = tid; r < k; r += kKnnThreads) {
+      out_i[r] = sorti[r];
+      if (out_d) out_d[r] = static_cast<float>(sortd[r]);
+    }
+    __syncthreads();
+  } else {
+    // exact fallback: k rounds of arg-min over (distance, index) greater than the last pick
+    double pd = -1.0;
+    int pj = -1;
+    for (int r = 0; r < k; ++r) {
+      double bd = INFINITY;
+      int bj = 0x7fffffff;
+      for (int j = tid; j < L; j += kKnnThreads) {
+        if (j == qi) continue;
+        double dj = exact_dist<T>(cb, d, qi, j);
+        bool after = dj > pd || (dj == pd && j > pj);
+        if (after && (dj < bd || (dj == bd && j < bj))) { bd = dj; bj = j; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        double od = __shfl_xor_sync(0xffffffffu, bd, o);
+        int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+        if (od < bd || (od == bd && oj < bj)) { bd = od; bj = oj; }
+      }
+      if ((tid & 31) == 0) { redd[tid >> 5] = bd; redi[tid >> 5] = bj; }
+      __syncthreads();
+      bd = redd[0]; bj = redi[0];
+      for (int w = 1; w < kKnnThreads / 32; ++w)
+        if (redd[w] < bd || (redd[w] == bd && redi[w] < bj)) { bd = redd[w]; bj = redi[w]; }
+      __syncthreads();
+      pd = bd; pj = bj;
+      if (tid == 0) {
+        out_i[r] = bj;
+        if (out_d) out_d[r] = static_cast<float>(bd);
+      }
+    }
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kKnnThreads) knn_kernel(const KnnArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -176,80 +238,60 @@ __global__ void __launch_bounds__(kKnnThreads) knn_kernel(const KnnArgs a) {
   // final ranking per query
   for (int q = 0; q < nq; ++q) {
     const int qi = q0 + q;
-    int32_t* out_i = a.nbr_idx + static_cast<long long>(qi) * k;
-    float* out_d = a.nbr_dist ? a.nbr_dist + static_cast<long long>(qi) * k : nullptr;
-    if (!ovf[q]) {
-      const int n = min(cnt[q], CAP);
-      const unsigned long long* bq = buf + static_cast<size_t>(q) * CAP;
-      for (int i = tid; i < CAP; i += kKnnThreads) {
-        if (i < n) {
-          int j = static_cast<int>(bq[i] & 0xffffffffu);
-          sorti[i] = j;
-          sortd[i] = exact_dist<T>(cb, d, qi, j);
-        } else {
-          sorti[i] = 0x7fffffff;
-          sortd[i] = INFINITY;
-        }
-      }
-      __syncthreads();
-      bitonic_pair(sortd, sorti, CAP);
-      for (int r = tid; r < k; r += kKnnThreads) {
-        out_i[r] = sorti[r];
-        if (out_d) out_d[r] = static_cast<float>(sortd[r]);
-      }
-      __syncthreads();
-    } else {
-      // exact fallback: k rounds of arg-min over (distance, index) greater than the last pick
-      double pd = -1.0;
-      int pj = -1;
-      for (int r = 0; r < k; ++r) {
-        double bd = INFINITY;
-        int bj = 0x7fffffff;
-        for (int j = tid; j < L; j += kKnnThreads) {
-          if (j == qi) continue;
-          double dj = exact_dist<T>(cb, d, qi, j);
-          bool after = dj > pd || (dj == pd && j > pj);
-          if (after && (dj < bd || (dj == bd && j < bj))) { bd = dj; bj = j; }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          double od = __shfl_xor_sync(0xffffffffu, bd, o);
-          int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-          if (od < bd || (od == bd && oj < bj)) { bd = od; bj = oj; }
-        }
-        if ((tid & 31) == 0) { redd[tid >> 5] = bd; redi[tid >> 5] = bj; }
-        __syncthreads();
-        bd = redd[0]; bj = redi[0];
-        for (int w = 1; w < kKnnThreads / 32; ++w)
-          if (redd[w] < bd || (redd[w] == bd && redi[w] < bj)) { bd = redd[w]; bj = redi[w]; }
-        __syncthreads();
-        pd = bd; pj = bj;
-        if (tid == 0) {
-          out_i[r] = bj;
-          if (out_d) out_d[r] = static_cast<float>(bd);
-        }
-      }
-    }
+    rank_query<T>(cb, L, d, k, qi, buf + static_cast<size_t>(q) * CAP, cnt[q], ovf[q] != 0, CAP, sortd, sorti, redd, redi,
+                  a.nbr_idx + static_cast<long long>(qi) * k,
+                  a.nbr_dist ? a.nbr_dist + static_cast<long long>(qi) * k : nullptr);
   }
 }
 
 }  // namespace lantern
 
+#include "knn_tc.cuh"
+
 using namespace lantern;
 
+// The tensor-core path is taken for bfloat16 codebooks with d a multiple of 16 in [32, 256] and
+// k small enough for its per-query buffers.
+static bool use_tensor_path(lantern_dtype dt, int L, int d, int k) {
+  return dt == LANTERN_BF16 && d % 16 == 0 && d >= 32 && d <= kTcMaxD && k <= 320 && L >= 64;
+}
+
 extern "C" size_t lantern_build_neighbors_workspace(lantern_dtype dt, int32_t L, int32_t d, int32_t k) {
-  (void)dt; (void)L; (void)d; (void)k;
-  return 0;   // the brute-force kernel keeps all of its state on chip
+  if (L < 2 || d < 1 || k < 1) return 0;
+  // squared norms of all rows and their maximum (tensor-core path); the brute-force kernel
+  // keeps all of its state on chip
+  return use_tensor_path(dt, L, d, k) ? (static_cast<size_t>(L) + 64) * sizeof(float) : 0;
 }
 
 extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_dtype dt, int32_t L, int32_t d,
                                                   int32_t k, int32_t* nbr_idx, float* nbr_dist, void* workspace,
                                                   size_t workspace_bytes, void* stream) {
-  (void)workspace; (void)workspace_bytes;
   if (!codebook || !nbr_idx) return LANTERN_ERR_INVALID_ARG;
   if (dt != LANTERN_F32 && dt != LANTERN_BF16) return LANTERN_ERR_INVALID_ARG;
   if (L < 2 || d < 1 || k < 1 || k > L - 1) return LANTERN_ERR_INVALID_ARG;
   if (k > 1024 || d > 4096) return LANTERN_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (use_tensor_path(dt, L, d, k)) {
+    const size_t need = lantern_build_neighbors_workspace(dt, L, d, k);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) % 256)) return LANTERN_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(codebook) % 16) return LANTERN_ERR_INVALID_ARG;
+    float* nrm = static_cast<float*>(workspace);
+    if (cudaMemsetAsync(nrm + L, 0, sizeof(float), st) != cudaSuccess) return LANTERN_ERR_CUDA;
+    knn_norms_kernel<<<(L * 32 + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(codebook), L, d, nrm);
+    if (cudaGetLastError() != cudaSuccess) return LANTERN_ERR_CUDA;
+    KnnTcArgs ta;
+    ta.cb = static_cast<const __nv_bfloat16*>(codebook); ta.nrm = nrm; ta.L = L; ta.d = d; ta.k = k;
+    ta.CAP = 256;
+    while (ta.CAP < k + 192) ta.CAP *= 2;
+    ta.nbr_idx = nbr_idx; ta.nbr_dist = nbr_dist;
+    const int ld = d + kTcPad;
+    const size_t tsm = static_cast<size_t>(kTcQT) * ta.CAP * 8 + static_cast<size_t>(kTcQT) * ld * 2 +
+                       static_cast<size_t>(2) * kTcCT * ld * 2 + 2 * kTcCT * 4 + 5 * kTcQT * 4 + 64;
+    if (cudaFuncSetAttribute(knn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tsm)) != cudaSuccess)
+      return LANTERN_ERR_CUDA;
+    knn_tc_kernel<<<(L + kTcQT - 1) / kTcQT, kKnnThreads, tsm, st>>>(ta);
+    return cudaGetLastError() == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
+  }
   KnnArgs a;
   a.cb = codebook; a.L = L; a.d = d; a.k = k; a.nbr_idx = nbr_idx; a.nbr_dist = nbr_dist;
   int cap = 512;
@@ -265,7 +307,6 @@ extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_
   while (a.QT > 1 && smem_for(a.QT, a.q_double) > 220 * 1024) a.QT /= 2;
   size_t smem = smem_for(a.QT, a.q_double);
   if (smem > 227 * 1024) return LANTERN_ERR_UNSUPPORTED;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int grid = (L + a.QT - 1) / a.QT;
   cudaError_t e;
   if (dt == LANTERN_F32) {

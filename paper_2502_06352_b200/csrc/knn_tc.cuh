@@ -1,0 +1,203 @@
+// Tensor-core path of the latent-neighbour table for bfloat16 codebooks whose embedding dimension
+// makes the distance matrix a real dense contraction (d a multiple of 16, 32 <= d <= 256).
+//
+//   approximate distance  f(i,j) = |c_i|^2 + |c_j|^2 - 2 <c_i, c_j>      (float32)
+// with the inner products from bf16 tensor-core MMAs (products exact, float32 accumulation).
+// |f - D| <= eps_i for the exact squared distance D, eps_i = (d+8) * 2^-21 * (|c_i|^2 + max_j |c_j|^2)
+// (accumulation of d exact products, the two norms, two final roundings, factor 2 of slack).
+// If tau is the k-th smallest f seen for a query, every true neighbour has f <= tau + 2 eps, so
+// the streaming filter keeps candidates with f <= tau + 2 eps and nothing else; the survivors are
+// then re-ranked exactly (double precision, ties by index) like in the brute-force kernel.
+//
+// A CTA owns 32 query rows (kept in shared memory for the whole kernel) and streams all rows
+// as candidate tiles of 64 through a cp.async double buffer; 8 warps each own a 16 x 16 block of
+// the 32 x 64 tile (mma.sync m16n8k16).  Rows are padded by 16 bytes in shared memory, which
+// makes the 32-bit fragment loads bank-conflict free.
+#pragma once
+
+#include "common.cuh"
+
+namespace lantern {
+
+constexpr int kTcQT = 32;          // query rows per CTA
+constexpr int kTcCT = 64;          // candidate rows per tile
+constexpr int kTcPad = 8;          // bf16 elements of padding per shared-memory row
+constexpr int kTcMaxD = 256;
+
+struct KnnTcArgs {
+  const __nv_bfloat16* cb;
+  const float* nrm;        // [L] squared norms, nrm[L] = their maximum
+  int L, d, k, CAP;
+  int32_t* nbr_idx;
+  float* nbr_dist;
+};
+
+// squared norms (float32) and their maximum
+__global__ void knn_norms_kernel(const __nv_bfloat16* __restrict__ cb, int L, int d, float* __restrict__ nrm) {
+  const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (row >= L) return;
+  float s = 0.f;
+  for (int t = lane; t < d; t += 32) {
+    const float v = __bfloat162float(cb[static_cast<long long>(row) * d + t]);
+    s = fmaf(v, v, s);
+  }
+  s = warp_sum(s);
+  if (lane == 0) {
+    nrm[row] = s;
+    atomicMax(reinterpret_cast<unsigned int*>(nrm + L), __float_as_uint(s));   // s >= 0: bit order = value order
+  }
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// stage rows [row0, row0 + rows) of the codebook into padded shared-memory rows (zero beyond L)
+__device__ __forceinline__ void stage_rows(const __nv_bfloat16* __restrict__ cb, int L, int d, int row0, int rows,
+                                           __nv_bfloat16* dst) {
+  const int chunks = d / 8;                   // 16-byte chunks per row
+  const int ld = d + kTcPad;
+  for (int i = threadIdx.x; i < rows * chunks; i += kKnnThreads) {
+    const int r = i / chunks, ch = i - r * chunks;
+    const int row = row0 + r;
+    const bool in = row < L;
+    const __nv_bfloat16* src = cb + static_cast<long long>(in ? row : 0) * d + ch * 8;
+    cp_async16(smem_u32(dst + r * ld + ch * 8), src, in ? 16u : 0u);
+  }
+}
+
+
+__global__ void __launch_bounds__(kKnnThreads) knn_tc_kernel(const KnnTcArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int d = a.d, L = a.L, k = a.k, CAP = a.CAP, ld = d + kTcPad;
+  const __nv_bfloat16* cb = a.cb;
+  unsigned long long* buf = reinterpret_cast<unsigned long long*>(smem_raw);            // [QT][CAP]
+  __nv_bfloat16* As = reinterpret_cast<__nv_bfloat16*>(buf + static_cast<size_t>(kTcQT) * CAP);   // [QT][ld]
+  __nv_bfloat16* Bs = As + kTcQT * ld;                                                  // [2][CT][ld]
+  float* ncs = reinterpret_cast<float*>(Bs + 2 * kTcCT * ld);                           // [2][CT]
+  float* nq = ncs + 2 * kTcCT;                                                          // [QT]
+  float* thr = nq + kTcQT;
+  float* eps2 = thr + kTcQT;
+  int* cnt = reinterpret_cast<int*>(eps2 + kTcQT);
+  int* ovf = cnt + kTcQT;
+  // after the main loop the tile buffers are reused by the exact ranking
+  double* sortd = reinterpret_cast<double*>(Bs);
+  double* redd = sortd + CAP;
+  int* sorti = reinterpret_cast<int*>(redd + 8);
+  int* redi = sorti + CAP;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int q0 = blockIdx.x * kTcQT;
+  const int ntiles = (L + kTcCT - 1) / kTcCT;
+  const float nmax = a.nrm[L];
+
+  stage_rows(cb, L, d, q0, kTcQT, As);
+  stage_rows(cb, L, d, 0, kTcCT, Bs);
+  cp_async_commit();
+  if (tid < kTcCT) ncs[tid] = tid < L ? a.nrm[tid] : 0.f;
+  if (tid < kTcQT) {
+    const float n = q0 + tid < L ? a.nrm[q0 + tid] : 0.f;
+    nq[tid] = n;
+    eps2[tid] = 2.f * static_cast<float>(d + 8) * 4.76837158203125e-7f * (n + nmax);     // 2 * eps, 2^-21
+    thr[tid] = INFINITY;
+    cnt[tid] = 0;
+    ovf[tid] = 0;
+  }
+
+  const int wq = warp & 1, wc = warp >> 1;
+  const int r0 = wq * 16 + (lane >> 2), r1 = r0 + 8;
+  const int kc = 2 * (lane & 3);
+
+  for (int t = 0; t < ntiles; ++t) {
+    const int cur = t & 1;
+    if (t + 1 < ntiles) {
+      stage_rows(cb, L, d, (t + 1) * kTcCT, kTcCT, Bs + (cur ^ 1) * kTcCT * ld);
+      cp_async_commit();
+      if (tid < kTcCT) {
+        const int j = (t + 1) * kTcCT + tid;
+        ncs[(cur ^ 1) * kTcCT + tid] = j < L ? a.nrm[j] : 0.f;
+      }
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
+    __syncthreads();
+    const __nv_bfloat16* Bt = Bs + cur * kTcCT * ld;
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    for (int kb = 0; kb < d; kb += 16) {
+      uint32_t af[4];
+      af[0] = *reinterpret_cast<const uint32_t*>(As + r0 * ld + kb + kc);
+      af[1] = *reinterpret_cast<const uint32_t*>(As + r1 * ld + kb + kc);
+      af[2] = *reinterpret_cast<const uint32_t*>(As + r0 * ld + kb + kc + 8);
+      af[3] = *reinterpret_cast<const uint32_t*>(As + r1 * ld + kb + kc + 8);
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        const __nv_bfloat16* bp = Bt + (wc * 16 + nt * 8 + (lane >> 2)) * ld + kb + kc;
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(bp);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(bp + 8);
+        mma_bf16_16816(acc[nt], af, b0, b1);
+      }
+    }
+    // epilogue: approximate distances, filter, append
+    const float thr0 = thr[r0], thr1 = thr[r1], nq0 = nq[r0], nq1 = nq[r1];
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int col = wc * 16 + nt * 8 + kc + (e & 1);
+        const int r = (e < 2) ? r0 : r1;
+        const int j = t * kTcCT + col;
+        const float f = fmaf(-2.f, acc[nt][e], ((e < 2) ? nq0 : nq1) + ncs[cur * kTcCT + col]);
+        if (j < L && q0 + r < L && j != q0 + r && f <= ((e < 2) ? thr0 : thr1)) {
+          const int pos = atomicAdd(&cnt[r], 1);
+          if (pos < CAP)
+            buf[static_cast<size_t>(r) * CAP + pos] =
+                (static_cast<unsigned long long>(float_key(f)) << 32) | static_cast<unsigned>(j);
+        }
+      }
+    }
+    __syncthreads();
+    // cut back buffers that might overflow during the next tile
+    for (int q = 0; q < kTcQT; ++q) {
+      const int n = cnt[q];
+      if (n <= CAP - kTcCT || ovf[q]) continue;            // uniform: shared values
+      unsigned long long* bq = buf + static_cast<size_t>(q) * CAP;
+      for (int i = n + tid; i < CAP; i += kKnnThreads) bq[i] = ~0ull;
+      __syncthreads();
+      bitonic_u64(bq, CAP);
+      if (tid == 0) {
+        const float tau = key_float(static_cast<uint32_t>(bq[k - 1] >> 32));
+        const float th = tau + eps2[q];
+        int lo = k, hi = n;                                 // first index in [k, n) whose f exceeds th
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (key_float(static_cast<uint32_t>(bq[mid] >> 32)) <= th) lo = mid + 1; else hi = mid;
+        }
+        thr[q] = th;
+        cnt[q] = lo;
+        if (lo > CAP - kTcCT) ovf[q] = 1;                   // too many rows within the error margin
+      }
+      __syncthreads();
+    }
+  }
+  __syncthreads();
+  for (int q = 0; q < kTcQT; ++q) {
+    const int qi = q0 + q;
+    if (qi >= L) break;
+    rank_query<__nv_bfloat16>(cb, L, d, k, qi, buf + static_cast<size_t>(q) * CAP, cnt[q], ovf[q] != 0, CAP, sortd, sorti,
+                              redd, redi, a.nbr_idx + static_cast<long long>(qi) * k,
+                              a.nbr_dist ? a.nbr_dist + static_cast<long long>(qi) * k : nullptr);
+  }
+}
+
+}  // namespace lantern

@@ -29,7 +29,8 @@ def _check(L, cb, k, rows=None):
 
 @pytest.mark.parametrize("n,d,k,dt", [(2, 1, 1, "f32"), (17, 3, 16, "f32"), (300, 8, 10, "f32"),
                                       (1000, 8, 50, "bf16"), (777, 64, 33, "bf16"), (600, 256, 200, "bf16"),
-                                      (1500, 40, 700, "f32")])
+                                      (1500, 40, 700, "f32"), (64, 32, 63, "bf16"), (2000, 128, 320, "bf16"),
+                                      (1000, 48, 321, "bf16"), (333, 256, 7, "bf16")])
 def test_small_codebooks_all_rows(L, n, d, k, dt):
     cb = W.make_codebook(n, d, dt, seed=n + d, dup_frac=0.05 if n > 50 else 0.0)
     _check(L, cb, k)
@@ -42,6 +43,21 @@ def test_duplicates_tie_by_index_and_zero_distance(L):
     idx, dist = _check(L, cb, 5)
     assert list(idx[3][:2]) == [10, 40] and list(dist[3][:2]) == [0, 0]
     assert list(idx[10][:2]) == [3, 40] and list(idx[40][:2]) == [3, 10]
+
+
+def test_tensor_path_margin_keeps_near_ties_exact(L):
+    """bf16 rows that differ in one low-order entry: approximate distances nearly tie, the exact
+    re-rank must still order them by true distance and then by index."""
+    g = torch.Generator().manual_seed(3)
+    base = (torch.randn((1, 64), generator=g) * 4).to(torch.bfloat16)
+    cb = base.repeat(512, 1).contiguous()
+    # row i differs from the base in entry (i % 64) by one bf16 step of that entry, sign by parity
+    for i in range(1, 512):
+        e = i % 64
+        v = cb[i, e].float()
+        step = 2.0 ** (torch.floor(torch.log2(v.abs())) - 7)
+        cb[i, e] = (v + step * (1 if i % 2 else -1) * (1 + i // 128)).to(torch.bfloat16)
+    _check(L, cb, 40)
 
 
 def test_massive_ties_take_the_exact_fallback(L):
