@@ -65,7 +65,8 @@ __global__ void __launch_bounds__(VT, 1) sample_children_kernel(const SampleArgs
   float* K = Z + SL;
   TopkSmem tk;
   tk.bins = reinterpret_cast<uint32_t*>(K + SL);
-  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
+  tk.gbins = tk.bins + 2 * kBins;
+  tk.wl = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
   tk.comp = tk.wl + 2 * kCandLocal;
   tk.all = tk.comp + 2 * kCandLocal;
   VCtx c;

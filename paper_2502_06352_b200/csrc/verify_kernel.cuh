@@ -21,8 +21,8 @@ namespace lantern {
 constexpr int VT = LANTERN_VT;    // threads per CTA (1024 or 512)
 constexpr int VW = VT / 32;       // warps per CTA
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kBins = 512;        // histogram bins of the top-k locator
-constexpr int kBinLog = 5;        // log2 of the bins per binade of d = max - z
+constexpr int kBins = 2048;       // histogram bins of the top-k locator
+constexpr int kBinLog = 7;        // log2 of the bins per binade of d = max - z
 constexpr int kBinShift = 23 - kBinLog;
 constexpr int kBinBase = (127 - 9) << kBinLog;        // 16 binades: d in [2^-9, 2^7)
 static_assert(VT == 1024 || VT == 512, "thread count");
@@ -49,7 +49,7 @@ struct VerifyArgs {
 constexpr int kMiscInts = 16;
 constexpr int kCntInts = 2 + 2 * kMaxCluster + 2;
 // fixed part of the dynamic shared memory behind the two row slices
-constexpr int kVerifyFixedSmem = 2 * kBins * 4 + 4 * kCandLocal * 4 + 2 * kCandTotal * 4 + 2 * VW * 4   // top-k
+constexpr int kVerifyFixedSmem = 4 * kBins * 4 + 4 * kCandLocal * 4 + 2 * kCandTotal * 4 + 2 * VW * 4   // top-k
                                  + 2 * VW * 4 * 4      // red (two buffers)
                                  + 2 * 4 * 4           // xch
                                  + kMaxCluster * 4 * 4 // gath
@@ -179,8 +179,9 @@ __device__ __forceinline__ int dist_bin(float mx, float z) {
 
 struct TopkSmem {
   uint32_t* bins;   // [2][kBins]
+  uint32_t* gbins;  // [2][kBins]  bins of the whole row (clusters only)
   float* wl;        // [2][VW][kCandLocal/VW] per-warp candidate lists
-  float* comp;      // [2][kCandLocal]   compacted candidates (first: staging of the row-wide bins)
+  float* comp;      // [2][kCandLocal]   compacted candidates
   float* all;       // [2][kCandTotal]
   int* wcnt;        // [2][VW]
   int* sel;         // [8]
@@ -214,7 +215,7 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
     }
   }
   csync(c);
-  uint32_t* gb = reinterpret_cast<uint32_t*>(s.comp);      // [2][kBins] bins of the whole row
+  uint32_t* gb = s.gbins;                                  // [2][kBins] bins of the whole row
   if (c.nrank > 1) {
     for (int i = tid; i < 2 * kBins; i += VT) {
       uint32_t g = 0;
@@ -248,11 +249,29 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
       if (lane == 31) wtot[it * VW + warp] = incl[it];
     }
     __syncthreads();
+    // offsets of the warps' blocks within each row: every warp scans its row's WPR block totals
+    // (WPR / 32 per lane), so no further barrier is needed
+    constexpr int PL = WPR / 32;
 #pragma unroll
     for (int it = 0; it < RPT; ++it) {
       const int g = it * VT + tid, r = g / kBins, bin = g % kBins, gw = it * VW + warp;
-      uint32_t before = 0;
-      for (int w = r * WPR; w < gw; ++w) before += wtot[w];
+      uint32_t part[PL], lsum = 0;
+#pragma unroll
+      for (int i = 0; i < PL; ++i) { part[i] = wtot[r * WPR + lane * PL + i]; lsum += part[i]; }
+      uint32_t linc = lsum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, linc, o);
+        if (lane >= o) linc += t;
+      }
+      // blocks before block (gw - r*WPR): whole lanes before its lane, then the lane's own prefix
+      const int blk = gw - r * WPR, bl = blk / PL, bo = blk % PL;
+      uint32_t before = __shfl_sync(0xffffffffu, linc - lsum, bl);
+#pragma unroll
+      for (int i = 0; i < PL; ++i) {
+        const uint32_t pv = __shfl_sync(0xffffffffu, part[i], bl);
+        if (i < bo) before += pv;
+      }
       const uint32_t need = static_cast<uint32_t>(kth[r] > 0 ? kth[r] : 0);
       const uint32_t hi = before + incl[it], lo_ = hi - cnt[it];
       if (kth[r] > 0 && lo_ < need && need <= hi) {
@@ -469,7 +488,8 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
   float* P = Q + SL;
   TopkSmem tk;
   tk.bins = reinterpret_cast<uint32_t*>(P + SL);
-  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
+  tk.gbins = tk.bins + 2 * kBins;
+  tk.wl = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
   tk.comp = tk.wl + 2 * kCandLocal;
   tk.all = tk.comp + 2 * kCandLocal;
   VCtx c;
