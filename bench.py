@@ -60,7 +60,7 @@ TRAFFIC = {"c2_llamagen512": {"kernel_sha256": "", "bytes": None}}
 def kernel_sha256():
     import hashlib
     h = hashlib.sha256()
-    for f in ("verify_kernel.cuh", "verify.cu", "rowops.cuh", "common.cuh"):
+    for f in ("verify_kernel.cuh", "verify_launch.cuh", "verify.cu", "rowops.cuh", "common.cuh"):
         with open(os.path.join(ROOT, "paper_2502_06352_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]

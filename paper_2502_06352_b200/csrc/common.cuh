@@ -129,4 +129,22 @@ __device__ __forceinline__ float uniform_open(uint32_t x) {       // (0,1), exac
   return (static_cast<float>(x >> 9) + 0.5f) * 1.1920928955078125e-7f;
 }
 
+// Arguments of the verify kernels (all thread-count variants).
+struct VerifyArgs {
+  const void *tc, *tu, *dc, *du;
+  long long row_stride, seq_stride;
+  const int32_t* tokens;
+  const float *u_acc, *u_res;
+  const int32_t* nbr;
+  int k_table, use_bulk;
+  const int32_t *first_child, *n_child, *order;
+  int B, N, V, kpad;
+  float g, inv_tau, lambda;
+  int topk_t, topk_d, k, code_offset, n_codes, allow_lo, allow_hi;
+  unsigned long long seed, step;
+  int32_t *node_next, *node_token;
+  float *node_mass, *node_thresh;
+  int32_t* status;
+};
+
 }  // namespace lantern

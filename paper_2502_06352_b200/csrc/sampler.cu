@@ -7,9 +7,13 @@
 // one sweep that forms the keys (Philox-4x32-10, four uniforms per counter) and the softmax
 // denominator.  Every thread keeps the best key of its own entries in registers; a round picks
 // the row-wide best (ties: lower token id) and only the winner's owner rescans its entries.
+#include "common.cuh"
+#define LANTERN_VT 1024
+#define LANTERN_VNS v1024
 #include "verify_kernel.cuh"
 
 namespace lantern {
+using namespace v1024;
 
 struct SampleArgs {
   const void *dc, *du;

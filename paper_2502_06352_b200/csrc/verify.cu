@@ -1,5 +1,24 @@
 // Relaxed verification of a static draft tree: host side of lantern_verify_tree and the walk.
+#include "common.cuh"
+
+namespace lantern {
+static int g_cluster_override = 0;
+}
+
+// two builds of the kernels: 1024 threads per CTA for rows that fit one CTA, 512 threads per CTA
+// for rows split over a cluster
+#define LANTERN_VT 1024
+#define LANTERN_VNS v1024
 #include "verify_kernel.cuh"
+#include "verify_launch.cuh"
+#undef LANTERN_VT
+#undef LANTERN_VNS
+#define LANTERN_VT 512
+#define LANTERN_VNS v512
+#include "verify_kernel.cuh"
+#include "verify_launch.cuh"
+#undef LANTERN_VT
+#undef LANTERN_VNS
 
 namespace lantern {
 
@@ -28,76 +47,6 @@ __global__ void walk_kernel(const int32_t* __restrict__ node_next, const int32_t
   on[len] = cur;
   accept_len[b] = len;
   for (int i = len + 1; i < D1; ++i) { ot[i] = -1; on[i] = -1; }
-}
-
-static int g_cluster_override = 0;
-
-struct LaunchShape { int cs, e; size_t smem; };
-constexpr int kMaxE = 16384 / VT;      // a CTA's slice holds at most 16384 row entries
-
-// Choose E (row entries per thread; a CTA's slice is 1024*E entries) and the cluster size.
-// `min_e` is 4 for float32 rows and 8 for bfloat16 rows (one 16-byte vector per thread).
-static bool choose_shape(int V, int rows, int max_children, int kpad, int min_e, LaunchShape* out) {
-  auto smem_for = [&](int e) {
-    return static_cast<size_t>(2) * VT * e * 4 + kVerifyFixedSmem + static_cast<size_t>(max_children) * kpad * 4;
-  };
-  auto cs_for = [&](int e) { int cs = (V + VT * e - 1) / (VT * e); return cs > 8 ? (cs > 16 ? 0 : 16) : cs; };
-  int e = 0;
-  if (g_cluster_override > 0) {
-    for (int cand = min_e; cand <= kMaxE; cand *= 2)
-      if (static_cast<long long>(VT) * cand * g_cluster_override >= V) { e = cand; break; }
-    if (e == 0) return false;
-    out->cs = g_cluster_override;
-  } else {
-    // the smallest slice that holds the row in one CTA, else the largest slice
-    for (int cand = min_e; cand <= kMaxE; cand *= 2)
-      if (VT * cand >= V) { e = cand; break; }
-    if (e == 0) e = kMaxE;
-    if (cs_for(e) == 0) return false;
-    // few rows: split each over more CTAs so that more SMs stream
-    while (e > min_e && static_cast<long long>(rows) * cs_for(e) < 74 && cs_for(e / 2) != 0 && cs_for(e / 2) <= 8) e /= 2;
-    out->cs = cs_for(e);
-  }
-  out->e = e;
-  out->smem = smem_for(e);
-  return out->smem <= 227 * 1024;
-}
-
-template <typename T, bool CFG, int E>
-static cudaError_t launch_verify_e(const VerifyArgs& a, const LaunchShape& sh, cudaStream_t st) {
-  auto kern = verify_nodes_kernel<T, CFG, E>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sh.smem));
-  if (e != cudaSuccess) return e;
-  if (sh.cs > 8) {
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-    if (e != cudaSuccess) return e;
-  }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(a.B) * a.N * sh.cs, 1, 1);
-  cfg.blockDim = dim3(VT, 1, 1);
-  cfg.dynamicSmemBytes = sh.smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = sh.cs;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, a);
-}
-
-template <typename T, bool CFG>
-static cudaError_t launch_verify(const VerifyArgs& a, const LaunchShape& sh, cudaStream_t st) {
-  if constexpr (kMaxE >= 32) {
-    if (sh.e == 32) return launch_verify_e<T, CFG, 32>(a, sh, st);
-  }
-  if (sh.e == 16) return launch_verify_e<T, CFG, 16>(a, sh, st);
-  if (sh.e == 8) return launch_verify_e<T, CFG, 8>(a, sh, st);
-  if constexpr (Vec<T>::N <= 4) {
-    if (sh.e == 4) return launch_verify_e<T, CFG, 4>(a, sh, st);
-  }
-  return cudaErrorInvalidValue;
 }
 
 }  // namespace lantern
@@ -172,15 +121,27 @@ extern "C" lantern_status lantern_verify_tree(
   a.seed = p->seed; a.step = p->step;
   a.node_next = node_next; a.node_token = node_token; a.node_mass = node_mass; a.node_thresh = node_thresh;
   a.status = device_status;
-  LaunchShape sh;
-  if (!choose_shape(V, batch * t->n_nodes, t->max_children, a.kpad, dt == LANTERN_F32 ? 4 : 8, &sh)) return LANTERN_ERR_UNSUPPORTED;
+  // rows that fit one CTA run the 1024-thread build; rows split over a cluster run the
+  // 512-thread build (cheaper barriers, half the per-thread fixed work per entry)
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = target_uncond != nullptr;
+  const bool f32 = dt == LANTERN_F32;
+  const int min_e = f32 ? 4 : 8, rows = batch * t->n_nodes;
   cudaError_t e;
-  if (dt == LANTERN_F32)
-    e = cfg ? launch_verify<float, true>(a, sh, st) : launch_verify<float, false>(a, sh, st);
-  else
-    e = cfg ? launch_verify<__nv_bfloat16, true>(a, sh, st) : launch_verify<__nv_bfloat16, false>(a, sh, st);
+  v1024::LaunchShape s1;
+  const bool ok1 = v1024::choose_shape(V, rows, t->max_children, a.kpad, min_e, &s1);
+  if (ok1 && s1.cs == 1) {
+    e = v1024::launch_any(a, s1, f32, cfg, st);
+  } else {
+    v512::LaunchShape s5;
+    if (v512::choose_shape(V, rows, t->max_children, a.kpad, min_e, &s5)) {
+      e = v512::launch_any(a, s5, f32, cfg, st);
+    } else if (ok1) {
+      e = v1024::launch_any(a, s1, f32, cfg, st);
+    } else {
+      return LANTERN_ERR_UNSUPPORTED;
+    }
+  }
   if (e != cudaSuccess) return LANTERN_ERR_CUDA;
   const int D1 = t->max_depth + 1;
   walk_kernel<<<(batch + 127) / 128, 128, 0, st>>>(node_next, node_token, tokens, batch, t->n_nodes, D1,

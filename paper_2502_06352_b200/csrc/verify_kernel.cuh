@@ -9,15 +9,19 @@
 // 128-bit streaming loads and post-processed (guidance, temperature, top-k, softmax); the
 // unnormalised distributions stay in shared memory: q_cur[j] = Q[j]*qs, p_cur[j] = P[j]/psum.
 // The sibling loop, the residual updates and the inverse-CDF draw run on chip.
-#pragma once
-
 #include "rowops.cuh"
-
-namespace lantern {
 
 #ifndef LANTERN_VT
 #define LANTERN_VT 1024
 #endif
+#ifndef LANTERN_VNS
+#define LANTERN_VNS v1024
+#endif
+
+// This header is compiled once per thread count, each time into its own namespace.
+namespace lantern {
+namespace LANTERN_VNS {
+
 constexpr int VT = LANTERN_VT;    // threads per CTA (1024 or 512)
 constexpr int VW = VT / 32;       // warps per CTA
 constexpr float kLog2e = 1.4426950408889634f;
@@ -29,22 +33,6 @@ static_assert(VT == 1024 || VT == 512, "thread count");
 constexpr int kCandLocal = 512;   // top-k candidates one CTA may contribute per row
 constexpr int kCandTotal = 1024;  // and the whole cluster
 
-struct VerifyArgs {
-  const void *tc, *tu, *dc, *du;
-  long long row_stride, seq_stride;
-  const int32_t* tokens;
-  const float *u_acc, *u_res;
-  const int32_t* nbr;
-  int k_table, use_bulk;
-  const int32_t *first_child, *n_child, *order;
-  int B, N, V, kpad;
-  float g, inv_tau, lambda;
-  int topk_t, topk_d, k, code_offset, n_codes, allow_lo, allow_hi;
-  unsigned long long seed, step;
-  int32_t *node_next, *node_token;
-  float *node_mass, *node_thresh;
-  int32_t* status;
-};
 
 constexpr int kMiscInts = 16;
 constexpr int kCntInts = 2 + 2 * kMaxCluster + 2;
@@ -888,4 +876,5 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
   if (!single) cluster_sync();    // peers may still be reading this CTA's shared memory
 }
 
+}  // namespace LANTERN_VNS
 }  // namespace lantern
