@@ -129,6 +129,20 @@ __device__ __forceinline__ float uniform_open(uint32_t x) {       // (0,1), exac
   return (static_cast<float>(x >> 9) + 0.5f) * 1.1920928955078125e-7f;
 }
 
+// ---------------------------------------------------------------- asynchronous 16-byte copies
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes = 16u) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds_u128(const void* p) {       // ordered shared-memory load
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(p)) : "memory");
+  return v;
+}
+
 // Arguments of the verify kernels (all thread-count variants).
 struct VerifyArgs {
   const void *tc, *tu, *dc, *du;

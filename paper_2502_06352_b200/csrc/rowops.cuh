@@ -13,6 +13,9 @@ template <> struct Vec<float> {
   __device__ static __forceinline__ void unpack(const V& v, float (&f)[4]) {
     f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
   }
+  __device__ static __forceinline__ void unpack_raw(const uint4& v, float (&f)[4]) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
   __device__ static __forceinline__ float widen(float x) { return x; }
 };
 template <> struct Vec<__nv_bfloat16> {
@@ -26,6 +29,7 @@ template <> struct Vec<__nv_bfloat16> {
       f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
     }
   }
+  __device__ static __forceinline__ void unpack_raw(const uint4& v, float (&f)[8]) { unpack(v, f); }
   __device__ static __forceinline__ float widen(__nv_bfloat16 x) { return __bfloat162float(x); }
 };
 

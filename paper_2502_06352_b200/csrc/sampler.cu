@@ -66,16 +66,19 @@ __global__ void __launch_bounds__(VT, 1) sample_children_kernel(const SampleArgs
   constexpr int NV4 = E / 4;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* Z = reinterpret_cast<float*>(smem_raw);
-  float* K = Z + SL;
+  float* K = Z + SL;                                    // keys; first the uncond staging buffer
+  unsigned char* nxt = reinterpret_cast<unsigned char*>(K + SL);
   TopkSmem tk;
-  tk.bins = reinterpret_cast<uint32_t*>(K + SL);
-  tk.gbins = tk.bins + 2 * kBins;
-  tk.wl = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
-  tk.comp = tk.wl + 2 * kCandLocal;
+  tk.gbins = reinterpret_cast<uint32_t*>(nxt);
+  tk.comp = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
   tk.all = tk.comp + 2 * kCandLocal;
+  nxt += kScratchBytes;
+  tk.bins = reinterpret_cast<uint32_t*>(nxt);
+  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
+  tk.wcnt = reinterpret_cast<int*>(tk.wl + 2 * kCandLocal);
+  tk.wtot = reinterpret_cast<uint32_t*>(tk.wcnt + 2 * VW);
   VCtx c;
-  tk.wcnt = reinterpret_cast<int*>(tk.all + 2 * kCandTotal);
-  c.red = reinterpret_cast<float*>(tk.wcnt + 2 * VW);
+  c.red = reinterpret_cast<float*>(tk.wtot + 2 * (kBins / 32));
   c.xch = c.red + 2 * VW * 4;
   c.gath = c.xch + 8;
   tk.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
@@ -98,9 +101,13 @@ __global__ void __launch_bounds__(VT, 1) sample_children_kernel(const SampleArgs
 
   const bool masked = a.allow_lo > 0 || a.allow_hi < a.V;
   float mx[2];
-  mx[0] = load_row<T, CFG, E>(static_cast<const T*>(a.dc) + row_off,
-                              CFG ? static_cast<const T*>(a.du) + row_off : nullptr, a.g, a.inv_tau, lo, len,
-                              a.allow_lo, a.allow_hi, masked, Z);
+  const T* dcp = static_cast<const T*>(a.dc) + row_off;
+  const T* dup = CFG ? static_cast<const T*>(a.du) + row_off : nullptr;
+  issue_row<T, E>(dcp, lo, len, Z);
+  if (CFG) issue_row<T, E>(dup, lo, len, K);
+  cp_async_commit();
+  cp_async_wait<0>();
+  mx[0] = finish_row<T, CFG, E>(dcp, dup, a.g, a.inv_tau, lo, len, a.allow_lo, a.allow_hi, masked, Z, K);
   mx[1] = -INFINITY;
   row_reduce<2, true>(c, mx);
   if (mx[0] == -INFINITY) {
@@ -211,7 +218,7 @@ static bool sampler_shape(int V, int rows, int min_e, int override_cs, int* cs_o
     *cs_out = cs_for(e);
   }
   *e_out = e;
-  *smem_out = static_cast<size_t>(2) * VT * e * 4 + kVerifyFixedSmem;
+  *smem_out = static_cast<size_t>(2) * VT * e * 4 + kScratchBytes + kSmallSmem;
   return *smem_out <= 227 * 1024;
 }
 

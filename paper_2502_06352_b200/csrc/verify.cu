@@ -129,12 +129,12 @@ extern "C" lantern_status lantern_verify_tree(
   const int min_e = f32 ? 4 : 8, rows = batch * t->n_nodes;
   cudaError_t e;
   v1024::LaunchShape s1;
-  const bool ok1 = v1024::choose_shape(V, rows, t->max_children, a.kpad, min_e, &s1);
+  const bool ok1 = v1024::choose_shape(V, rows, t->max_children, a.kpad, min_e, cfg, &s1);
   if (ok1 && s1.cs == 1) {
     e = v1024::launch_any(a, s1, f32, cfg, st);
   } else {
     v512::LaunchShape s5;
-    if (v512::choose_shape(V, rows, t->max_children, a.kpad, min_e, &s5)) {
+    if (v512::choose_shape(V, rows, t->max_children, a.kpad, min_e, cfg, &s5)) {
       e = v512::launch_any(a, s5, f32, cfg, st);
     } else if (ok1) {
       e = v1024::launch_any(a, s1, f32, cfg, st);

@@ -36,12 +36,20 @@ constexpr int kCandTotal = 1024;  // and the whole cluster
 
 constexpr int kMiscInts = 16;
 constexpr int kCntInts = 2 + 2 * kMaxCluster + 2;
-// fixed part of the dynamic shared memory behind the two row slices
-constexpr int kVerifyFixedSmem = 4 * kBins * 4 + 4 * kCandLocal * 4 + 2 * kCandTotal * 4 + 2 * VW * 4   // top-k
-                                 + 2 * VW * 4 * 4      // red (two buffers)
-                                 + 2 * 4 * 4           // xch
-                                 + kMaxCluster * 4 * 4 // gath
-                                 + 8 * 4 + kCntInts * 4 + kMiscInts * 4 + 16;
+// Dynamic shared memory: [Q][P]([U] with guidance) [scratch] [small] [neighbour rows].
+// scratch = buffers that only the top-k routine needs while the rows still hold pre-softmax
+// values (row-wide bins, compacted and gathered candidates); with guidance it aliases U, which is
+// dead once the rows are loaded, when U is large enough.
+constexpr int kScratchBytes = 2 * kBins * 4 + 2 * kCandLocal * 4 + 2 * kCandTotal * 4;
+constexpr int kSmallSmem = 2 * kBins * 4 + 2 * kCandLocal * 4 + 2 * VW * 4 + 2 * (kBins / 32) * 4   // bins, lists, counts, block totals
+                           + 2 * VW * 4 * 4      // red (two buffers)
+                           + 2 * 4 * 4           // xch
+                           + kMaxCluster * 4 * 4 // gath
+                           + 8 * 4 + kCntInts * 4 + kMiscInts * 4 + 16;
+__host__ __device__ constexpr bool scratch_aliases_u(bool cfg, int e) { return cfg && VT * e * 4 >= kScratchBytes; }
+__host__ __device__ constexpr size_t row_smem_bytes(bool cfg, int e) {
+  return static_cast<size_t>(cfg ? 3 : 2) * VT * e * 4 + (scratch_aliases_u(cfg, e) ? 0 : kScratchBytes) + kSmallSmem;
+}
 
 struct VCtx {
   uint32_t rank, nrank;
@@ -102,25 +110,36 @@ __device__ __forceinline__ void row_reduce(VCtx& c, float (&v)[NV]) {
   c.parity ^= 1;
 }
 
-// Pre-softmax values of one row slice -> shared memory (entries beyond the row end and
-// outside the allowed token range become -inf).  Returns this thread's maximum.
-template <typename T, bool CFG, int E>
-__device__ __forceinline__ float load_row(const T* __restrict__ cond, const T* __restrict__ uncond, float g,
-                                          float inv_tau, int lo, int len, int allow_lo, int allow_hi,
-                                          bool masked, float* __restrict__ dst) {
-  using VTT = Vec<T>;
-  constexpr int VN = VTT::N, NV = E / VN;
+// Loading a row slice is split in two so that several operands can be in flight at once:
+// issue_row starts asynchronous 16-byte copies of this thread's chunks of one operand straight
+// into shared memory (no registers are held), finish_row turns the landed chunks into
+// pre-softmax values in place.  A thread only ever touches the chunks it issued itself, so the
+// two need no block-wide barrier between them, only the thread's own cp.async wait.
+// float32 chunks land where their 4 values will live; bfloat16 chunks (8 values, 16 bytes) land
+// in the upper half of the 32 bytes their 8 float32 values will occupy.
+template <typename T, int E>
+__device__ __forceinline__ void issue_row(const T* __restrict__ src, int lo, int len, float* __restrict__ dst) {
+  constexpr int VN = Vec<T>::N, NV = E / VN;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int wb = warp * 32 * E + lane * VN;
-  typename VTT::V cr[NV], ur[NV];
 #pragma unroll
   for (int v = 0; v < NV; ++v) {
     const int j = wb + v * 32 * VN;
-    if (j + VN <= len) {
-      cr[v] = __ldcs(reinterpret_cast<const typename VTT::V*>(cond + lo + j));
-      if (CFG) ur[v] = __ldcs(reinterpret_cast<const typename VTT::V*>(uncond + lo + j));
-    }
+    if (j + VN <= len) cp_async16(smem_u32(dst + j + (VN == 8 ? 4 : 0)), src + lo + j);
   }
+}
+
+// Pre-softmax values of one row slice, in place (entries beyond the row end and outside the
+// allowed token range become -inf).  `dst` holds the landed cond chunks, `ubuf` the uncond
+// chunks; the ragged last vector of a row is read with scalar loads.  Returns this thread's max.
+template <typename T, bool CFG, int E>
+__device__ __forceinline__ float finish_row(const T* __restrict__ cond, const T* __restrict__ uncond, float g,
+                                            float inv_tau, int lo, int len, int allow_lo, int allow_hi,
+                                            bool masked, float* __restrict__ dst, const float* __restrict__ ubuf) {
+  using VTT = Vec<T>;
+  constexpr int VN = VTT::N, NV = E / VN, OFF = (VN == 8 ? 4 : 0);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int wb = warp * 32 * E + lane * VN;
   float mx = -INFINITY;
 #pragma unroll
   for (int v = 0; v < NV; ++v) {
@@ -128,8 +147,12 @@ __device__ __forceinline__ float load_row(const T* __restrict__ cond, const T* _
     float zf[VN];
     if (j + VN <= len) {
       float cf[VN], uf[VN];
-      VTT::unpack(cr[v], cf);
-      if (CFG) VTT::unpack(ur[v], uf);
+      const uint4 cr = lds_u128(dst + j + OFF);
+      VTT::unpack_raw(cr, cf);
+      if (CFG) {
+        const uint4 ur = lds_u128(ubuf + j + OFF);
+        VTT::unpack_raw(ur, uf);
+      }
 #pragma unroll
       for (int e = 0; e < VN; ++e) zf[e] = combine<CFG>(cf[e], CFG ? uf[e] : 0.f, g, inv_tau);
     } else {
@@ -170,6 +193,7 @@ struct TopkSmem {
   uint32_t* gbins;  // [2][kBins]  bins of the whole row (clusters only)
   float* wl;        // [2][VW][kCandLocal/VW] per-warp candidate lists
   float* comp;      // [2][kCandLocal]   compacted candidates
+  uint32_t* wtot;   // [2][kBins/32] inclusive totals of 32-bin blocks
   float* all;       // [2][kCandTotal]
   int* wcnt;        // [2][VW]
   int* sel;         // [8]
@@ -223,7 +247,7 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
     constexpr int RPT = 2 * kBins / VT;
     constexpr int WPR = kBins / 32;                            // warps' worth of bins per row
     uint32_t cnt[RPT], incl[RPT];
-    uint32_t* wtot = reinterpret_cast<uint32_t*>(s.all);       // [2 * WPR] inclusive totals
+    uint32_t* wtot = s.wtot;                                   // [2 * WPR] inclusive totals
 #pragma unroll
     for (int it = 0; it < RPT; ++it) {
       const int g = it * VT + tid, r = g / kBins;
@@ -474,15 +498,20 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* Q = reinterpret_cast<float*>(smem_raw);
   float* P = Q + SL;
+  float* U = P + SL;                                   // uncond staging (guidance only)
+  unsigned char* nxt = reinterpret_cast<unsigned char*>(P + (CFG ? 2 : 1) * SL);
+  unsigned char* scratch = reinterpret_cast<unsigned char*>(U);
+  if (!scratch_aliases_u(CFG, E)) { scratch = nxt; nxt += kScratchBytes; }
   TopkSmem tk;
-  tk.bins = reinterpret_cast<uint32_t*>(P + SL);
-  tk.gbins = tk.bins + 2 * kBins;
-  tk.wl = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
-  tk.comp = tk.wl + 2 * kCandLocal;
+  tk.gbins = reinterpret_cast<uint32_t*>(scratch);
+  tk.comp = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
   tk.all = tk.comp + 2 * kCandLocal;
+  tk.bins = reinterpret_cast<uint32_t*>(nxt);
+  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
+  tk.wcnt = reinterpret_cast<int*>(tk.wl + 2 * kCandLocal);
+  tk.wtot = reinterpret_cast<uint32_t*>(tk.wcnt + 2 * VW);
   VCtx c;
-  tk.wcnt = reinterpret_cast<int*>(tk.all + 2 * kCandTotal);
-  c.red = reinterpret_cast<float*>(tk.wcnt + 2 * VW);
+  c.red = reinterpret_cast<float*>(tk.wtot + 2 * (kBins / 32));
   c.xch = c.red + 2 * VW * 4;
   c.gath = c.xch + 8;
   tk.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
@@ -564,17 +593,31 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
     reinterpret_cast<float*>(misc)[8 + tid] = u;
   }
 
-  // ---- read the rows once: z_q -> Q, z_p -> P
+  // ---- read the rows once: every operand is copied asynchronously straight into shared
+  // memory, target cond / uncond and drafter cond all in flight together; the drafter's uncond
+  // row follows as soon as this thread has consumed its target chunks of U
   const bool masked = a.allow_lo > 0 || a.allow_hi < a.V;
+  const T* tc = static_cast<const T*>(a.tc) + row_off;
+  const T* tu = CFG ? static_cast<const T*>(a.tu) + row_off : nullptr;
+  const T* dc = nc > 0 ? static_cast<const T*>(a.dc) + row_off : nullptr;
+  const T* du = (CFG && nc > 0) ? static_cast<const T*>(a.du) + row_off : nullptr;
+  issue_row<T, E>(tc, lo, len, Q);
+  if (CFG) issue_row<T, E>(tu, lo, len, U);
+  cp_async_commit();
+  if (nc > 0) issue_row<T, E>(dc, lo, len, P);
+  cp_async_commit();
+  cp_async_wait<1>();
   float mx[2];
-  mx[0] = load_row<T, CFG, E>(static_cast<const T*>(a.tc) + row_off,
-                              CFG ? static_cast<const T*>(a.tu) + row_off : nullptr, a.g, a.inv_tau, lo, len,
-                              a.allow_lo, a.allow_hi, masked, Q);
+  mx[0] = finish_row<T, CFG, E>(tc, tu, a.g, a.inv_tau, lo, len, a.allow_lo, a.allow_hi, masked, Q, U);
   mx[1] = -INFINITY;
-  if (nc > 0)
-    mx[1] = load_row<T, CFG, E>(static_cast<const T*>(a.dc) + row_off,
-                                CFG ? static_cast<const T*>(a.du) + row_off : nullptr, a.g, a.inv_tau, lo, len,
-                                a.allow_lo, a.allow_hi, masked, P);
+  if (nc > 0) {
+    if (CFG) {
+      issue_row<T, E>(du, lo, len, U);
+      cp_async_commit();
+    }
+    cp_async_wait<0>();
+    mx[1] = finish_row<T, CFG, E>(dc, du, a.g, a.inv_tau, lo, len, a.allow_lo, a.allow_hi, masked, P, U);
+  }
   row_reduce<2, true>(c, mx);
   if (mx[0] == -INFINITY || (nc > 0 && mx[1] == -INFINITY)) {
     if (tid == 0 && c.rank == 0) vflag(a.status, LANTERN_DEV_EMPTY_ROW);

@@ -8,9 +8,9 @@ constexpr int kMaxE = 16384 / VT;      // a CTA's slice holds at most 16384 row 
 
 // Choose E (row entries per thread; a CTA's slice is 1024*E entries) and the cluster size.
 // `min_e` is 4 for float32 rows and 8 for bfloat16 rows (one 16-byte vector per thread).
-static bool choose_shape(int V, int rows, int max_children, int kpad, int min_e, LaunchShape* out) {
+static bool choose_shape(int V, int rows, int max_children, int kpad, int min_e, bool cfg, LaunchShape* out) {
   auto smem_for = [&](int e) {
-    return static_cast<size_t>(2) * VT * e * 4 + kVerifyFixedSmem + static_cast<size_t>(max_children) * kpad * 4;
+    return row_smem_bytes(cfg, e) + static_cast<size_t>(max_children) * kpad * 4;
   };
   auto cs_for = [&](int e) { int cs = (V + VT * e - 1) / (VT * e); return cs > 8 ? (cs > 16 ? 0 : 16) : cs; };
   int e = 0;
@@ -27,6 +27,8 @@ static bool choose_shape(int V, int rows, int max_children, int kpad, int min_e,
     if (cs_for(e) == 0) return false;
     // few rows: split each over more CTAs so that more SMs stream
     while (e > min_e && static_cast<long long>(rows) * cs_for(e) < 74 && cs_for(e / 2) != 0 && cs_for(e / 2) <= 8) e /= 2;
+    // shared memory: halve the slice (more CTAs per row) until the CTA fits
+    while (smem_for(e) > 227 * 1024 && e > min_e && cs_for(e / 2) != 0) e /= 2;
     out->cs = cs_for(e);
   }
   out->e = e;
