@@ -159,6 +159,7 @@ struct VerifyArgs {
   int32_t *node_next, *node_token;
   float *node_mass, *node_thresh;
   int32_t* status;
+  const int32_t* only;     // [B*N] or NULL: process only the nodes whose entry is non-zero
 };
 
 }  // namespace lantern

@@ -41,4 +41,57 @@ __device__ __forceinline__ float combine(float c, float u, float g, float inv_ta
   return __fmul_rn(c, inv_tau);
 }
 
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ void vflag(int32_t* status, int bit) {
+  if (status) atomicOr(status, bit);
+}
+
+// ---- histogram bins of the top-k locator: a monotone, coarse position of an entry below the
+// row maximum (128 bins per binade of d = max - z, 16 binades: d in [2^-9, 2^7), clamped)
+constexpr int kBins = 2048;
+constexpr int kBinLog = 7;
+constexpr int kBinShift = 23 - kBinLog;
+constexpr int kBinBase = (127 - 9) << kBinLog;
+__device__ __forceinline__ int dist_bin(float mx, float z) {
+  const float d = mx - z;
+  const int b = static_cast<int>(__float_as_uint(d) >> kBinShift) - kBinBase;
+  return min(max(b, 0), kBins - 1);
+}
+// bit patterns of d that fall into bin b: [bin_lo_bits(b), bin_hi_bits(b)] (the end bins are open)
+__device__ __forceinline__ uint32_t bin_lo_bits(int b) {
+  return b == 0 ? 0u : static_cast<uint32_t>(b + kBinBase) << kBinShift;
+}
+__device__ __forceinline__ uint32_t bin_hi_bits(int b) {
+  return b == kBins - 1 ? 0xffffffffu : (static_cast<uint32_t>(b + kBinBase + 1) << kBinShift) - 1u;
+}
+
+// ---- bounded wait on an mbarrier phase; false when the limit was reached
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t phase) {
+  for (int it = 0; it < (1 << 22); ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(mbar), "r"(phase) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+// 16-byte streaming load (read once: no L1 allocation)
+__device__ __forceinline__ uint4 ldg_stream_u128(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
 }  // namespace lantern

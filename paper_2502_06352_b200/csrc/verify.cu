@@ -3,6 +3,18 @@
 
 namespace lantern {
 static int g_cluster_override = 0;
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      n = v;
+    else
+      return 148;
+  }
+  return n;
+}
 }
 
 // two builds of the kernels: 1024 threads per CTA for rows that fit one CTA, 512 threads per CTA
@@ -19,8 +31,31 @@ static int g_cluster_override = 0;
 #include "verify_launch.cuh"
 #undef LANTERN_VT
 #undef LANTERN_VNS
+#include "verify_sparse.cuh"
 
 namespace lantern {
+
+// ---- launch of the sparse (top-k) kernel: one CTA per node
+template <typename T, bool CFG, int E>
+static cudaError_t launch_sparse_e(const VerifyArgs& a, int32_t* redo, size_t smem, cudaStream_t st) {
+  auto kern = sparse::verify_sparse_kernel<T, CFG, E>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  kern<<<static_cast<unsigned>(a.B) * a.N, sparse::ST, smem, st>>>(a, redo);
+  return cudaGetLastError();
+}
+template <typename T, bool CFG>
+static cudaError_t launch_sparse(const VerifyArgs& a, int32_t* redo, int e, size_t smem, cudaStream_t st) {
+  if (e == 8) return launch_sparse_e<T, CFG, 8>(a, redo, smem, st);
+  if (e == 16) return launch_sparse_e<T, CFG, 16>(a, redo, smem, st);
+  return launch_sparse_e<T, CFG, 32>(a, redo, smem, st);
+}
+static cudaError_t launch_sparse_any(const VerifyArgs& a, int32_t* redo, int e, size_t smem, bool f32, bool cfg,
+                                     cudaStream_t st) {
+  if (f32) return cfg ? launch_sparse<float, true>(a, redo, e, smem, st) : launch_sparse<float, false>(a, redo, e, smem, st);
+  return cfg ? launch_sparse<__nv_bfloat16, true>(a, redo, e, smem, st)
+             : launch_sparse<__nv_bfloat16, false>(a, redo, e, smem, st);
+}
 
 // ---- walk (Sec. 2.1): follow accepted children from the root
 __global__ void walk_kernel(const int32_t* __restrict__ node_next, const int32_t* __restrict__ node_token,
@@ -64,7 +99,7 @@ extern "C" int32_t lantern_set_cluster_size(int32_t ctas_per_row) {
 extern "C" size_t lantern_verify_tree_workspace(const lantern_tree* tree, int32_t batch) {
   if (!tree || batch <= 0) return 0;
   const TreeDev* t = reinterpret_cast<const TreeDev*>(tree);
-  return static_cast<size_t>(2) * batch * t->n_nodes * sizeof(int32_t);
+  return static_cast<size_t>(3) * batch * t->n_nodes * sizeof(int32_t);     // node_next, node_token, repair flags
 }
 
 extern "C" lantern_status lantern_verify_tree(
@@ -98,13 +133,15 @@ extern "C" lantern_status lantern_verify_tree(
     if (q && (reinterpret_cast<uintptr_t>(q) % 16)) return LANTERN_ERR_INVALID_ARG;
   if (static_cast<int64_t>(batch) * t->n_nodes > (1 << 24)) return LANTERN_ERR_UNSUPPORTED;
 
+  const size_t ws_need = lantern_verify_tree_workspace(tree, batch);
+  const bool have_ws = workspace && workspace_bytes >= ws_need && (reinterpret_cast<uintptr_t>(workspace) % 256) == 0;
   if (!node_next || !node_token) {
-    size_t need = lantern_verify_tree_workspace(tree, batch);
-    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) % 256)) return LANTERN_ERR_WORKSPACE;
+    if (!have_ws) return LANTERN_ERR_WORKSPACE;
     int32_t* w = static_cast<int32_t*>(workspace);
     if (!node_next) node_next = w;
     if (!node_token) node_token = w + static_cast<size_t>(batch) * t->n_nodes;
   }
+  int32_t* redo = have_ws ? static_cast<int32_t*>(workspace) + static_cast<size_t>(2) * batch * t->n_nodes : nullptr;
 
   VerifyArgs a;
   a.tc = target_cond; a.tu = target_uncond; a.dc = draft_cond; a.du = draft_uncond;
@@ -121,13 +158,25 @@ extern "C" lantern_status lantern_verify_tree(
   a.seed = p->seed; a.step = p->step;
   a.node_next = node_next; a.node_token = node_token; a.node_mass = node_mass; a.node_thresh = node_thresh;
   a.status = device_status;
-  // rows that fit one CTA run the 1024-thread build; rows split over a cluster run the
-  // 512-thread build (cheaper barriers, half the per-thread fixed work per entry)
+  a.only = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = target_uncond != nullptr;
   const bool f32 = dt == LANTERN_F32;
   const int min_e = f32 ? 4 : 8, rows = batch * t->n_nodes;
   cudaError_t e;
+  // Rows truncated to a moderate top-k on every side that is read take the sparse kernel; the
+  // dense kernel then repairs the nodes it could not hold (a.only) and usually finds none.
+  auto topk_fits = [&](int k) { return k > 0 && k < V && k <= sparse::kMaxTopK; };
+  const bool use_sparse = redo && g_cluster_override == 0 && V <= sparse::kMaxV && topk_fits(p->top_k_target) &&
+                          (t->n_internal == 0 || topk_fits(p->top_k_draft)) && t->max_children <= 20;
+  if (use_sparse) {
+    const int se = V <= sparse::ST * 8 ? 8 : (V <= sparse::ST * 16 ? 16 : 32);
+    e = launch_sparse_any(a, redo, se, sparse::smem_bytes(se, t->max_children, a.kpad), f32, cfg, st);
+    if (e != cudaSuccess) return LANTERN_ERR_CUDA;
+    a.only = redo;
+  }
+  // rows that fit one CTA run the 1024-thread build; rows split over a cluster run the
+  // 512-thread build (cheaper barriers, half the per-thread fixed work per entry)
   v1024::LaunchShape s1;
   const bool ok1 = v1024::choose_shape(V, rows, t->max_children, a.kpad, min_e, cfg, &s1);
   if (ok1 && s1.cs == 1) {
@@ -156,7 +205,7 @@ extern "C" lantern_status lantern_verify_tree(
 // that is part of the library image; every GPU that loads the library holds it until exit.
 namespace {
 constexpr int kStaticMaxNodes = 1 << 16;       // batch * tree nodes the built-in scratch can hold
-static __device__ __align__(256) int32_t g_static_scratch[2 * kStaticMaxNodes];
+static __device__ __align__(256) int32_t g_static_scratch[3 * kStaticMaxNodes];
 constexpr int kMaxDevices = 64;
 void* g_static_scratch_ptr[kMaxDevices] = {};  // device address of the array, per device
 
@@ -194,5 +243,5 @@ extern "C" lantern_status lantern_verify_tree_static(
   return lantern_verify_tree(p, tree, nbr_idx, k_table, target_cond, target_uncond, draft_cond, draft_uncond, dt,
                              row_stride, seq_stride, batch, tokens, u_accept, u_resample, accept_len, out_tokens,
                              out_nodes, nullptr, nullptr, node_mass, node_thresh, device_status, scratch,
-                             sizeof(int32_t) * 2 * kStaticMaxNodes, stream);
+                             sizeof(int32_t) * 3 * kStaticMaxNodes, stream);
 }

@@ -24,11 +24,6 @@ namespace LANTERN_VNS {
 
 constexpr int VT = LANTERN_VT;    // threads per CTA (1024 or 512)
 constexpr int VW = VT / 32;       // warps per CTA
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kBins = 2048;       // histogram bins of the top-k locator
-constexpr int kBinLog = 7;        // log2 of the bins per binade of d = max - z
-constexpr int kBinShift = 23 - kBinLog;
-constexpr int kBinBase = (127 - 9) << kBinLog;        // 16 binades: d in [2^-9, 2^7)
 static_assert(VT == 1024 || VT == 512, "thread count");
 constexpr int kCandLocal = 512;   // top-k candidates one CTA may contribute per row
 constexpr int kCandTotal = 1024;  // and the whole cluster
@@ -59,16 +54,6 @@ struct VCtx {
   float* gath;     // [kMaxCluster*4] per-rank values of the last reduction
   float* last_red; // red buffer of the last reduction (per-warp values)
 };
-
-__device__ __forceinline__ void vflag(int32_t* status, int bit) {
-  if (status) atomicOr(status, bit);
-}
-
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 
 __device__ __forceinline__ void csync(const VCtx& c) {       // whole row: block or cluster
   if (c.nrank > 1) cluster_sync(); else __syncthreads();
@@ -179,13 +164,6 @@ __device__ __forceinline__ float finish_row(const T* __restrict__ cond, const T*
     for (int e = 0; e < VN; e += 4) d4[e / 4] = make_float4(zf[e], zf[e + 1], zf[e + 2], zf[e + 3]);
   }
   return mx;
-}
-
-// Coarse position of an entry below the row maximum: a monotone function of z.
-__device__ __forceinline__ int dist_bin(float mx, float z) {
-  const float d = mx - z;
-  const int b = static_cast<int>(__float_as_uint(d) >> kBinShift) - kBinBase;
-  return min(max(b, 0), kBins - 1);
 }
 
 struct TopkSmem {
@@ -473,59 +451,14 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
 }
 
 
-// ---- bounded wait on an mbarrier phase; false when the limit was reached
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t phase) {
-  for (int it = 0; it < (1 << 22); ++it) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(mbar), "r"(phase) : "memory");
-    if (ok) return true;
-  }
-  return false;
-}
-
-// E = row entries per thread; the CTA's slice holds SL = 1024 * E entries.
-#ifndef LANTERN_MINB
-#define LANTERN_MINB 1
-#endif
+// One tree node: rows into shared memory, post-processing, sibling loop, resampling.
 template <typename T, bool CFG, int E>
-__global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const VerifyArgs a) {
+__device__ __forceinline__ void verify_node(const VerifyArgs& a, const int idx, VCtx& c, const TopkSmem& tk,
+                                            float* __restrict__ Q, float* __restrict__ P, float* __restrict__ U,
+                                            int* misc, const uint32_t mbar_a, uint32_t& mphase, int* nbr_s) {
   constexpr int SL = VT * E;
   constexpr int NV4 = E / 4;                 // float4 per thread in a shared-memory sweep
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* Q = reinterpret_cast<float*>(smem_raw);
-  float* P = Q + SL;
-  float* U = P + SL;                                   // uncond staging (guidance only)
-  unsigned char* nxt = reinterpret_cast<unsigned char*>(P + (CFG ? 2 : 1) * SL);
-  unsigned char* scratch = reinterpret_cast<unsigned char*>(U);
-  if (!scratch_aliases_u(CFG, E)) { scratch = nxt; nxt += kScratchBytes; }
-  TopkSmem tk;
-  tk.gbins = reinterpret_cast<uint32_t*>(scratch);
-  tk.comp = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
-  tk.all = tk.comp + 2 * kCandLocal;
-  tk.bins = reinterpret_cast<uint32_t*>(nxt);
-  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
-  tk.wcnt = reinterpret_cast<int*>(tk.wl + 2 * kCandLocal);
-  tk.wtot = reinterpret_cast<uint32_t*>(tk.wcnt + 2 * VW);
-  VCtx c;
-  c.red = reinterpret_cast<float*>(tk.wtot + 2 * (kBins / 32));
-  c.xch = c.red + 2 * VW * 4;
-  c.gath = c.xch + 8;
-  tk.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
-  tk.cnts = tk.sel + 8;
-  int* misc = tk.cnts + kCntInts;
-  uint64_t* mbar = reinterpret_cast<uint64_t*>(misc + kMiscInts);
-  int* nbr_s = reinterpret_cast<int*>(mbar + 2);
-  c.rank = cluster_ctarank();
-  c.nrank = cluster_nctarank();
-  c.parity = 0;
-  c.last_red = c.red;
-
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int idx = blockIdx.x / c.nrank;
   const int b = idx % a.B;
   const int n = a.order[idx / a.B];
   const int fc = a.first_child[n], nc = a.n_child[n];
@@ -539,12 +472,9 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
 
   // ---- stage the children's neighbour rows (bulk async copy when rows are 16-byte aligned)
   const bool want_nbr = nc > 0 && a.k > 0;
-  const uint32_t mbar_a = smem_u32(mbar);
   bool bulk_issued = false;
   if (want_nbr && a.use_bulk) {
     if (tid == 0) {
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar_a) : "memory");
-      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       uint32_t bytes = 0;
       const uint32_t row_bytes = static_cast<uint32_t>(((a.k + 3) & ~3) * 4);
       for (int ci = 0; ci < nc; ++ci) {
@@ -673,7 +603,8 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
 
   // ---- neighbour rows must have landed
   if (bulk_issued) {
-    bool ok = mbar_wait_bounded(mbar_a, 0);
+    bool ok = mbar_wait_bounded(mbar_a, mphase);
+    mphase ^= 1u;
     if (!__syncthreads_and(ok)) {
       if (tid == 0) vflag(a.status, LANTERN_DEV_TIMEOUT);
       for (int ci = 0; ci < nc; ++ci) {
@@ -916,7 +847,66 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
     a.node_token[out_b + n] = -1;
   }
   if (c.rank == 0 && tid == 0) a.node_next[out_b + n] = accepted;
-  if (!single) cluster_sync();    // peers may still be reading this CTA's shared memory
+}
+
+// E = row entries per thread; the CTA's slice holds SL = 1024 * E entries.
+#ifndef LANTERN_MINB
+#define LANTERN_MINB 1
+#endif
+template <typename T, bool CFG, int E>
+__global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const VerifyArgs a) {
+  constexpr int SL = VT * E;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* Q = reinterpret_cast<float*>(smem_raw);
+  float* P = Q + SL;
+  float* U = P + SL;                                   // uncond staging (guidance only)
+  unsigned char* nxt = reinterpret_cast<unsigned char*>(P + (CFG ? 2 : 1) * SL);
+  unsigned char* scratch = reinterpret_cast<unsigned char*>(U);
+  if (!scratch_aliases_u(CFG, E)) { scratch = nxt; nxt += kScratchBytes; }
+  TopkSmem tk;
+  tk.gbins = reinterpret_cast<uint32_t*>(scratch);
+  tk.comp = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
+  tk.all = tk.comp + 2 * kCandLocal;
+  tk.bins = reinterpret_cast<uint32_t*>(nxt);
+  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
+  tk.wcnt = reinterpret_cast<int*>(tk.wl + 2 * kCandLocal);
+  tk.wtot = reinterpret_cast<uint32_t*>(tk.wcnt + 2 * VW);
+  VCtx c;
+  c.red = reinterpret_cast<float*>(tk.wtot + 2 * (kBins / 32));
+  c.xch = c.red + 2 * VW * 4;
+  c.gath = c.xch + 8;
+  tk.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
+  tk.cnts = tk.sel + 8;
+  int* misc = tk.cnts + kCntInts;
+  uint64_t* mbar = reinterpret_cast<uint64_t*>(misc + kMiscInts);
+  int* nbr_s = reinterpret_cast<int*>(mbar + 2);
+  c.rank = cluster_ctarank();
+  c.nrank = cluster_nctarank();
+  c.parity = 0;
+  c.last_red = c.red;
+
+  const int tid = threadIdx.x;
+  const uint32_t mbar_a = smem_u32(mbar);
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar_a) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  uint32_t mphase = 0;
+  // A regular launch has one CTA (cluster) per node.  A repair launch (a.only given) has fewer:
+  // cluster g of G takes the flagged nodes idx = g (mod G) one after another, and leaves at once
+  // when none of them is flagged.
+  const int rows = a.B * a.N, G = gridDim.x / c.nrank, g0 = blockIdx.x / c.nrank;
+  if (a.only) {
+    bool any = false;
+    for (long long i = g0 + static_cast<long long>(tid) * G; i < rows; i += static_cast<long long>(VT) * G)
+      any |= a.only[i] != 0;
+    if (!__syncthreads_or(any)) return;      // the same flags, hence the same decision, in every CTA of a cluster
+  }
+  for (int idx = g0; idx < rows; idx += G) {
+    if (a.only && a.only[idx] == 0) continue;
+    verify_node<T, CFG, E>(a, idx, c, tk, Q, P, U, misc, mbar_a, mphase, nbr_s);
+    csync(c);     // peers may still be reading this CTA's shared memory; the next node overwrites it
+  }
 }
 
 }  // namespace LANTERN_VNS

@@ -46,7 +46,14 @@ static cudaError_t launch_verify_e(const VerifyArgs& a, const LaunchShape& sh, c
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(a.B) * a.N * sh.cs, 1, 1);
+  // one cluster per node; a repair launch (a.only) gets about one cluster per SM and lets each
+  // walk its share of the flagged nodes
+  unsigned clusters = static_cast<unsigned>(a.B) * a.N;
+  if (a.only) {
+    const unsigned per_wave = static_cast<unsigned>(sm_count() / sh.cs > 0 ? sm_count() / sh.cs : 1);
+    if (clusters > per_wave) clusters = per_wave;
+  }
+  cfg.gridDim = dim3(clusters * sh.cs, 1, 1);
   cfg.blockDim = dim3(VT, 1, 1);
   cfg.dynamicSmemBytes = sh.smem;
   cfg.stream = st;

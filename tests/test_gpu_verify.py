@@ -56,6 +56,42 @@ def test_parameter_variants(L, kw):
     _run(L, case)
 
 
+@pytest.mark.parametrize("cs", [0, 1, 2])
+@pytest.mark.parametrize("kw", [
+    dict(vocab=3001, codebook_size=3001, top_k=200, k=12),
+    dict(vocab=9000, codebook_size=2000, code_offset=500, top_k=1000, k=20, dtype="bf16", cfg_scale=None),
+])
+def test_topk_rows_on_every_path(L, cs, kw):
+    # cs = 0: the list-based top-k kernel (rows of at most 16384 entries); cs = 1, 2: the dense
+    # kernel in one CTA / a cluster of two
+    case = Case(small_config(**kw), seed=13, pad=3 if kw.get("dtype", "f32") == "f32" else 8)   # rows stay 16-byte aligned
+    old = L.set_cluster_size(cs)
+    try:
+        _run(L, case)
+    finally:
+        L.set_cluster_size(old)
+
+
+def test_topk_target_only_and_leaf_only_tree(L):
+    # top-k on the target side only: the drafter rows are dense, so the dense kernel runs
+    case = Case(small_config(top_k=0), seed=14, top_k_target=60, top_k_draft=0)
+    _run(L, case)
+    # a tree without internal nodes never reads a drafter row
+    leaf = Case(small_config(batch=3, top_k=40), parent=[-1], seed=15)
+    _run(L, leaf)
+
+
+def test_topk_with_massive_ties_is_repaired_by_the_dense_kernel(L):
+    # logits on a grid of 2.0: a handful of distinct values per row, so the k-th largest value
+    # is shared by far more entries than the list kernel's buffers hold (512 ties); those nodes
+    # must come out right all the same
+    case = Case(small_config(vocab=8000, codebook_size=1000, top_k=300, cfg_scale=None, batch=2), seed=16)
+    for v in case.padded.values():
+        if v is not None:
+            v.copy_(torch.round(v / 2.0) * 2.0)
+    _run(L, case)
+
+
 def test_allowed_range_and_topk_counts_only_allowed(L):
     case = Case(small_config(vocab=2048, codebook_size=512, code_offset=256, k=6, top_k=40), seed=3,
                 allowed=(256, 768))
