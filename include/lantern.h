@@ -148,8 +148,11 @@ lantern_status lantern_sample_draft_tree(const lantern_params* params, const lan
  *   node_mass, node_thresh [B][N] float32 m and accept probability per tested child, -1 where
  *                  a node was not tested; or NULL
  *   device_status  one int32, OR-ed with LANTERN_DEV_* bits; or NULL
- *   workspace      device scratch >= lantern_verify_tree_workspace() bytes (0 bytes needed when
- *                  node_next and node_token are both given), 256-byte aligned                    */
+ *   workspace      device scratch >= lantern_verify_tree_workspace() bytes (12 bytes per node:
+ *                  node_next, node_token and one repair flag), 256-byte aligned.  It may be
+ *                  NULL when node_next and node_token are both given; rows truncated by top-k
+ *                  then take the dense kernel instead of the faster list-based one, which needs
+ *                  the flags.                                                                    */
 size_t lantern_verify_tree_workspace(const lantern_tree* tree, int32_t batch);
 lantern_status lantern_verify_tree(const lantern_params* params, const lantern_tree* tree,
                                    const int32_t* nbr_idx, int32_t k_table,
@@ -169,9 +172,9 @@ lantern_status lantern_verify_tree(const lantern_params* params, const lantern_t
  * cannot, allocate device memory around the call: code running inside a memory pool that is
  * already fully handed out, a serving loop that forbids cudaMalloc because it synchronises the
  * device, or a host that only passes buffers it was given.  It is lantern_verify_tree with the
- * per-node scratch (accepted child and drawn token of every node, 8 bytes per node) taken from a
- * fixed array inside the library instead of a caller workspace.  The array holds
- * lantern_verify_tree_static_max_nodes() = 65536 nodes (512 KB), so batch * n_nodes must not
+ * per-node scratch (accepted child, drawn token and repair flag of every node, 12 bytes per node)
+ * taken from a fixed array inside the library instead of a caller workspace.  The array holds
+ * lantern_verify_tree_static_max_nodes() = 65536 nodes (768 KB), so batch * n_nodes must not
  * exceed that: larger calls return LANTERN_ERR_UNSUPPORTED and launch nothing.  Every GPU that
  * loads the library keeps the array until the process exits.
  *  - Nothing is allocated or freed, by this call or by anything it calls.
