@@ -61,8 +61,8 @@ constexpr int kBinShift = 23 - kBinLog;
 constexpr int kBinBase = (127 - 9) << kBinLog;
 __device__ __forceinline__ int dist_bin(float mx, float z) {
   const float d = mx - z;
-  const int b = static_cast<int>(__float_as_uint(d) >> kBinShift) - kBinBase;
-  return min(max(b, 0), kBins - 1);
+  // max(min(bits - base, last), 0) in one instruction
+  return __viaddmin_s32_relu(static_cast<int>(__float_as_uint(d) >> kBinShift), -kBinBase, kBins - 1);
 }
 // bit patterns of d that fall into bin b: [bin_lo_bits(b), bin_hi_bits(b)] (the end bins are open)
 __device__ __forceinline__ uint32_t bin_lo_bits(int b) {

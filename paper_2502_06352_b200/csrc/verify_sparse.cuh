@@ -32,12 +32,13 @@ constexpr int kMisc = 32;
 
 __host__ __device__ constexpr int z_floats(int e) { return ST * e > 3 * kUCap ? ST * e : 3 * kUCap; }
 __host__ __device__ constexpr size_t smem_bytes(int e, int max_children, int kpad) {
-  return static_cast<size_t>(z_floats(e)) * 4 + 4 * kCap * 4 + kBins * 4 + kCand * 4 + 2 * SW * 2 * 4 + SW * 4 +
-         kMisc * 4 + 16 + static_cast<size_t>(max_children) * kpad * 4;
+  return static_cast<size_t>(z_floats(e)) * 4 + 4 * kCap * 4 + kBins * 4 + 3 * kWords * 4 + kCand * 4 +
+         2 * SW * 2 * 4 + SW * 4 + kMisc * 4 + 16 + static_cast<size_t>(max_children) * kpad * 4;
 }
 
 struct Ctx {
   float* red;      // [2][SW*2]
+  float* last_red; // buffer of the last reduction: per-warp partials at [w*2 + i]
   int parity;
 };
 
@@ -55,6 +56,7 @@ __device__ __forceinline__ void block_reduce2(Ctx& c, float (&v)[2]) {
     const float t = lane < SW ? red[lane * 2 + i] : (IS_MAX ? -INFINITY : 0.f);
     v[i] = IS_MAX ? warp_max(t) : warp_sum(t);
   }
+  c.last_red = red;
   c.parity ^= 1;
 }
 
@@ -129,26 +131,31 @@ __device__ __forceinline__ float load_row(const T* __restrict__ cond, const T* _
 
 struct Smem {
   float* Z;          // [z_floats]   dense row; later the union arrays
-  int* ltok[2];      // [kCap]       survivors of the target / drafter row
+  int* ltok[2];      // [kCap]       survivors of the target / drafter row: token, pre-softmax value
   float* lval[2];
-  uint32_t* bins;    // [kBins]      later: bitmap [kWords], ranks [kWords]
+  uint32_t* bins;    // [kBins]
+  uint32_t* bm[2];   // [kWords]     support bitmaps of the two lists
+  uint32_t* rk;      // [kWords]     union entries before bitmap word w
   float* cand;       // [kCand]
   uint32_t* wtot;    // [SW]
   int* misc;         // [kMisc]
 };
 
-// Survivors of one row: every entry of Z that is >= the k-th largest becomes a list entry
-// (token, 2^((z - max) log2 e)); entries of the located bin below the threshold stay in the list
-// with value 0.  Returns false when the fixed buffers cannot hold the row.  The order of the list
+// Survivors of one row: every entry of Z in a histogram bin up to the one that holds the k-th
+// largest becomes a list entry (token, z) and a bit of the side's bitmap; theta = the exact k-th
+// largest value (ranking inside the located bin).  List entries below theta are dropped later
+// (value 0).  Returns false when the fixed buffers cannot hold the row.  The order of the list
 // depends on the order in which the warps reserve their ranges; nothing that is summed may
 // depend on it.
 template <int E>
-__device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, int kth, int& n_list) {
+__device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, int kth, int& n_list,
+                                             float& theta) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int NV4 = E / 4;
   const float* Z = s.Z;
   int* ltok = s.ltok[side];
   float* lval = s.lval[side];
+  uint32_t* bm = s.bm[side];
   // bins were cleared before the row was loaded (a barrier lies in between)
 #pragma unroll
   for (int v = 0; v < NV4; ++v) {
@@ -158,7 +165,7 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
     atomicAdd(&s.bins[dist_bin(mx, q.z)], 1u);
     atomicAdd(&s.bins[dist_bin(mx, q.w)], 1u);
   }
-  if (tid == 0) { s.misc[8] = 0; s.misc[9] = 0; }        // list and candidate counters
+  if (tid == 0) s.misc[8] = 0;                            // packed list / candidate counter
   __syncthreads();
   {
     // smallest bin whose cumulative count reaches k: thread t scans bins 4t .. 4t+3
@@ -194,47 +201,53 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
   __syncthreads();
   const int bstar = s.misc[0], krem = s.misc[1], nb = s.misc[2];
   if (nb > kCand || kth - krem + nb > kCap) return false;          // same decision in every thread
-  // Entries of the bins up to the located one -> list.  Each thread marks its entries in a bit
-  // mask, a warp reserves its range of the list with one atomic, then the marked entries are
-  // written; those of the located bin also go to the candidate array.
+  // Entries of the bins up to the located one -> list; those of the located bin also -> the
+  // candidate array.  Each thread marks its entries in two bit masks; a warp reserves its ranges
+  // of both arrays with one atomic on a packed counter (list count | candidate count << 16).
   const uint32_t hi_bits = bin_hi_bits(bstar), lo_bits = bin_lo_bits(bstar);
-  uint32_t mask = 0;
+  uint32_t mask = 0, cmask = 0;
 #pragma unroll
   for (int v = 0; v < NV4; ++v) {
     const float4 q = *reinterpret_cast<const float4*>(Z + warp * 32 * E + v * 128 + lane * 4);
-    mask |= (__float_as_uint(mx - q.x) <= hi_bits ? 1u : 0u) << (4 * v);
-    mask |= (__float_as_uint(mx - q.y) <= hi_bits ? 1u : 0u) << (4 * v + 1);
-    mask |= (__float_as_uint(mx - q.z) <= hi_bits ? 1u : 0u) << (4 * v + 2);
-    mask |= (__float_as_uint(mx - q.w) <= hi_bits ? 1u : 0u) << (4 * v + 3);
+    const float ev[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint32_t d = __float_as_uint(mx - ev[e]);
+      mask |= (d <= hi_bits ? 1u : 0u) << (4 * v + e);
+      cmask |= (d >= lo_bits ? 1u : 0u) << (4 * v + e);
+    }
   }
+  cmask &= mask;
   {
-    const int cnt = __popc(mask);
-    int incl = cnt;
+    const uint32_t cnt = static_cast<uint32_t>(__popc(mask)) | (static_cast<uint32_t>(__popc(cmask)) << 16);
+    uint32_t incl = cnt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, incl, o);
+      const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += t;
     }
-    int base = 0;
-    if (lane == 31) base = atomicAdd(&s.misc[8], incl);
-    base = __shfl_sync(0xffffffffu, base, 31);
-    int pos = base + incl - cnt;
+    uint32_t base = 0;
+    if (lane == 31) base = atomicAdd(reinterpret_cast<uint32_t*>(&s.misc[8]), incl);
+    base = __shfl_sync(0xffffffffu, base, 31) + incl - cnt;
+    int pos = static_cast<int>(base & 0xffffu), cpos = static_cast<int>(base >> 16);
     while (mask) {
       const int i = __ffs(mask) - 1;
-      mask &= mask - 1;
       const int j = warp * 32 * E + (i >> 2) * 128 + lane * 4 + (i & 3);
       const float z = Z[j];
       if (pos < kCap) { ltok[pos] = j; lval[pos] = z; }
       ++pos;
-      if (__float_as_uint(mx - z) >= lo_bits) {
-        const int cp = atomicAdd(&s.misc[9], 1);
-        if (cp < kCand) s.cand[cp] = z;
+      atomicOr(&bm[j >> 5], 1u << (j & 31));
+      if ((cmask >> i) & 1u) {
+        if (cpos < kCand) s.cand[cpos] = z;
+        ++cpos;
       }
+      mask &= mask - 1;
     }
   }
   __syncthreads();
-  n_list = min(s.misc[8], kCap);
-  const int ncand = min(s.misc[9], kCand);
+  const uint32_t packed = static_cast<uint32_t>(s.misc[8]);
+  n_list = min(static_cast<int>(packed & 0xffffu), kCap);
+  const int ncand = min(static_cast<int>(packed >> 16), kCand);
   // exact rank by counting inside the located bin: theta = v with #(> v) < krem <= #(>= v);
   // eight lanes share the comparisons of one candidate
   {
@@ -256,16 +269,9 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
     }
   }
   __syncthreads();
-  const float theta = reinterpret_cast<const float*>(s.misc)[3];
-  const float c0 = -mx * kLog2e;
-  for (int i = tid; i < n_list; i += ST) {
-    const float z = lval[i];
-    lval[i] = z >= theta ? ex2_approx(fmaf(z, kLog2e, c0)) : 0.f;
-  }
-  __syncthreads();         // the row buffer, the bins and the counters may be reused
+  theta = reinterpret_cast<const float*>(s.misc)[3];
   return true;
 }
-
 
 // E = row entries per thread (V <= 512 * E).  `redo[b*N + n]` is set to 1 when node (b, n) has to
 // be processed by the dense kernel instead, else to 0.
@@ -279,9 +285,13 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
   s.ltok[1] = reinterpret_cast<int*>(s.lval[0] + kCap);
   s.lval[1] = reinterpret_cast<float*>(s.ltok[1] + kCap);
   s.bins = reinterpret_cast<uint32_t*>(s.lval[1] + kCap);
-  s.cand = reinterpret_cast<float*>(s.bins + kBins);
+  s.bm[0] = s.bins + kBins;
+  s.bm[1] = s.bm[0] + kWords;
+  s.rk = s.bm[1] + kWords;
+  s.cand = reinterpret_cast<float*>(s.rk + kWords);
   Ctx c;
   c.red = s.cand + kCand;
+  c.last_red = c.red;
   c.parity = 0;
   s.wtot = reinterpret_cast<uint32_t*>(c.red + 2 * SW * 2);
   s.misc = reinterpret_cast<int*>(s.wtot + SW);
@@ -355,11 +365,15 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     }
     miscf[12 + tid] = u;
   }
+  static_assert(kWords == ST, "one bitmap word per thread");
+  s.bm[0][tid] = 0;
+  s.bm[1][tid] = 0;
 
   // ---- both rows, one after the other through the same row buffer
   const bool masked = a.allow_lo > 0 || a.allow_hi < a.V;
   const int nside = nc > 0 ? 2 : 1;
   int n_list[2] = {0, 0};
+  float theta[2] = {INFINITY, INFINITY}, mxs[2] = {0.f, 0.f};
   bool ok = true;
   for (int side = 0; side < nside && ok; ++side) {
     const T* cond = static_cast<const T*>(side ? a.dc : a.tc) + row_off;
@@ -370,7 +384,8 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     mx[1] = -INFINITY;
     block_reduce2<true>(c, mx);
     if (mx[0] == -INFINITY) { ok = false; break; }           // no finite logit: the dense kernel reports it
-    ok = compact_topk<E>(s, side, mx[0], side ? a.topk_d : a.topk_t, n_list[side]);
+    mxs[side] = mx[0];
+    ok = compact_topk<E>(s, side, mx[0], side ? a.topk_d : a.topk_t, n_list[side], theta[side]);
   }
   if (!ok) {
     // finish the outstanding bulk copy before leaving (bounded), then hand the node over
@@ -379,22 +394,14 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     return;
   }
 
-  // ---- union of the two supports, ordered by token: bitmap, popcount ranks, scatter
-  uint32_t* bm = s.bins;              // [kWords]
-  uint32_t* rk = s.bins + kWords;     // [kWords] union entries before word w
+  // ---- union of the two supports, ordered by token: popcount ranks of the OR-ed bitmaps, then
+  // every list entry is scattered to its rank as 2^((z - max) log2 e), or 0 below the threshold
   int* ut = reinterpret_cast<int*>(s.Z);
   float* uq = s.Z + kUCap;
   float* up = uq + kUCap;
-  for (int i = tid; i < kWords; i += ST) bm[i] = 0;
-  for (int i = tid; i < kUCap; i += ST) { uq[i] = 0.f; up[i] = 0.f; }
-  __syncthreads();
-  for (int i = tid; i < n_list[0]; i += ST) { const int t = s.ltok[0][i]; atomicOr(&bm[t >> 5], 1u << (t & 31)); }
-  for (int i = tid; i < n_list[1]; i += ST) { const int t = s.ltok[1][i]; atomicOr(&bm[t >> 5], 1u << (t & 31)); }
-  __syncthreads();
   int n_u;
   {
-    static_assert(kWords == ST, "one bitmap word per thread");
-    const int cnt = __popc(bm[tid]);
+    const int cnt = __popc(s.bm[0][tid] | s.bm[1][tid]);
     int incl = cnt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -409,29 +416,37 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
       const int t = __shfl_up_sync(0xffffffffu, wincl, o);
       if (lane >= o) wincl += t;
     }
-    rk[tid] = static_cast<uint32_t>(__shfl_sync(0xffffffffu, wincl - wt, warp) + incl - cnt);
+    s.rk[tid] = static_cast<uint32_t>(__shfl_sync(0xffffffffu, wincl - wt, warp) + incl - cnt);
     n_u = __shfl_sync(0xffffffffu, wincl, SW - 1);
   }
   __syncthreads();
   // position of token t in the union arrays, or -1
   auto uidx = [&](int t) -> int {
-    const uint32_t w = bm[t >> 5], bit = 1u << (t & 31);
-    return (w & bit) ? static_cast<int>(rk[t >> 5]) + __popc(w & (bit - 1u)) : -1;
+    const uint32_t w = s.bm[0][t >> 5] | s.bm[1][t >> 5], bit = 1u << (t & 31);
+    return (w & bit) ? static_cast<int>(s.rk[t >> 5]) + __popc(w & (bit - 1u)) : -1;
   };
-  for (int i = tid; i < n_list[0]; i += ST) {
-    const int t = s.ltok[0][i], u = uidx(t);
-    ut[u] = t;
-    uq[u] = s.lval[0][i];
-  }
-  for (int i = tid; i < n_list[1]; i += ST) {
-    const int t = s.ltok[1][i], u = uidx(t);
-    ut[u] = t;
-    up[u] = s.lval[1][i];
+#pragma unroll
+  for (int side = 0; side < 2; ++side) {
+    const float c0 = -mxs[side] * kLog2e;
+    float* mine = side ? up : uq;
+    float* other = side ? uq : up;
+    const uint32_t* obm = s.bm[side ^ 1];
+    for (int i = tid; i < n_list[side]; i += ST) {
+      const int t = s.ltok[side][i], u = uidx(t);
+      const float z = s.lval[side][i];
+      ut[u] = t;
+      mine[u] = z >= theta[side] ? ex2_approx(fmaf(z, kLog2e, c0)) : 0.f;
+      if (!((obm[t >> 5] >> (t & 31)) & 1u)) other[u] = 0.f;
+    }
   }
   __syncthreads();
-  // row totals in token order (the same from run to run)
+  // From here on thread t owns the union entries [t*per, t*per + per) in every sweep, so that a
+  // thread re-reads only what it wrote itself and the per-warp partial sums of a reduction are
+  // sums over consecutive tokens.  per is odd: consecutive threads hit different banks.
+  const int per = ((n_u + ST - 1) / ST) | 1;
+  const int i0 = min(tid * per, n_u), i1 = min(i0 + per, n_u);
   float tot[2] = {0.f, 0.f};
-  for (int i = tid; i < n_u; i += ST) { tot[0] += uq[i]; tot[1] += up[i]; }
+  for (int i = i0; i < i1; ++i) { tot[0] += uq[i]; tot[1] += up[i]; }
   block_reduce2<false>(c, tot);
   float qtot = tot[0];
   float qs = qtot > 0.f ? 1.f / qtot : 0.f;
@@ -448,24 +463,25 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
           for (int r = tid; r < a.k; r += ST)
             nbr_s[ci * a.kpad + r] = a.nbr[static_cast<long long>(code) * a.k_table + r];
       }
+      __syncthreads();
     }
   }
-  __syncthreads();
 
   if (n == 0 && tid == 0) {
     if (a.node_mass) a.node_mass[out_b] = -1.f;
     if (a.node_thresh) a.node_thresh[out_b] = -1.f;
   }
 
-  // ---- sibling loop (Sec. 4; Eq. 1-2) on the union arrays
+  // ---- sibling loop (Sec. 4; Eq. 1-2) on the union arrays.  Warp 0 evaluates a child: relaxed
+  // mass, decision and, on rejection, q~ (the mass of A moved onto x); one barrier publishes all
+  // of it, the residual sweep and its reduction follow.
   int accepted = -1;
-  for (int ci = 0; ci < nc; ++ci) {
+  for (int ci = 0; ci < nc && accepted < 0; ++ci) {
     const int child = fc + ci;
     const int x = tok_b[child];
-    const bool skip = accepted >= 0 || x < 0 || x >= a.V;
-    if (skip) {
+    if (x < 0 || x >= a.V) {
       if (tid == 0) {
-        if (accepted < 0 && x >= a.V) vflag(a.status, LANTERN_DEV_BAD_INDEX);
+        if (x >= a.V) vflag(a.status, LANTERN_DEV_BAD_INDEX);
         if (a.node_mass) a.node_mass[out_b + child] = -1.f;
         if (a.node_thresh) a.node_thresh[out_b + child] = -1.f;
       }
@@ -518,11 +534,20 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
       if (__any_sync(0xffffffffu, bad) && lane == 0) vflag(a.status, LANTERN_DEV_BAD_INDEX);
       const float m = cum;
       const float thr = px > 0.f ? fminf(1.f, m / px) : (m > 0.f ? 1.f : 0.f);
-      const float u = miscf[12 + ci];
+      const bool acc = miscf[12 + ci] < thr;
+      if (!acc) {
+        // q~: the first nA neighbours give their mass to x
+        __syncwarp();
+        for (int r = lane; r < nA; r += 32) {
+          const int t = a.code_offset + nrow[r];
+          const int it = (t >= 0 && t < a.V) ? uidx(t) : -1;
+          if (it >= 0) uq[it] = 0.f;
+        }
+        __syncwarp();
+        if (lane == 0 && ix >= 0) uq[ix] = qs > 0.f ? m / qs : 0.f;
+      }
       if (lane == 0) {
-        misc[0] = (u < thr) ? 1 : 0;
-        misc[1] = nA;
-        miscf[2] = m;
+        misc[0] = acc ? 1 : 0;
         miscf[3] = pxraw;
         misc[4] = ix;
         if (a.node_mass) a.node_mass[out_b + child] = m;
@@ -530,30 +555,18 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
       }
     }
     __syncthreads();
-    const int acc = misc[0];
-    const int nA = misc[1];
-    const float m = miscf[2];
+    if (misc[0]) {
+      accepted = child;       // leaves the loop: misc is not rewritten
+      break;
+    }
     const float pxraw = miscf[3];
     const int ix = misc[4];
-    if (acc) {
-      accepted = child;
-      __syncthreads();       // misc is rewritten by the next tested child
-      continue;
-    }
-    // ---- rejection: q~ (mass of A moved onto x), residual, drafter without x
-    for (int r = tid; r < nA; r += ST) {
-      const int t = a.code_offset + nrow[r];
-      const int it = (t >= 0 && t < a.V) ? uidx(t) : -1;
-      if (it >= 0) uq[it] = 0.f;
-    }
-    if (tid == 0 && ix >= 0) uq[ix] = qs > 0.f ? m / qs : 0.f;
-    __syncthreads();
     // Q <- [Q * rho - P]_+ with rho = qs * psum: the residual of Eq. 2 in the (unnormalised)
     // units of P.  The drafter mass left without x is psum - P[x] unless that cancels badly.
     const bool resum = pxraw > 0.5f * psum;
     const float rho = psum > 0.f ? qs * psum : qs;
     float zs[2] = {0.f, 0.f};
-    for (int i = tid; i < n_u; i += ST) {
+    for (int i = i0; i < i1; ++i) {
       float p = up[i];
       const float q = fmaxf(fmaf(uq[i], rho, -p), 0.f);
       uq[i] = q;
@@ -570,7 +583,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     } else {
       // q~ <= p_cur everywhere: both sum to one, so q~ equals p_cur (before x was dropped)
       float s2[2] = {0.f, 0.f};
-      for (int i = tid; i < n_u; i += ST) {
+      for (int i = i0; i < i1; ++i) {
         const float p = i == ix ? pxraw : up[i];
         uq[i] = p;
         s2[0] += p;
@@ -580,19 +593,22 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
       qs = ps_old;
     }
   }
+  // children that were not tested because an earlier sibling was accepted
+  if (accepted >= 0 && tid > accepted - fc && tid < nc) {
+    if (a.node_mass) a.node_mass[out_b + fc + tid] = -1.f;
+    if (a.node_thresh) a.node_thresh[out_b + fc + tid] = -1.f;
+  }
 
-  // ---- no child accepted (or leaf): draw node_token from q_cur by inverse CDF in token order
+  // ---- no child accepted (or leaf): draw node_token from q_cur by inverse CDF in token order.
+  // The last reduction left the sums of uq over each warp's (consecutive) entries in
+  // c.last_red[w*2]; a thread re-reads only the entries it wrote itself.
   if (accepted < 0) {
     if (tid == 0) { misc[5] = 0x7fffffff; misc[6] = -1; }
     const float target = miscf[7] * qtot;
-    const int per = (n_u + ST - 1) / ST;
-    const int i0 = min(tid * per, n_u), i1 = min(i0 + per, n_u);
     float sc = 0.f;
     for (int i = i0; i < i1; ++i) sc += uq[i];
     const float incl = warp_incl_scan(sc, lane);
-    if (lane == 31) reinterpret_cast<float*>(s.wtot)[warp] = incl;
-    __syncthreads();               // also orders the last sweep's writes of uq before the reads below
-    const float wt = lane < SW ? reinterpret_cast<const float*>(s.wtot)[lane] : 0.f;
+    const float wt = lane < SW ? c.last_red[lane * 2] : 0.f;
     const float wincl = warp_incl_scan(wt, lane);
     float run = __shfl_sync(0xffffffffu, wincl - wt, warp) + (incl - sc);
     int cand = 0x7fffffff, lastp = -1;
@@ -604,6 +620,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
         if (cand == 0x7fffffff && run > target) cand = i;
       }
     }
+    __syncthreads();               // misc[5], misc[6] are initialised
     if (cand != 0x7fffffff) atomicMin(&misc[5], cand);
     if (lastp >= 0) atomicMax(&misc[6], lastp);
     __syncthreads();
