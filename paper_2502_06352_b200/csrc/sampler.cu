@@ -28,7 +28,13 @@ struct SampleArgs {
   int32_t* tokens;
   float* draft_prob;
   int32_t* status;
+  int n_parents;       // parents per sequence in this launch
+  int repair;          // non-zero: draw only the parents whose first child's token is the redo marker
 };
+
+}  // namespace lantern
+#include "sampler_sparse.cuh"
+namespace lantern {
 
 __device__ __forceinline__ bool better(float ka, int ia, float kb, int ib) {   // a beats b
   return ka > kb || (ka == kb && ia < ib);
@@ -60,36 +66,13 @@ __device__ __forceinline__ void thread_best(const float* __restrict__ K, int lo,
   }
 }
 
+// One parent: drafter row into shared memory, keys, s selection rounds.
 template <typename T, bool CFG, int E>
-__global__ void __launch_bounds__(VT, 1) sample_children_kernel(const SampleArgs a) {
+__device__ __forceinline__ void sample_node(const SampleArgs& a, const int idx, VCtx& c, const TopkSmem& tk,
+                                            float* __restrict__ Z, float* __restrict__ K) {
   constexpr int SL = VT * E;
   constexpr int NV4 = E / 4;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* Z = reinterpret_cast<float*>(smem_raw);
-  float* K = Z + SL;                                    // keys; first the uncond staging buffer
-  unsigned char* nxt = reinterpret_cast<unsigned char*>(K + SL);
-  TopkSmem tk;
-  tk.gbins = reinterpret_cast<uint32_t*>(nxt);
-  tk.comp = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
-  tk.all = tk.comp + 2 * kCandLocal;
-  nxt += kScratchBytes;
-  tk.bins = reinterpret_cast<uint32_t*>(nxt);
-  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
-  tk.wcnt = reinterpret_cast<int*>(tk.wl + 2 * kCandLocal);
-  tk.wtot = reinterpret_cast<uint32_t*>(tk.wcnt + 2 * VW);
-  VCtx c;
-  c.red = reinterpret_cast<float*>(tk.wtot + 2 * (kBins / 32));
-  c.xch = c.red + 2 * VW * 4;
-  c.gath = c.xch + 8;
-  tk.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
-  tk.cnts = tk.sel + 8;
-  c.rank = cluster_ctarank();
-  c.nrank = cluster_nctarank();
-  c.parity = 0;
-  c.last_red = c.red;
-
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int idx = blockIdx.x / c.nrank;
   const int b = idx % a.B;
   const int n = a.order[a.order_begin + idx / a.B];
   const int fc = a.first_child[n], nc = a.n_child[n];
@@ -192,7 +175,57 @@ __global__ void __launch_bounds__(VT, 1) sample_children_kernel(const SampleArgs
       if (a.draft_prob) a.draft_prob[out_b + fc + round] = 0.f;
     }
   }
-  if (!single) cluster_sync();
+}
+
+template <typename T, bool CFG, int E>
+__global__ void __launch_bounds__(VT, 1) sample_children_kernel(const SampleArgs a) {
+  constexpr int SL = VT * E;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* Z = reinterpret_cast<float*>(smem_raw);
+  float* K = Z + SL;                                    // keys; first the uncond staging buffer
+  unsigned char* nxt = reinterpret_cast<unsigned char*>(K + SL);
+  TopkSmem tk;
+  tk.gbins = reinterpret_cast<uint32_t*>(nxt);
+  tk.comp = reinterpret_cast<float*>(tk.gbins + 2 * kBins);
+  tk.all = tk.comp + 2 * kCandLocal;
+  nxt += kScratchBytes;
+  tk.bins = reinterpret_cast<uint32_t*>(nxt);
+  tk.wl = reinterpret_cast<float*>(tk.bins + 2 * kBins);
+  tk.wcnt = reinterpret_cast<int*>(tk.wl + 2 * kCandLocal);
+  tk.wtot = reinterpret_cast<uint32_t*>(tk.wcnt + 2 * VW);
+  VCtx c;
+  c.red = reinterpret_cast<float*>(tk.wtot + 2 * (kBins / 32));
+  c.xch = c.red + 2 * VW * 4;
+  c.gath = c.xch + 8;
+  tk.sel = reinterpret_cast<int*>(c.gath + kMaxCluster * 4);
+  tk.cnts = tk.sel + 8;
+  c.rank = cluster_ctarank();
+  c.nrank = cluster_nctarank();
+  c.parity = 0;
+  c.last_red = c.red;
+
+  // A regular launch has one CTA (cluster) per parent.  A repair launch has fewer: cluster g of
+  // G takes the marked parents idx = g (mod G) one after another, and leaves at once when none of
+  // them is marked.
+  const int tid = threadIdx.x;
+  const int np = static_cast<int>(a.n_parents), rows = a.B * np;
+  const int G = gridDim.x / c.nrank, g0 = blockIdx.x / c.nrank;
+  auto marked = [&](int idx) {
+    const int n = a.order[a.order_begin + idx / a.B];
+    return a.tokens[static_cast<long long>(idx % a.B) * a.N + a.first_child[n]] == sparse::kRedoToken;
+  };
+  if (a.repair) {
+    bool any = false;
+    for (long long i = g0 + static_cast<long long>(tid) * G; i < rows; i += static_cast<long long>(VT) * G)
+      any |= marked(static_cast<int>(i));
+    if (!__syncthreads_or(any)) return;      // the same marks, hence the same decision, in every CTA of a cluster
+  }
+  for (int idx = g0; idx < rows; idx += G) {
+    if (a.repair && !marked(idx)) continue;
+    csync(c);     // every CTA of the row has read the mark before the row's first token is rewritten
+    sample_node<T, CFG, E>(a, idx, c, tk, Z, K);
+    csync(c);     // peers may still be reading this CTA's shared memory; the next parent overwrites it
+  }
 }
 
 }  // namespace lantern
@@ -232,7 +265,16 @@ static cudaError_t launch_sampler_e(const SampleArgs& a, int n_parents, int cs, 
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(a.B) * n_parents * cs, 1, 1);
+  unsigned clusters = static_cast<unsigned>(a.B) * n_parents;
+  if (a.repair) {        // about one cluster per SM; each walks its share of the marked parents
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      sms = 148;
+    const unsigned per_wave = static_cast<unsigned>(sms / cs > 0 ? sms / cs : 1);
+    if (clusters > per_wave) clusters = per_wave;
+  }
+  cfg.gridDim = dim3(clusters * cs, 1, 1);
   cfg.blockDim = dim3(VT, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
@@ -257,6 +299,23 @@ static cudaError_t launch_sampler(const SampleArgs& a, int n_parents, int cs, in
     if (e == 4) return launch_sampler_e<T, CFG, 4>(a, n_parents, cs, smem, st);
   }
   return cudaErrorInvalidValue;
+}
+
+// ---- launch of the list-based kernel: one CTA per parent
+template <typename T, bool CFG, int E>
+static cudaError_t launch_sample_sparse_e(const SampleArgs& a, cudaStream_t st) {
+  auto kern = sparse::sample_sparse_kernel<T, CFG, E>;
+  const size_t smem = sparse::sampler_smem_bytes(E);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  kern<<<static_cast<unsigned>(a.B) * a.n_parents, sparse::ST, smem, st>>>(a);
+  return cudaGetLastError();
+}
+template <typename T, bool CFG>
+static cudaError_t launch_sample_sparse(const SampleArgs& a, int V, cudaStream_t st) {
+  if (V <= sparse::ST * 8) return launch_sample_sparse_e<T, CFG, 8>(a, st);
+  if (V <= sparse::ST * 16) return launch_sample_sparse_e<T, CFG, 16>(a, st);
+  return launch_sample_sparse_e<T, CFG, 32>(a, st);
 }
 
 }  // namespace lantern
@@ -303,6 +362,8 @@ extern "C" lantern_status lantern_sample_draft_tree(
   a.topk_d = p->top_k_draft; a.allow_lo = allow_lo; a.allow_hi = allow_hi;
   a.seed = p->seed; a.step = p->step;
   a.tokens = tokens; a.draft_prob = draft_prob; a.status = device_status;
+  a.n_parents = i1 - i0;
+  a.repair = 0;
   int cs, e;
   size_t smem;
   const int ov = lantern_set_cluster_size(-1);     // -1 is not a valid size: reads the current value
@@ -310,6 +371,16 @@ extern "C" lantern_status lantern_sample_draft_tree(
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = draft_uncond != nullptr;
   cudaError_t err;
+  // Rows truncated to a moderate top-k take the list-based kernel; the dense kernel then draws
+  // the parents it marked as not fitting (usually none).
+  if (ov == 0 && V <= sparse::kMaxV && p->top_k_draft > 0 && p->top_k_draft < V && p->top_k_draft <= sparse::kMaxTopK) {
+    if (dt == LANTERN_F32)
+      err = cfg ? launch_sample_sparse<float, true>(a, V, st) : launch_sample_sparse<float, false>(a, V, st);
+    else
+      err = cfg ? launch_sample_sparse<__nv_bfloat16, true>(a, V, st) : launch_sample_sparse<__nv_bfloat16, false>(a, V, st);
+    if (err != cudaSuccess) return LANTERN_ERR_CUDA;
+    a.repair = 1;
+  }
   if (dt == LANTERN_F32)
     err = cfg ? launch_sampler<float, true>(a, i1 - i0, cs, e, smem, st) : launch_sampler<float, false>(a, i1 - i0, cs, e, smem, st);
   else

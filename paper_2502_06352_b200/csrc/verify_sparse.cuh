@@ -147,7 +147,9 @@ struct Smem {
 // (value 0).  Returns false when the fixed buffers cannot hold the row.  The order of the list
 // depends on the order in which the warps reserve their ranges; nothing that is summed may
 // depend on it.
-template <int E>
+// With DET the warps' ranges follow warp order (one more barrier instead of the atomic), so the
+// list order is the same from run to run.
+template <int E, bool DET = false>
 __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, int kth, int& n_list,
                                              float& theta) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -227,8 +229,22 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
       if (lane >= o) incl += t;
     }
     uint32_t base = 0;
-    if (lane == 31) base = atomicAdd(reinterpret_cast<uint32_t*>(&s.misc[8]), incl);
-    base = __shfl_sync(0xffffffffu, base, 31) + incl - cnt;
+    if (DET) {
+      if (lane == 31) s.wtot[warp] = incl;
+      __syncthreads();
+      uint32_t wt = lane < SW ? s.wtot[lane] : 0u, wincl = wt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, wincl, o);
+        if (lane >= o) wincl += t;
+      }
+      base = __shfl_sync(0xffffffffu, wincl - wt, warp) + incl - cnt;
+      const uint32_t total = __shfl_sync(0xffffffffu, wincl, SW - 1);
+      if (tid == 0) s.misc[8] = static_cast<int>(total);
+    } else {
+      if (lane == 31) base = atomicAdd(reinterpret_cast<uint32_t*>(&s.misc[8]), incl);
+      base = __shfl_sync(0xffffffffu, base, 31) + incl - cnt;
+    }
     int pos = static_cast<int>(base & 0xffffu), cpos = static_cast<int>(base >> 16);
     while (mask) {
       const int i = __ffs(mask) - 1;

@@ -84,6 +84,40 @@ def test_cluster_sizes_and_allowed_range(L, cs):
     assert np.all((gtok[:, 1:] >= 256) & (gtok[:, 1:] < 768))
 
 
+@pytest.mark.parametrize("cs", [0, 1])
+@pytest.mark.parametrize("kw", [dict(vocab=3001, codebook_size=3001, top_k=200),
+                                dict(vocab=9000, codebook_size=2000, top_k=1000, dtype="bf16", cfg_scale=None)])
+def test_topk_rows_list_and_dense_kernels(L, cs, kw):
+    # cs = 0: the list-based kernel; cs = 1: the dense kernel.  Philox uniforms, so the list kernel
+    # has to pick the right word of each token's counter block.
+    case = Case(small_config(**kw), seed=25, tokens="random", pad=3 if kw.get("dtype", "f32") == "f32" else 8)
+    seed, step = 0x5EED, 11
+    gum = np.empty((case.B, case.N, case.V), dtype=np.float32)
+    for b in range(case.B):
+        for n in range(case.N):
+            gum[b, n] = oracle.stream_uniforms(seed, step, b * case.N + n, 0, count=case.V)
+    old = L.set_cluster_size(cs)
+    try:
+        gtok, gprob, _ = _gpu_sample(L, case, seed_step=(seed, step))
+    finally:
+        L.set_cluster_size(old)
+    assert _compare(case, gum, gtok, gprob) <= 1
+
+
+def test_topk_with_massive_ties_is_redrawn_by_the_dense_kernel(L):
+    # logits on a grid of 2.0: the k-th largest value is shared by more entries than the list
+    # kernel holds, so it marks every parent and the dense kernel draws them
+    case = Case(small_config(vocab=8000, codebook_size=1000, top_k=300, cfg_scale=None, batch=2), seed=26,
+                tokens="random")
+    for v in case.padded.values():
+        if v is not None:
+            v.copy_(torch.round(v / 2.0) * 2.0)
+    gum = W.make_gumbel_uniforms(case.B, case.N, case.V, 77)
+    gtok, gprob, _ = _gpu_sample(L, case, gumbel=gum)
+    assert _compare(case, gum.numpy(), gtok, gprob) <= 1
+    assert np.all(gtok[:, 1:] >= 0)
+
+
 def test_philox_uniforms_and_level_by_level(L):
     case = Case(small_config(batch=2), seed=23, tokens="random")
     seed, step = 0xABCDEF12345, 7
