@@ -160,6 +160,37 @@ struct VerifyArgs {
   float *node_mass, *node_thresh;
   int32_t* status;
   const int32_t* only;     // [B*N] or NULL: process only the nodes whose entry is non-zero
+  // set together with `only`: the last CTA to finish also walks the trees (no separate launch)
+  int32_t* done;           // one counter, zero before the launch and again after it
+  int32_t *accept_len, *out_tokens, *out_nodes;
+  int D1;
 };
+
+// ---- walk (Sec. 2.1): follow accepted children from the root of sequence b.  L2 loads: the
+// per-node results may have been written by other CTAs of the same launch.
+__device__ __forceinline__ void walk_sequence(const int32_t* __restrict__ node_next,
+                                              const int32_t* __restrict__ node_token,
+                                              const int32_t* __restrict__ tokens, int b, int N, int D1,
+                                              int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
+                                              int32_t* __restrict__ out_nodes) {
+  const int32_t* nx = node_next + static_cast<long long>(b) * N;
+  const int32_t* nt = node_token + static_cast<long long>(b) * N;
+  const int32_t* tk = tokens + static_cast<long long>(b) * N;
+  int32_t* ot = out_tokens + static_cast<long long>(b) * D1;
+  int32_t* on = out_nodes + static_cast<long long>(b) * D1;
+  int cur = 0, len = 0;
+  while (len < D1 - 1) {
+    const int nxt = __ldcg(nx + cur);
+    if (nxt <= cur || nxt >= N) break;      // -1, or anything that is not a forward edge
+    cur = nxt;
+    ot[len] = tk[cur];
+    on[len] = cur;
+    ++len;
+  }
+  ot[len] = __ldcg(nt + cur);
+  on[len] = cur;
+  accept_len[b] = len;
+  for (int i = len + 1; i < D1; ++i) { ot[i] = -1; on[i] = -1; }
+}
 
 }  // namespace lantern

@@ -57,31 +57,14 @@ static cudaError_t launch_sparse_any(const VerifyArgs& a, int32_t* redo, int e, 
              : launch_sparse<__nv_bfloat16, false>(a, redo, e, smem, st);
 }
 
-// ---- walk (Sec. 2.1): follow accepted children from the root
+// ---- walk (Sec. 2.1) as a launch of its own: one thread per sequence
 __global__ void walk_kernel(const int32_t* __restrict__ node_next, const int32_t* __restrict__ node_token,
                             const int32_t* __restrict__ tokens, int B, int N, int D1,
                             int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
                             int32_t* __restrict__ out_nodes) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
-  const int32_t* nx = node_next + static_cast<long long>(b) * N;
-  const int32_t* nt = node_token + static_cast<long long>(b) * N;
-  const int32_t* tk = tokens + static_cast<long long>(b) * N;
-  int32_t* ot = out_tokens + static_cast<long long>(b) * D1;
-  int32_t* on = out_nodes + static_cast<long long>(b) * D1;
-  int cur = 0, len = 0;
-  while (len < D1 - 1) {
-    int nxt = nx[cur];
-    if (nxt <= cur || nxt >= N) break;      // -1, or anything that is not a forward edge
-    cur = nxt;
-    ot[len] = tk[cur];
-    on[len] = cur;
-    ++len;
-  }
-  ot[len] = nt[cur];
-  on[len] = cur;
-  accept_len[b] = len;
-  for (int i = len + 1; i < D1; ++i) { ot[i] = -1; on[i] = -1; }
+  walk_sequence(node_next, node_token, tokens, b, N, D1, accept_len, out_tokens, out_nodes);
 }
 
 }  // namespace lantern
@@ -96,10 +79,13 @@ extern "C" int32_t lantern_set_cluster_size(int32_t ctas_per_row) {
   return old;
 }
 
+namespace { constexpr int kWsTailInts = 64; }
+
 extern "C" size_t lantern_verify_tree_workspace(const lantern_tree* tree, int32_t batch) {
   if (!tree || batch <= 0) return 0;
   const TreeDev* t = reinterpret_cast<const TreeDev*>(tree);
-  return static_cast<size_t>(3) * batch * t->n_nodes * sizeof(int32_t);     // node_next, node_token, repair flags
+  // node_next, node_token, repair flags, and the completion counter of the repair launch
+  return (static_cast<size_t>(3) * batch * t->n_nodes + kWsTailInts) * sizeof(int32_t);
 }
 
 extern "C" lantern_status lantern_verify_tree(
@@ -159,6 +145,9 @@ extern "C" lantern_status lantern_verify_tree(
   a.node_next = node_next; a.node_token = node_token; a.node_mass = node_mass; a.node_thresh = node_thresh;
   a.status = device_status;
   a.only = nullptr;
+  a.done = nullptr;
+  const int D1 = t->max_depth + 1;
+  a.accept_len = accept_len; a.out_tokens = out_tokens; a.out_nodes = out_nodes; a.D1 = D1;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = target_uncond != nullptr;
   const bool f32 = dt == LANTERN_F32;
@@ -171,6 +160,7 @@ extern "C" lantern_status lantern_verify_tree(
                           (t->n_internal == 0 || topk_fits(p->top_k_draft)) && t->max_children <= 20;
   if (use_sparse) {
     const int se = V <= sparse::ST * 8 ? 8 : (V <= sparse::ST * 16 ? 16 : 32);
+    a.done = redo + static_cast<size_t>(batch) * t->n_nodes;       // the sparse kernel clears it
     e = launch_sparse_any(a, redo, se, sparse::smem_bytes(se, t->max_children, a.kpad), f32, cfg, st);
     if (e != cudaSuccess) return LANTERN_ERR_CUDA;
     a.only = redo;
@@ -192,10 +182,11 @@ extern "C" lantern_status lantern_verify_tree(
     }
   }
   if (e != cudaSuccess) return LANTERN_ERR_CUDA;
-  const int D1 = t->max_depth + 1;
-  walk_kernel<<<(batch + 127) / 128, 128, 0, st>>>(node_next, node_token, tokens, batch, t->n_nodes, D1,
-                                                    accept_len, out_tokens, out_nodes);
-  if (cudaGetLastError() != cudaSuccess) return LANTERN_ERR_CUDA;
+  if (!a.done) {      // otherwise the repair launch has walked the trees
+    walk_kernel<<<(batch + 127) / 128, 128, 0, st>>>(node_next, node_token, tokens, batch, t->n_nodes, D1,
+                                                      accept_len, out_tokens, out_nodes);
+    if (cudaGetLastError() != cudaSuccess) return LANTERN_ERR_CUDA;
+  }
   return LANTERN_OK;
 }
 
@@ -205,7 +196,7 @@ extern "C" lantern_status lantern_verify_tree(
 // that is part of the library image; every GPU that loads the library holds it until exit.
 namespace {
 constexpr int kStaticMaxNodes = 1 << 16;       // batch * tree nodes the built-in scratch can hold
-static __device__ __align__(256) int32_t g_static_scratch[3 * kStaticMaxNodes];
+static __device__ __align__(256) int32_t g_static_scratch[3 * kStaticMaxNodes + 64];
 constexpr int kMaxDevices = 64;
 void* g_static_scratch_ptr[kMaxDevices] = {};  // device address of the array, per device
 
@@ -243,5 +234,5 @@ extern "C" lantern_status lantern_verify_tree_static(
   return lantern_verify_tree(p, tree, nbr_idx, k_table, target_cond, target_uncond, draft_cond, draft_uncond, dt,
                              row_stride, seq_stride, batch, tokens, u_accept, u_resample, accept_len, out_tokens,
                              out_nodes, nullptr, nullptr, node_mass, node_thresh, device_status, scratch,
-                             sizeof(int32_t) * 3 * kStaticMaxNodes, stream);
+                             sizeof(int32_t) * (3 * kStaticMaxNodes + 64), stream);
 }

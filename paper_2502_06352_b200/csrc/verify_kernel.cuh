@@ -896,16 +896,34 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
   // cluster g of G takes the flagged nodes idx = g (mod G) one after another, and leaves at once
   // when none of them is flagged.
   const int rows = a.B * a.N, G = gridDim.x / c.nrank, g0 = blockIdx.x / c.nrank;
+  bool work = true;
   if (a.only) {
     bool any = false;
     for (long long i = g0 + static_cast<long long>(tid) * G; i < rows; i += static_cast<long long>(VT) * G)
       any |= a.only[i] != 0;
-    if (!__syncthreads_or(any)) return;      // the same flags, hence the same decision, in every CTA of a cluster
+    work = __syncthreads_or(any) != 0;       // the same flags, hence the same decision, in every CTA of a cluster
   }
-  for (int idx = g0; idx < rows; idx += G) {
-    if (a.only && a.only[idx] == 0) continue;
-    verify_node<T, CFG, E>(a, idx, c, tk, Q, P, U, misc, mbar_a, mphase, nbr_s);
-    csync(c);     // peers may still be reading this CTA's shared memory; the next node overwrites it
+  if (work) {
+    for (int idx = g0; idx < rows; idx += G) {
+      if (a.only && a.only[idx] == 0) continue;
+      verify_node<T, CFG, E>(a, idx, c, tk, Q, P, U, misc, mbar_a, mphase, nbr_s);
+      csync(c);     // peers may still be reading this CTA's shared memory; the next node overwrites it
+    }
+  }
+  if (a.done) {
+    // The CTA that finishes last (the counter wraps back to zero with it) walks every tree.
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      const unsigned old = atomicInc(reinterpret_cast<unsigned*>(a.done), gridDim.x - 1);
+      misc[0] = old == gridDim.x - 1 ? 1 : 0;
+    }
+    __syncthreads();
+    if (misc[0]) {
+      __threadfence();
+      for (int b = tid; b < a.B; b += VT)
+        walk_sequence(a.node_next, a.node_token, a.tokens, b, a.N, a.D1, a.accept_len, a.out_tokens, a.out_nodes);
+    }
   }
 }
 

@@ -28,7 +28,7 @@ constexpr int kMaxTopK = 1280;     // largest top-k routed here (slack for the l
 constexpr int kCand = 512;         // entries of the located bin that are ranked exactly
 constexpr int kUCap = 2 * kCap;    // union of both supports
 constexpr int kWords = kMaxV / 32; // bitmap words
-constexpr int kMisc = 32;
+constexpr int kMisc = 64;
 
 __host__ __device__ constexpr int z_floats(int e) { return ST * e > 3 * kUCap ? ST * e : 3 * kUCap; }
 __host__ __device__ constexpr size_t smem_bytes(int e, int max_children, int kpad) {
@@ -167,7 +167,7 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
     atomicAdd(&s.bins[dist_bin(mx, q.z)], 1u);
     atomicAdd(&s.bins[dist_bin(mx, q.w)], 1u);
   }
-  if (tid == 0) s.misc[8] = 0;                            // packed list / candidate counter
+  if (tid == 0) { s.misc[8] = 0; s.misc[9] = 0; }        // list and candidate counters
   __syncthreads();
   {
     // smallest bin whose cumulative count reaches k: thread t scans bins 4t .. 4t+3
@@ -204,66 +204,61 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
   const int bstar = s.misc[0], krem = s.misc[1], nb = s.misc[2];
   if (nb > kCand || kth - krem + nb > kCap) return false;          // same decision in every thread
   // Entries of the bins up to the located one -> list; those of the located bin also -> the
-  // candidate array.  Each thread marks its entries in two bit masks; a warp reserves its ranges
-  // of both arrays with one atomic on a packed counter (list count | candidate count << 16).
+  // candidate array.  Each thread marks its entries in a bit mask, a warp reserves its range of the
+  // list with one atomic (or, with DET, by a scan over the warps' counts).
   const uint32_t hi_bits = bin_hi_bits(bstar), lo_bits = bin_lo_bits(bstar);
-  uint32_t mask = 0, cmask = 0;
+  uint32_t mask = 0;
 #pragma unroll
   for (int v = 0; v < NV4; ++v) {
     const float4 q = *reinterpret_cast<const float4*>(Z + warp * 32 * E + v * 128 + lane * 4);
-    const float ev[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const uint32_t d = __float_as_uint(mx - ev[e]);
-      mask |= (d <= hi_bits ? 1u : 0u) << (4 * v + e);
-      cmask |= (d >= lo_bits ? 1u : 0u) << (4 * v + e);
-    }
+    if (__float_as_uint(mx - q.x) <= hi_bits) mask |= 1u << (4 * v);
+    if (__float_as_uint(mx - q.y) <= hi_bits) mask |= 1u << (4 * v + 1);
+    if (__float_as_uint(mx - q.z) <= hi_bits) mask |= 1u << (4 * v + 2);
+    if (__float_as_uint(mx - q.w) <= hi_bits) mask |= 1u << (4 * v + 3);
   }
-  cmask &= mask;
   {
-    const uint32_t cnt = static_cast<uint32_t>(__popc(mask)) | (static_cast<uint32_t>(__popc(cmask)) << 16);
-    uint32_t incl = cnt;
+    const int cnt = __popc(mask);
+    int incl = cnt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+      const int t = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += t;
     }
-    uint32_t base = 0;
+    int base = 0;
     if (DET) {
-      if (lane == 31) s.wtot[warp] = incl;
+      if (lane == 31) s.wtot[warp] = static_cast<uint32_t>(incl);
       __syncthreads();
-      uint32_t wt = lane < SW ? s.wtot[lane] : 0u, wincl = wt;
+      int wt = lane < SW ? static_cast<int>(s.wtot[lane]) : 0, wincl = wt;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, wincl, o);
+        const int t = __shfl_up_sync(0xffffffffu, wincl, o);
         if (lane >= o) wincl += t;
       }
       base = __shfl_sync(0xffffffffu, wincl - wt, warp) + incl - cnt;
-      const uint32_t total = __shfl_sync(0xffffffffu, wincl, SW - 1);
-      if (tid == 0) s.misc[8] = static_cast<int>(total);
+      const int total = __shfl_sync(0xffffffffu, wincl, SW - 1);
+      if (tid == 0) s.misc[8] = total;
     } else {
-      if (lane == 31) base = atomicAdd(reinterpret_cast<uint32_t*>(&s.misc[8]), incl);
+      if (lane == 31) base = atomicAdd(&s.misc[8], incl);
       base = __shfl_sync(0xffffffffu, base, 31) + incl - cnt;
     }
-    int pos = static_cast<int>(base & 0xffffu), cpos = static_cast<int>(base >> 16);
+    int pos = base;
     while (mask) {
       const int i = __ffs(mask) - 1;
+      mask &= mask - 1;
       const int j = warp * 32 * E + (i >> 2) * 128 + lane * 4 + (i & 3);
       const float z = Z[j];
       if (pos < kCap) { ltok[pos] = j; lval[pos] = z; }
       ++pos;
       atomicOr(&bm[j >> 5], 1u << (j & 31));
-      if ((cmask >> i) & 1u) {
-        if (cpos < kCand) s.cand[cpos] = z;
-        ++cpos;
+      if (__float_as_uint(mx - z) >= lo_bits) {
+        const int cp = atomicAdd(&s.misc[9], 1);
+        if (cp < kCand) s.cand[cp] = z;
       }
-      mask &= mask - 1;
     }
   }
   __syncthreads();
-  const uint32_t packed = static_cast<uint32_t>(s.misc[8]);
-  n_list = min(static_cast<int>(packed & 0xffffu), kCap);
-  const int ncand = min(static_cast<int>(packed >> 16), kCand);
+  n_list = min(s.misc[8], kCap);
+  const int ncand = min(s.misc[9], kCand);
   // exact rank by counting inside the located bin: theta = v with #(> v) < krem <= #(>= v);
   // eight lanes share the comparisons of one candidate
   {
@@ -318,6 +313,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int idx = blockIdx.x;
+  if (idx == 0 && tid == 0 && a.done) *a.done = 0;      // counter of the repair launch that follows
   const int b = idx % a.B;
   const int n = a.order[idx / a.B];
   const int fc = a.first_child[n], nc = a.n_child[n];
@@ -435,6 +431,19 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     s.rk[tid] = static_cast<uint32_t>(__shfl_sync(0xffffffffu, wincl - wt, warp) + incl - cnt);
     n_u = __shfl_sync(0xffffffffu, wincl, SW - 1);
   }
+  // ---- neighbour rows must have landed
+  if (bulk_issued) {
+    bool landed = mbar_wait_bounded(mbar_a, 0);
+    if (!__syncthreads_and(landed)) {
+      if (tid == 0) vflag(a.status, LANTERN_DEV_TIMEOUT);
+      for (int ci = 0; ci < nc; ++ci) {
+        int code = tok_b[fc + ci] - a.code_offset;
+        if (code >= 0 && code < a.n_codes)
+          for (int r = tid; r < a.k; r += ST)
+            nbr_s[ci * a.kpad + r] = a.nbr[static_cast<long long>(code) * a.k_table + r];
+      }
+    }
+  }
   __syncthreads();
   // position of token t in the union arrays, or -1
   auto uidx = [&](int t) -> int {
@@ -455,6 +464,15 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
       if (!((obm[t >> 5] >> (t & 31)) & 1u)) other[u] = 0.f;
     }
   }
+  // the staged neighbour codes become positions in the union arrays (-1: not in either support,
+  // -2: outside the vocabulary), so that the serial sibling loop below only follows one index
+  if (want_nbr) {
+    for (int i = tid; i < nc * a.k; i += ST) {
+      const int ci = i / a.k, r = i - ci * a.k;
+      const int t = a.code_offset + nbr_s[ci * a.kpad + r];
+      nbr_s[ci * a.kpad + r] = (t >= 0 && t < a.V) ? uidx(t) : -2;
+    }
+  }
   __syncthreads();
   // From here on thread t owns the union entries [t*per, t*per + per) in every sweep, so that a
   // thread re-reads only what it wrote itself and the per-warp partial sums of a reduction are
@@ -467,21 +485,6 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
   float qtot = tot[0];
   float qs = qtot > 0.f ? 1.f / qtot : 0.f;
   float psum = tot[1];
-
-  // ---- neighbour rows must have landed
-  if (bulk_issued) {
-    bool landed = mbar_wait_bounded(mbar_a, 0);
-    if (!__syncthreads_and(landed)) {
-      if (tid == 0) vflag(a.status, LANTERN_DEV_TIMEOUT);
-      for (int ci = 0; ci < nc; ++ci) {
-        int code = tok_b[fc + ci] - a.code_offset;
-        if (code >= 0 && code < a.n_codes)
-          for (int r = tid; r < a.k; r += ST)
-            nbr_s[ci * a.kpad + r] = a.nbr[static_cast<long long>(code) * a.k_table + r];
-      }
-      __syncthreads();
-    }
-  }
 
   if (n == 0 && tid == 0) {
     if (a.node_mass) a.node_mass[out_b] = -1.f;
@@ -523,13 +526,9 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
           const int r = base8 + i * 32 + lane;
           qa[i] = 0.f;
           if (r < a.k) {
-            const int t = a.code_offset + nrow[r];
-            if (t >= 0 && t < a.V) {
-              const int it = uidx(t);
-              if (it >= 0) qa[i] = uq[it] * qs;
-            } else {
-              bad = true;
-            }
+            const int it = nrow[r];
+            if (it >= 0) qa[i] = uq[it] * qs;
+            bad |= it == -2;
           }
         }
 #pragma unroll
@@ -555,8 +554,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
         // q~: the first nA neighbours give their mass to x
         __syncwarp();
         for (int r = lane; r < nA; r += 32) {
-          const int t = a.code_offset + nrow[r];
-          const int it = (t >= 0 && t < a.V) ? uidx(t) : -1;
+          const int it = nrow[r];
           if (it >= 0) uq[it] = 0.f;
         }
         __syncwarp();
@@ -619,7 +617,6 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
   // The last reduction left the sums of uq over each warp's (consecutive) entries in
   // c.last_red[w*2]; a thread re-reads only the entries it wrote itself.
   if (accepted < 0) {
-    if (tid == 0) { misc[5] = 0x7fffffff; misc[6] = -1; }
     const float target = miscf[7] * qtot;
     float sc = 0.f;
     for (int i = i0; i < i1; ++i) sc += uq[i];
@@ -636,14 +633,18 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
         if (cand == 0x7fffffff && run > target) cand = i;
       }
     }
-    __syncthreads();               // misc[5], misc[6] are initialised
-    if (cand != 0x7fffffff) atomicMin(&misc[5], cand);
-    if (lastp >= 0) atomicMax(&misc[6], lastp);
+    cand = __reduce_min_sync(0xffffffffu, cand);      // first crossing / last positive entry of the warp
+    lastp = __reduce_max_sync(0xffffffffu, lastp);
+    if (lane == 0) { misc[32 + warp] = cand; misc[48 + warp] = lastp; }
     __syncthreads();
-    if (tid == 0) {
-      const int found = misc[5] != 0x7fffffff ? misc[5] : misc[6];
-      a.node_token[out_b + n] = found >= 0 ? ut[found] : -1;
-      if (found < 0) vflag(a.status, LANTERN_DEV_EMPTY_ROW);
+    if (warp == 0) {
+      cand = __reduce_min_sync(0xffffffffu, lane < SW ? misc[32 + lane] : 0x7fffffff);
+      lastp = __reduce_max_sync(0xffffffffu, lane < SW ? misc[48 + lane] : -1);
+      if (lane == 0) {
+        const int found = cand != 0x7fffffff ? cand : lastp;
+        a.node_token[out_b + n] = found >= 0 ? ut[found] : -1;
+        if (found < 0) vflag(a.status, LANTERN_DEV_EMPTY_ROW);
+      }
     }
   } else if (tid == 0) {
     a.node_token[out_b + n] = -1;
