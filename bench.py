@@ -60,7 +60,7 @@ TRAFFIC = {"c2_llamagen512": {"kernel_sha256": "", "bytes": None}}
 def kernel_sha256():
     import hashlib
     h = hashlib.sha256()
-    for f in ("verify_kernel.cuh", "verify_launch.cuh", "verify.cu", "rowops.cuh", "common.cuh"):
+    for f in ("verify_sparse.cuh", "verify_kernel.cuh", "verify_launch.cuh", "verify.cu", "rowops.cuh", "common.cuh"):
         with open(os.path.join(ROOT, "paper_2502_06352_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -438,6 +438,12 @@ def main():
         e2e_ms = float(t.item())
     e2e_value = world * B * N * KE / (e2e_ms * 1e-3)
 
+    # which kernels ran (the library decides from the parameters; this only reports it)
+    lists_v = L.verify_tree_path(params, tree) == 1
+    lists_s = L.sample_draft_tree_path(params) == 1
+    verify_kernels = ("verify_sparse_kernel + verify_nodes_kernel (repair launch, walks the trees)" if lists_v
+                      else "verify_nodes_kernel + walk_kernel")
+    launches_per_step = (2 if lists_s else 1) + 2
     if rank == 0:
         peak, peak_kind = peak_hbm()
         achieved = alg_bytes / (verify_avg_ms * 1e-3) / 1e9
@@ -449,16 +455,16 @@ def main():
                        "cfg_scale": cfg.cfg_scale, "top_k": cfg.top_k, "neighbours_k": cfg.k, "lambda": cfg.lam,
                        "codebook": [cfg.codebook_size, cfg.codebook_dim], "parallelism": "dp%d" % world,
                        "l2_policy": "ring of %d input sets, %.0f MB in total (> 126 MB L2)" % (ring, ring * set_bytes / 1e6),
-                       "step": "sample_draft_tree + verify_tree (+ walk)",
+                       "step": "sample_draft_tree + verify_tree (incl. walk), %d kernel launches" % launches_per_step,
                        "launch": "cuda graph of %d steps, replayed" % per_graph if g_step is not None else "eager"},
-            "roofline": {"bound": "hbm", "kernel": "verify_nodes_kernel (+ walk_kernel)", "achieved": achieved, "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": verify_kernels, "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": measured_traffic(cfg.name),
                          "algorithmic_bytes": alg_bytes, "launch_ms_avg": verify_avg_ms,
                          "launch_ms_median": verify_ms[len(verify_ms) // 2],
                          "step_bytes_incl_sampler": alg_bytes + sampler_bytes,
                          "step_gbs": (alg_bytes + sampler_bytes) / (elapsed_ms / K * 1e-3) / 1e9},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": KE},
-            "gpu_launches": 3 * K,
+            "gpu_launches": launches_per_step * K,
             "clocks": clk,
             "table_build": {"ms": table_ms, "L": cfg.codebook_size, "d": cfg.codebook_dim, "k": cfg.k,
                             "dtype": cfg.codebook_dtype},

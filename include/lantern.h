@@ -149,7 +149,7 @@ lantern_status lantern_sample_draft_tree(const lantern_params* params, const lan
  *                  a node was not tested; or NULL
  *   device_status  one int32, OR-ed with LANTERN_DEV_* bits; or NULL
  *   workspace      device scratch >= lantern_verify_tree_workspace() bytes (12 bytes per node:
- *                  node_next, node_token and one repair flag), 256-byte aligned.  It may be
+ *                  node_next, node_token and one repair flag; plus 256 bytes), 256-byte aligned.  It may be
  *                  NULL when node_next and node_token are both given; rows truncated by top-k
  *                  then take the dense kernel instead of the faster list-based one, which needs
  *                  the flags.                                                                    */
@@ -166,6 +166,20 @@ lantern_status lantern_verify_tree(const lantern_params* params, const lantern_t
                                    float* node_mass, float* node_thresh,
                                    int32_t* device_status, void* workspace, size_t workspace_bytes,
                                    void* stream);
+
+/* ---- which kernels a call launches ---------------------------------------------------------------
+ * Rows that App. B's top-k truncation cuts to at most 1280 entries, in vocabularies of at most
+ * 16384 tokens, are handled by list-based kernels (the row is compacted to its survivors; everything
+ * after works on those), followed by a launch of the dense kernels that redoes the nodes whose
+ * rows did not fit the lists' fixed buffers (massive ties; usually none).  All other calls run the
+ * dense kernels alone.  Results are the same either way; these queries only tell which it will be
+ * (lantern_verify_tree additionally needs its full workspace for the list path).
+ * lantern_sample_draft_tree launches 1 (dense) or 2 (lists) kernels, lantern_verify_tree always 2
+ * (dense + walk, or lists + repair launch that also walks).  Returns -1 on NULL arguments.       */
+#define LANTERN_PATH_DENSE 0
+#define LANTERN_PATH_LISTS 1
+int32_t lantern_verify_tree_path(const lantern_params* params, const lantern_tree* tree);
+int32_t lantern_sample_draft_tree_path(const lantern_params* params);
 
 /* ---- relaxed verification without any allocation ---------------------------------------------
  * The paper has no counterpart to this entry point; it exists for callers that must not, or

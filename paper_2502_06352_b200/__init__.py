@@ -15,5 +15,7 @@ from .binding import (  # noqa: F401
     verify_tree_static,
     philox_raw,
     set_cluster_size,
+    verify_tree_path,
+    sample_draft_tree_path,
     lib,
 )

@@ -93,6 +93,10 @@ def _load():
                                      ctypes.c_uint32, i32, vp, vp]
     L.lantern_set_cluster_size.restype = i32
     L.lantern_set_cluster_size.argtypes = [i32]
+    L.lantern_verify_tree_path.restype = i32
+    L.lantern_verify_tree_path.argtypes = [ctypes.POINTER(_CParams), vp]
+    L.lantern_sample_draft_tree_path.restype = i32
+    L.lantern_sample_draft_tree_path.argtypes = [ctypes.POINTER(_CParams)]
     return L
 
 
@@ -259,6 +263,18 @@ def philox_raw(seed, first, c1, c2, c3, n, device="cuda"):
     with torch.cuda.device(out.device):
         _check(lib.lantern_philox_raw(seed, first, c1, c2, c3, n, _ptr(out), _stream()), "lantern_philox_raw")
     return out.to(torch.int64) & 0xFFFFFFFF
+
+
+def verify_tree_path(params: "Params", tree: "Tree") -> int:
+    """lantern_verify_tree_path: 0 = dense kernels, 1 = list-based kernels + repair launch."""
+    cp = params.c()
+    return lib.lantern_verify_tree_path(ctypes.byref(cp), tree.handle)
+
+
+def sample_draft_tree_path(params: "Params") -> int:
+    """lantern_sample_draft_tree_path: 0 = dense kernel, 1 = list-based kernel + repair launch."""
+    cp = params.c()
+    return lib.lantern_sample_draft_tree_path(ctypes.byref(cp))
 
 
 def set_cluster_size(ctas_per_row: int) -> int:

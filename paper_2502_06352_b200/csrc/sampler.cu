@@ -324,6 +324,20 @@ using namespace lantern;
 
 extern "C" int32_t lantern_set_cluster_size(int32_t);
 
+namespace {
+// Rows truncated to a moderate top-k can take the list-based kernel.
+bool sampler_uses_lists(const lantern_params* p) {
+  const int V = p->vocab;
+  const int ov = lantern_set_cluster_size(-1);     // -1 is not a valid size: reads the current value
+  return ov == 0 && V <= sparse::kMaxV && p->top_k_draft > 0 && p->top_k_draft < V && p->top_k_draft <= sparse::kMaxTopK;
+}
+}  // namespace
+
+extern "C" int32_t lantern_sample_draft_tree_path(const lantern_params* p) {
+  if (!p) return -1;
+  return sampler_uses_lists(p) ? LANTERN_PATH_LISTS : LANTERN_PATH_DENSE;
+}
+
 extern "C" lantern_status lantern_sample_draft_tree(
     const lantern_params* p, const lantern_tree* tree, const void* draft_cond, const void* draft_uncond,
     lantern_dtype dt, int64_t row_stride, int64_t seq_stride, int32_t batch, int32_t parent_begin,
@@ -373,7 +387,7 @@ extern "C" lantern_status lantern_sample_draft_tree(
   cudaError_t err;
   // Rows truncated to a moderate top-k take the list-based kernel; the dense kernel then draws
   // the parents it marked as not fitting (usually none).
-  if (ov == 0 && V <= sparse::kMaxV && p->top_k_draft > 0 && p->top_k_draft < V && p->top_k_draft <= sparse::kMaxTopK) {
+  if (sampler_uses_lists(p)) {
     if (dt == LANTERN_F32)
       err = cfg ? launch_sample_sparse<float, true>(a, V, st) : launch_sample_sparse<float, false>(a, V, st);
     else

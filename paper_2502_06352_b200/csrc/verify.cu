@@ -41,7 +41,10 @@ static cudaError_t launch_sparse_e(const VerifyArgs& a, int32_t* redo, size_t sm
   auto kern = sparse::verify_sparse_kernel<T, CFG, E>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  kern<<<static_cast<unsigned>(a.B) * a.N, sparse::ST, smem, st>>>(a, redo);
+  const int chunk = sm_count();
+  const int nI = a.B * a.n_internal, nL = a.B * (a.N - a.n_internal);
+  const int blocks = (nI + chunk - 1) / chunk + (nL + chunk - 1) / chunk;
+  kern<<<static_cast<unsigned>(blocks) * chunk, sparse::ST, smem, st>>>(a, redo, chunk);
   return cudaGetLastError();
 }
 template <typename T, bool CFG>
@@ -79,7 +82,21 @@ extern "C" int32_t lantern_set_cluster_size(int32_t ctas_per_row) {
   return old;
 }
 
-namespace { constexpr int kWsTailInts = 64; }
+namespace {
+constexpr int kWsTailInts = 64;
+// Rows truncated to a moderate top-k on every side that is read can take the list-based kernel.
+bool verify_uses_lists(const lantern_params* p, const TreeDev* t) {
+  const int V = p->vocab;
+  auto topk_fits = [&](int k) { return k > 0 && k < V && k <= sparse::kMaxTopK; };
+  return g_cluster_override == 0 && V <= sparse::kMaxV && topk_fits(p->top_k_target) &&
+         (t->n_internal == 0 || topk_fits(p->top_k_draft)) && t->max_children <= 8;
+}
+}  // namespace
+
+extern "C" int32_t lantern_verify_tree_path(const lantern_params* p, const lantern_tree* tree) {
+  if (!p || !tree) return -1;
+  return verify_uses_lists(p, reinterpret_cast<const TreeDev*>(tree)) ? LANTERN_PATH_LISTS : LANTERN_PATH_DENSE;
+}
 
 extern "C" size_t lantern_verify_tree_workspace(const lantern_tree* tree, int32_t batch) {
   if (!tree || batch <= 0) return 0;
@@ -136,7 +153,7 @@ extern "C" lantern_status lantern_verify_tree(
   a.nbr = nbr_idx; a.k_table = k_table;
   a.use_bulk = (p->k > 0 && k_table % 4 == 0 && reinterpret_cast<uintptr_t>(nbr_idx) % 16 == 0) ? 1 : 0;
   a.first_child = t->d_first_child; a.n_child = t->d_n_child; a.order = t->d_order;
-  a.B = batch; a.N = t->n_nodes; a.V = V;
+  a.B = batch; a.N = t->n_nodes; a.V = V; a.n_internal = t->n_internal;
   a.kpad = (p->k + 3) & ~3;
   a.g = p->cfg_scale; a.inv_tau = 1.0f / p->temperature; a.lambda = p->lambda;
   a.topk_t = p->top_k_target; a.topk_d = p->top_k_draft; a.k = p->k;
@@ -155,9 +172,7 @@ extern "C" lantern_status lantern_verify_tree(
   cudaError_t e;
   // Rows truncated to a moderate top-k on every side that is read take the sparse kernel; the
   // dense kernel then repairs the nodes it could not hold (a.only) and usually finds none.
-  auto topk_fits = [&](int k) { return k > 0 && k < V && k <= sparse::kMaxTopK; };
-  const bool use_sparse = redo && g_cluster_override == 0 && V <= sparse::kMaxV && topk_fits(p->top_k_target) &&
-                          (t->n_internal == 0 || topk_fits(p->top_k_draft)) && t->max_children <= 20;
+  const bool use_sparse = redo && verify_uses_lists(p, t);
   if (use_sparse) {
     const int se = V <= sparse::ST * 8 ? 8 : (V <= sparse::ST * 16 ? 16 : 32);
     a.done = redo + static_cast<size_t>(batch) * t->n_nodes;       // the sparse kernel clears it

@@ -28,7 +28,8 @@ constexpr int kMaxTopK = 1280;     // largest top-k routed here (slack for the l
 constexpr int kCand = 512;         // entries of the located bin that are ranked exactly
 constexpr int kUCap = 2 * kCap;    // union of both supports
 constexpr int kWords = kMaxV / 32; // bitmap words
-constexpr int kMisc = 64;
+constexpr int kMisc = 96;     // [12..19] accept uniforms, [20..27] child tokens, [28..35] their union
+                              // positions, [64..95] per-warp results of the draw
 
 __host__ __device__ constexpr int z_floats(int e) { return ST * e > 3 * kUCap ? ST * e : 3 * kUCap; }
 __host__ __device__ constexpr size_t smem_bytes(int e, int max_children, int kpad) {
@@ -287,7 +288,7 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
 // E = row entries per thread (V <= 512 * E).  `redo[b*N + n]` is set to 1 when node (b, n) has to
 // be processed by the dense kernel instead, else to 0.
 template <typename T, bool CFG, int E>
-__global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a, int32_t* __restrict__ redo) {
+__global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a, int32_t* __restrict__ redo, const int chunk) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem s;
   s.Z = reinterpret_cast<float*>(smem_raw);
@@ -312,8 +313,28 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
   float* miscf = reinterpret_cast<float*>(s.misc);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int idx = blockIdx.x;
-  if (idx == 0 && tid == 0 && a.done) *a.done = 0;      // counter of the repair launch that follows
+  if (blockIdx.x == 0 && tid == 0 && a.done) *a.done = 0;      // counter of the repair launch that follows
+  // Launch order: blocks of `chunk` CTAs (one per SM) alternate between internal nodes (two rows,
+  // sibling loop) and leaves (one row), so that the two CTAs sharing an SM start in different
+  // phases and one's streaming overlaps the other's on-chip work.  The grid is padded to whole
+  // blocks; CTAs beyond the last node of their kind leave at once.
+  int idx;
+  {
+    const int nI = a.B * a.n_internal, nL = a.B * (a.N - a.n_internal);
+    const int mI = (nI + chunk - 1) / chunk, mL = (nL + chunk - 1) / chunk;
+    const int c = blockIdx.x / chunk, off = blockIdx.x - c * chunk;
+    const int both = 2 * min(mI, mL);
+    int kind, k;
+    if (c < both) {
+      kind = c & 1;
+      k = (c >> 1) * chunk + off;
+    } else {
+      kind = mI > mL ? 0 : 1;
+      k = (min(mI, mL) + (c - both)) * chunk + off;
+    }
+    if (k >= (kind ? nL : nI)) return;
+    idx = kind ? nI + k : k;            // position in the internal-first node order
+  }
   const int b = idx % a.B;
   const int n = a.order[idx / a.B];
   const int fc = a.first_child[n], nc = a.n_child[n];
@@ -376,6 +397,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
       u = uniform_halfopen(philox_stream(a.seed, a.step, static_cast<uint32_t>(out_b + fc + tid), kStreamAccept, 0).x);
     }
     miscf[12 + tid] = u;
+    misc[20 + tid] = tok_b[fc + tid];
   }
   static_assert(kWords == ST, "one bitmap word per thread");
   s.bm[0][tid] = 0;
@@ -466,6 +488,10 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
   }
   // the staged neighbour codes become positions in the union arrays (-1: not in either support,
   // -2: outside the vocabulary), so that the serial sibling loop below only follows one index
+  if (tid < nc) {
+    const int x = misc[20 + tid];
+    misc[28 + tid] = (x >= 0 && x < a.V) ? uidx(x) : -1;
+  }
   if (want_nbr) {
     for (int i = tid; i < nc * a.k; i += ST) {
       const int ci = i / a.k, r = i - ci * a.k;
@@ -497,7 +523,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
   int accepted = -1;
   for (int ci = 0; ci < nc && accepted < 0; ++ci) {
     const int child = fc + ci;
-    const int x = tok_b[child];
+    const int x = misc[20 + ci];
     if (x < 0 || x >= a.V) {
       if (tid == 0) {
         if (x >= a.V) vflag(a.status, LANTERN_DEV_BAD_INDEX);
@@ -511,7 +537,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     const int* nrow = nbr_s + ci * a.kpad;
     const float ps = psum > 0.f ? 1.f / psum : 0.f;
     if (warp == 0) {
-      const int ix = uidx(x);
+      const int ix = misc[28 + ci];
       const float qx = ix >= 0 ? uq[ix] * qs : 0.f;
       const float pxraw = ix >= 0 ? up[ix] : 0.f;
       const float px = pxraw * ps;
@@ -635,11 +661,11 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     }
     cand = __reduce_min_sync(0xffffffffu, cand);      // first crossing / last positive entry of the warp
     lastp = __reduce_max_sync(0xffffffffu, lastp);
-    if (lane == 0) { misc[32 + warp] = cand; misc[48 + warp] = lastp; }
+    if (lane == 0) { misc[64 + warp] = cand; misc[80 + warp] = lastp; }
     __syncthreads();
     if (warp == 0) {
-      cand = __reduce_min_sync(0xffffffffu, lane < SW ? misc[32 + lane] : 0x7fffffff);
-      lastp = __reduce_max_sync(0xffffffffu, lane < SW ? misc[48 + lane] : -1);
+      cand = __reduce_min_sync(0xffffffffu, lane < SW ? misc[64 + lane] : 0x7fffffff);
+      lastp = __reduce_max_sync(0xffffffffu, lane < SW ? misc[80 + lane] : -1);
       if (lane == 0) {
         const int found = cand != 0x7fffffff ? cand : lastp;
         a.node_token[out_b + n] = found >= 0 ? ut[found] : -1;
