@@ -166,31 +166,47 @@ struct VerifyArgs {
   int D1;
 };
 
-// ---- walk (Sec. 2.1): follow accepted children from the root of sequence b.  L2 loads: the
-// per-node results may have been written by other CTAs of the same launch.
-__device__ __forceinline__ void walk_sequence(const int32_t* __restrict__ node_next,
-                                              const int32_t* __restrict__ node_token,
-                                              const int32_t* __restrict__ tokens, int b, int N, int D1,
-                                              int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
-                                              int32_t* __restrict__ out_nodes) {
-  const int32_t* nx = node_next + static_cast<long long>(b) * N;
-  const int32_t* nt = node_token + static_cast<long long>(b) * N;
-  const int32_t* tk = tokens + static_cast<long long>(b) * N;
-  int32_t* ot = out_tokens + static_cast<long long>(b) * D1;
-  int32_t* on = out_nodes + static_cast<long long>(b) * D1;
+// ---- walk (Sec. 2.1): follow accepted children from the root of one sequence.  nx / nt are the
+// sequence's node_next / node_token rows (staged in shared memory by the callers: the walk is a
+// chain of dependent reads), tk its draft tokens, ot / on its output rows.
+__device__ __forceinline__ void walk_rows(const int32_t* nx, const int32_t* nt, const int32_t* __restrict__ tk,
+                                          int N, int D1, int32_t* __restrict__ accept_len,
+                                          int32_t* __restrict__ ot, int32_t* __restrict__ on) {
   int cur = 0, len = 0;
   while (len < D1 - 1) {
-    const int nxt = __ldcg(nx + cur);
+    const int nxt = nx[cur];
     if (nxt <= cur || nxt >= N) break;      // -1, or anything that is not a forward edge
     cur = nxt;
     ot[len] = tk[cur];
     on[len] = cur;
     ++len;
   }
-  ot[len] = __ldcg(nt + cur);
+  ot[len] = nt[cur];
   on[len] = cur;
-  accept_len[b] = len;
+  *accept_len = len;
   for (int i = len + 1; i < D1; ++i) { ot[i] = -1; on[i] = -1; }
+}
+
+// Walks of sequences [b0, b0 + nb) by the calling CTA: both per-node arrays are first copied to
+// `stage` (2 * nb * N ints of shared memory) with coalesced L2 loads (other CTAs of the same launch
+// may have written them), then thread i walks sequence b0 + i.
+__device__ __forceinline__ void walk_staged(const int32_t* __restrict__ node_next, const int32_t* __restrict__ node_token,
+                                            const int32_t* __restrict__ tokens, int b0, int nb, int N, int D1,
+                                            int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
+                                            int32_t* __restrict__ out_nodes, int32_t* stage) {
+  const long long off = static_cast<long long>(b0) * N;
+  const int cnt = nb * N;
+  for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+    stage[i] = __ldcg(node_next + off + i);
+    stage[cnt + i] = __ldcg(node_token + off + i);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < nb; i += blockDim.x) {
+    const int b = b0 + i;
+    walk_rows(stage + i * N, stage + cnt + i * N, tokens + static_cast<long long>(b) * N, N, D1, accept_len + b,
+              out_tokens + static_cast<long long>(b) * D1, out_nodes + static_cast<long long>(b) * D1);
+  }
+  __syncthreads();
 }
 
 }  // namespace lantern

@@ -1,4 +1,6 @@
 // Relaxed verification of a static draft tree: host side of lantern_verify_tree and the walk.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace lantern {
@@ -60,14 +62,19 @@ static cudaError_t launch_sparse_any(const VerifyArgs& a, int32_t* redo, int e, 
              : launch_sparse<__nv_bfloat16, false>(a, redo, e, smem, st);
 }
 
-// ---- walk (Sec. 2.1) as a launch of its own: one thread per sequence
-__global__ void walk_kernel(const int32_t* __restrict__ node_next, const int32_t* __restrict__ node_token,
-                            const int32_t* __restrict__ tokens, int B, int N, int D1,
-                            int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
-                            int32_t* __restrict__ out_nodes) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= B) return;
-  walk_sequence(node_next, node_token, tokens, b, N, D1, accept_len, out_tokens, out_nodes);
+// ---- walk (Sec. 2.1) as a launch of its own: a CTA stages the per-node results of `seqs`
+// sequences in shared memory (at most 48 KB) and walks them
+constexpr int kWalkThreads = 128;
+__global__ void __launch_bounds__(kWalkThreads) walk_kernel(const int32_t* __restrict__ node_next,
+                                                            const int32_t* __restrict__ node_token,
+                                                            const int32_t* __restrict__ tokens, int B, int N, int D1,
+                                                            int seqs, int32_t* __restrict__ accept_len,
+                                                            int32_t* __restrict__ out_tokens,
+                                                            int32_t* __restrict__ out_nodes) {
+  extern __shared__ int32_t walk_stage[];
+  const int b0 = blockIdx.x * seqs;
+  walk_staged(node_next, node_token, tokens, b0, min(seqs, B - b0), N, D1, accept_len, out_tokens, out_nodes,
+              walk_stage);
 }
 
 }  // namespace lantern
@@ -198,8 +205,9 @@ extern "C" lantern_status lantern_verify_tree(
   }
   if (e != cudaSuccess) return LANTERN_ERR_CUDA;
   if (!a.done) {      // otherwise the repair launch has walked the trees
-    walk_kernel<<<(batch + 127) / 128, 128, 0, st>>>(node_next, node_token, tokens, batch, t->n_nodes, D1,
-                                                      accept_len, out_tokens, out_nodes);
+    const int seqs = std::max(1, std::min(16, 6144 / t->n_nodes));      // 2 * seqs * N ints <= 48 KB
+    walk_kernel<<<(batch + seqs - 1) / seqs, kWalkThreads, sizeof(int32_t) * 2 * seqs * t->n_nodes, st>>>(
+        node_next, node_token, tokens, batch, t->n_nodes, D1, seqs, accept_len, out_tokens, out_nodes);
     if (cudaGetLastError() != cudaSuccess) return LANTERN_ERR_CUDA;
   }
   return LANTERN_OK;

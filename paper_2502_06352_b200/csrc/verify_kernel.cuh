@@ -921,8 +921,11 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
     __syncthreads();
     if (misc[0]) {
       __threadfence();
-      for (int b = tid; b < a.B; b += VT)
-        walk_sequence(a.node_next, a.node_token, a.tokens, b, a.N, a.D1, a.accept_len, a.out_tokens, a.out_nodes);
+      int32_t* stage = reinterpret_cast<int32_t*>(Q);          // Q and P: 2 * SL ints, free by now
+      const int per_pass = max(1, SL / a.N);                    // sequences whose rows fit the stage
+      for (int b0 = 0; b0 < a.B; b0 += per_pass)
+        walk_staged(a.node_next, a.node_token, a.tokens, b0, min(per_pass, a.B - b0), a.N, a.D1, a.accept_len,
+                    a.out_tokens, a.out_nodes, stage);
     }
   }
 }
