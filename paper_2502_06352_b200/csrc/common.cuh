@@ -63,6 +63,17 @@ __device__ __forceinline__ uint32_t dsmem_ld_u32(uint32_t addr) {
   return v;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of a decode step starts with this: wait until the kernel launched before it on the
+// stream has finished and its writes are visible, then let the kernel launched after it be set up
+// early (its CTAs start as SMs drain and wait at the same place).  Launched with
+// launch_after_previous() below, consecutive kernels lose the launch gap between them; launched
+// any other way, both instructions do nothing.
+__device__ __forceinline__ void grid_dependency_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---------------------------------------------------------------- warp / block reductions
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -207,6 +218,33 @@ __device__ __forceinline__ void walk_staged(const int32_t* __restrict__ node_nex
               out_tokens + static_cast<long long>(b) * D1, out_nodes + static_cast<long long>(b) * D1);
   }
   __syncthreads();
+}
+
+// Host side: launch `kern` with programmatic stream serialisation (and, when cluster > 1, that
+// cluster size).  The kernel must call grid_dependency_sync() before it touches global memory.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_after_previous(void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                                                cudaStream_t st, int cluster, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(block, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[na].val.programmaticStreamSerializationAllowed = 1;
+  ++na;
+  if (cluster > 1) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = static_cast<unsigned>(cluster);
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
 }  // namespace lantern

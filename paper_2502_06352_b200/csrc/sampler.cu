@@ -179,6 +179,7 @@ __device__ __forceinline__ void sample_node(const SampleArgs& a, const int idx, 
 
 template <typename T, bool CFG, int E>
 __global__ void __launch_bounds__(VT, 1) sample_children_kernel(const SampleArgs a) {
+  grid_dependency_sync();
   constexpr int SL = VT * E;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* Z = reinterpret_cast<float*>(smem_raw);
@@ -264,7 +265,6 @@ static cudaError_t launch_sampler_e(const SampleArgs& a, int n_parents, int cs, 
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
   }
-  cudaLaunchConfig_t cfg = {};
   unsigned clusters = static_cast<unsigned>(a.B) * n_parents;
   if (a.repair) {        // about one cluster per SM; each walks its share of the marked parents
     int dev = 0, sms = 0;
@@ -274,18 +274,7 @@ static cudaError_t launch_sampler_e(const SampleArgs& a, int n_parents, int cs, 
     const unsigned per_wave = static_cast<unsigned>(sms / cs > 0 ? sms / cs : 1);
     if (clusters > per_wave) clusters = per_wave;
   }
-  cfg.gridDim = dim3(clusters * cs, 1, 1);
-  cfg.blockDim = dim3(VT, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = cs;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, a);
+  return launch_after_previous(kern, clusters * cs, VT, smem, st, cs, a);
 }
 
 template <typename T, bool CFG>
@@ -308,8 +297,7 @@ static cudaError_t launch_sample_sparse_e(const SampleArgs& a, cudaStream_t st) 
   const size_t smem = sparse::sampler_smem_bytes(E);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  kern<<<static_cast<unsigned>(a.B) * a.n_parents, sparse::ST, smem, st>>>(a);
-  return cudaGetLastError();
+  return launch_after_previous(kern, static_cast<unsigned>(a.B) * a.n_parents, sparse::ST, smem, st, 1, a);
 }
 template <typename T, bool CFG>
 static cudaError_t launch_sample_sparse(const SampleArgs& a, int V, cudaStream_t st) {

@@ -34,6 +34,7 @@ __device__ __forceinline__ void warp_key_best(float& k, int& i) {
 
 template <typename T, bool CFG, int E>
 __global__ void __launch_bounds__(ST, 2) sample_sparse_kernel(const SampleArgs a) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem s;
   s.Z = reinterpret_cast<float*>(smem_raw);

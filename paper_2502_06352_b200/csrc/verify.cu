@@ -46,8 +46,7 @@ static cudaError_t launch_sparse_e(const VerifyArgs& a, int32_t* redo, size_t sm
   const int chunk = sm_count();
   const int nI = a.B * a.n_internal, nL = a.B * (a.N - a.n_internal);
   const int blocks = (nI + chunk - 1) / chunk + (nL + chunk - 1) / chunk;
-  kern<<<static_cast<unsigned>(blocks) * chunk, sparse::ST, smem, st>>>(a, redo, chunk);
-  return cudaGetLastError();
+  return launch_after_previous(kern, static_cast<unsigned>(blocks) * chunk, sparse::ST, smem, st, 1, a, redo, chunk);
 }
 template <typename T, bool CFG>
 static cudaError_t launch_sparse(const VerifyArgs& a, int32_t* redo, int e, size_t smem, cudaStream_t st) {
@@ -72,6 +71,7 @@ __global__ void __launch_bounds__(kWalkThreads) walk_kernel(const int32_t* __res
                                                             int32_t* __restrict__ out_tokens,
                                                             int32_t* __restrict__ out_nodes) {
   extern __shared__ int32_t walk_stage[];
+  grid_dependency_sync();
   const int b0 = blockIdx.x * seqs;
   walk_staged(node_next, node_token, tokens, b0, min(seqs, B - b0), N, D1, accept_len, out_tokens, out_nodes,
               walk_stage);
@@ -206,8 +206,10 @@ extern "C" lantern_status lantern_verify_tree(
   if (e != cudaSuccess) return LANTERN_ERR_CUDA;
   if (!a.done) {      // otherwise the repair launch has walked the trees
     const int seqs = std::max(1, std::min(16, 6144 / t->n_nodes));      // 2 * seqs * N ints <= 48 KB
-    walk_kernel<<<(batch + seqs - 1) / seqs, kWalkThreads, sizeof(int32_t) * 2 * seqs * t->n_nodes, st>>>(
-        node_next, node_token, tokens, batch, t->n_nodes, D1, seqs, accept_len, out_tokens, out_nodes);
+    if (launch_after_previous(walk_kernel, static_cast<unsigned>((batch + seqs - 1) / seqs), kWalkThreads,
+                              sizeof(int32_t) * 2 * seqs * t->n_nodes, st, 1, node_next, node_token, tokens, batch,
+                              t->n_nodes, D1, seqs, accept_len, out_tokens, out_nodes) != cudaSuccess)
+      return LANTERN_ERR_CUDA;
     if (cudaGetLastError() != cudaSuccess) return LANTERN_ERR_CUDA;
   }
   return LANTERN_OK;

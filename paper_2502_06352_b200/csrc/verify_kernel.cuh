@@ -855,6 +855,7 @@ __device__ __forceinline__ void verify_node(const VerifyArgs& a, const int idx, 
 #endif
 template <typename T, bool CFG, int E>
 __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const VerifyArgs a) {
+  grid_dependency_sync();
   constexpr int SL = VT * E;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* Q = reinterpret_cast<float*>(smem_raw);

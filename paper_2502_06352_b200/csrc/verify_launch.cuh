@@ -45,7 +45,6 @@ static cudaError_t launch_verify_e(const VerifyArgs& a, const LaunchShape& sh, c
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
   }
-  cudaLaunchConfig_t cfg = {};
   // one cluster per node; a repair launch (a.only) gets about one cluster per SM and lets each
   // walk its share of the flagged nodes
   unsigned clusters = static_cast<unsigned>(a.B) * a.N;
@@ -53,18 +52,7 @@ static cudaError_t launch_verify_e(const VerifyArgs& a, const LaunchShape& sh, c
     const unsigned per_wave = static_cast<unsigned>(sm_count() / sh.cs > 0 ? sm_count() / sh.cs : 1);
     if (clusters > per_wave) clusters = per_wave;
   }
-  cfg.gridDim = dim3(clusters * sh.cs, 1, 1);
-  cfg.blockDim = dim3(VT, 1, 1);
-  cfg.dynamicSmemBytes = sh.smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = sh.cs;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, a);
+  return launch_after_previous(kern, clusters * sh.cs, VT, sh.smem, st, sh.cs, a);
 }
 
 template <typename T, bool CFG>

@@ -289,6 +289,7 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
 // be processed by the dense kernel instead, else to 0.
 template <typename T, bool CFG, int E>
 __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a, int32_t* __restrict__ redo, const int chunk) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem s;
   s.Z = reinterpret_cast<float*>(smem_raw);
