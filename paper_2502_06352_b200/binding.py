@@ -59,7 +59,7 @@ class Params:
 def _load():
     if not os.path.exists(LIB_PATH):
         raise ImportError(
-            "liblantern.so is missing: build it with `python -m paper_2502_06352_b200.build` "
+            "liblantern.so is missing: build it with `python paper_2502_06352_b200/build.py` "
             "(needs nvcc; there is no CPU fallback)")
     L = ctypes.CDLL(LIB_PATH)
     vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
