@@ -44,17 +44,17 @@ struct Ctx {
 };
 
 // Block-wide sum or max of two values per thread; every thread gets the result.
-template <bool IS_MAX>
+template <bool IS_MAX, int NW = SW>
 __device__ __forceinline__ void block_reduce2(Ctx& c, float (&v)[2]) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  float* red = c.red + c.parity * (SW * 2);
+  float* red = c.red + c.parity * (NW * 2);
 #pragma unroll
   for (int i = 0; i < 2; ++i) v[i] = IS_MAX ? warp_max(v[i]) : warp_sum(v[i]);
   if (lane == 0) { red[warp * 2] = v[0]; red[warp * 2 + 1] = v[1]; }
   __syncthreads();
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
-    const float t = lane < SW ? red[lane * 2 + i] : (IS_MAX ? -INFINITY : 0.f);
+    const float t = lane < NW ? red[lane * 2 + i] : (IS_MAX ? -INFINITY : 0.f);
     v[i] = IS_MAX ? warp_max(t) : warp_sum(t);
   }
   c.last_red = red;
@@ -150,7 +150,7 @@ struct Smem {
 // depend on it.
 // With DET the warps' ranges follow warp order (one more barrier instead of the atomic), so the
 // list order is the same from run to run.
-template <int E, bool DET = false>
+template <int E, bool DET = false, bool BITMAP = true>
 __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, int kth, int& n_list,
                                              float& theta) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -250,7 +250,7 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
       const float z = Z[j];
       if (pos < kCap) { ltok[pos] = j; lval[pos] = z; }
       ++pos;
-      atomicOr(&bm[j >> 5], 1u << (j & 31));
+      if (BITMAP) atomicOr(&bm[j >> 5], 1u << (j & 31));
       if (__float_as_uint(mx - z) >= lo_bits) {
         const int cp = atomicAdd(&s.misc[9], 1);
         if (cp < kCand) s.cand[cp] = z;
@@ -285,65 +285,37 @@ __device__ __forceinline__ bool compact_topk(const Smem& s, int side, float mx, 
   return true;
 }
 
-// E = row entries per thread (V <= 512 * E).  `redo[b*N + n]` is set to 1 when node (b, n) has to
-// be processed by the dense kernel instead, else to 0.
-template <typename T, bool CFG, int E>
-__global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a, int32_t* __restrict__ redo, const int chunk) {
-  grid_dependency_sync();
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  Smem s;
-  s.Z = reinterpret_cast<float*>(smem_raw);
-  s.ltok[0] = reinterpret_cast<int*>(s.Z + z_floats(E));
-  s.lval[0] = reinterpret_cast<float*>(s.ltok[0] + kCap);
-  s.ltok[1] = reinterpret_cast<int*>(s.lval[0] + kCap);
-  s.lval[1] = reinterpret_cast<float*>(s.ltok[1] + kCap);
-  s.bins = reinterpret_cast<uint32_t*>(s.lval[1] + kCap);
-  s.bm[0] = s.bins + kBins;
-  s.bm[1] = s.bm[0] + kWords;
-  s.rk = s.bm[1] + kWords;
-  s.cand = reinterpret_cast<float*>(s.rk + kWords);
-  Ctx c;
-  c.red = s.cand + kCand;
-  c.last_red = c.red;
-  c.parity = 0;
-  s.wtot = reinterpret_cast<uint32_t*>(c.red + 2 * SW * 2);
-  s.misc = reinterpret_cast<int*>(s.wtot + SW);
-  uint64_t* mbar = reinterpret_cast<uint64_t*>(s.misc + kMisc);
-  int* nbr_s = reinterpret_cast<int*>(mbar + 2);
-  int* misc = s.misc;
-  float* miscf = reinterpret_cast<float*>(s.misc);
+// Shared memory and identity of the per-node part (union build, sibling loop, draw), which the
+// kernel runs after compacting its two rows.
+struct NodeSmem {
+  int* ut;           // [kUCap]  union arrays: token, target mass, drafter mass
+  float* uq;
+  float* up;
+  uint32_t* bm[2];   // [kWords] support bitmaps of the two lists
+  uint32_t* rk;      // [kWords] union entries before bitmap word w
+  uint32_t* wtot;    // [NT/32]
+  int* misc;         // [kMisc]
+  uint64_t* mbar;
+  int* nbr_s;        // [max_children][kpad]
+};
+struct NodeId {
+  int b, n, fc, nc;
+  long long out_b;
+  const int32_t* tok_b;
+};
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (blockIdx.x == 0 && tid == 0 && a.done) *a.done = 0;      // counter of the repair launch that follows
-  // Launch order: blocks of `chunk` CTAs (one per SM) alternate between internal nodes (two rows,
-  // sibling loop) and leaves (one row), so that the two CTAs sharing an SM start in different
-  // phases and one's streaming overlaps the other's on-chip work.  The grid is padded to whole
-  // blocks; CTAs beyond the last node of their kind leave at once.
-  int idx;
-  {
-    const int nI = a.B * a.n_internal, nL = a.B * (a.N - a.n_internal);
-    const int mI = (nI + chunk - 1) / chunk, mL = (nL + chunk - 1) / chunk;
-    const int c = blockIdx.x / chunk, off = blockIdx.x - c * chunk;
-    const int both = 2 * min(mI, mL);
-    int kind, k;
-    if (c < both) {
-      kind = c & 1;
-      k = (c >> 1) * chunk + off;
-    } else {
-      kind = mI > mL ? 0 : 1;
-      k = (min(mI, mL) + (c - both)) * chunk + off;
-    }
-    if (k >= (kind ? nL : nI)) return;
-    idx = kind ? nI + k : k;            // position in the internal-first node order
-  }
-  const int b = idx % a.B;
-  const int n = a.order[idx / a.B];
-  const int fc = a.first_child[n], nc = a.n_child[n];
-  const int len = min(a.V, ST * E);
-  const long long row_off = static_cast<long long>(b) * a.seq_stride + static_cast<long long>(n) * a.row_stride;
-  const int32_t* tok_b = a.tokens + static_cast<long long>(b) * a.N;
-  const long long out_b = static_cast<long long>(b) * a.N;
-
+// Starts the copy of the children's neighbour rows and fetches the node's uniforms and draft
+// tokens.  Returns whether a bulk copy is in flight (to be awaited by node_tail).
+template <int NT>
+__device__ __forceinline__ bool node_prologue(const VerifyArgs& a, const NodeSmem& ns, const NodeId& id) {
+  const int tid = threadIdx.x;
+  const int n = id.n, fc = id.fc, nc = id.nc;
+  const long long out_b = id.out_b;
+  const int32_t* tok_b = id.tok_b;
+  int* misc = ns.misc;
+  float* miscf = reinterpret_cast<float*>(ns.misc);
+  int* nbr_s = ns.nbr_s;
+  uint64_t* mbar = ns.mbar;
   // ---- stage the children's neighbour rows (bulk async copy when rows are 16-byte aligned)
   const bool want_nbr = nc > 0 && a.k > 0;
   const uint32_t mbar_a = smem_u32(mbar);
@@ -375,7 +347,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     for (int ci = 0; ci < nc; ++ci) {
       int code = tok_b[fc + ci] - a.code_offset;
       if (code >= 0 && code < a.n_codes)
-        for (int r = tid; r < a.k; r += ST)
+        for (int r = tid; r < a.k; r += NT)
           nbr_s[ci * a.kpad + r] = a.nbr[static_cast<long long>(code) * a.k_table + r];
     }
   }
@@ -400,59 +372,60 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     miscf[12 + tid] = u;
     misc[20 + tid] = tok_b[fc + tid];
   }
-  static_assert(kWords == ST, "one bitmap word per thread");
-  s.bm[0][tid] = 0;
-  s.bm[1][tid] = 0;
+  return bulk_issued;
+}
 
-  // ---- both rows, one after the other through the same row buffer
-  const bool masked = a.allow_lo > 0 || a.allow_hi < a.V;
-  const int nside = nc > 0 ? 2 : 1;
-  int n_list[2] = {0, 0};
-  float theta[2] = {INFINITY, INFINITY}, mxs[2] = {0.f, 0.f};
-  bool ok = true;
-  for (int side = 0; side < nside && ok; ++side) {
-    const T* cond = static_cast<const T*>(side ? a.dc : a.tc) + row_off;
-    const T* uncond = CFG ? static_cast<const T*>(side ? a.du : a.tu) + row_off : nullptr;
-    for (int i = tid; i < kBins; i += ST) s.bins[i] = 0;
-    float mx[2];
-    mx[0] = load_row<T, CFG, E>(cond, uncond, a.g, a.inv_tau, len, a.allow_lo, a.allow_hi, masked, s.Z);
-    mx[1] = -INFINITY;
-    block_reduce2<true>(c, mx);
-    if (mx[0] == -INFINITY) { ok = false; break; }           // no finite logit: the dense kernel reports it
-    mxs[side] = mx[0];
-    ok = compact_topk<E>(s, side, mx[0], side ? a.topk_d : a.topk_t, n_list[side], theta[side]);
-  }
-  if (!ok) {
-    // finish the outstanding bulk copy before leaving (bounded), then hand the node over
-    if (bulk_issued) mbar_wait_bounded(mbar_a, 0);
-    if (tid == 0) redo[out_b + n] = 1;
-    return;
-  }
-
+// The per-node part: merges the two lists (token, unnormalised probability; the bitmaps hold their
+// supports) into the union arrays, runs the sibling loop (Sec. 4; App. A.2 Eq. 1-2) and the
+// inverse-CDF draw, and writes the node's results.  NT threads; a barrier must separate the last
+// write of the bitmaps and lists from the call.
+template <int NT>
+__device__ __forceinline__ void node_tail(const VerifyArgs& a, Ctx& c, const NodeSmem& ns, const NodeId& id,
+                                          const bool bulk_issued, const int* ltok0, const float* lval0, const int n0,
+                                          const int* ltok1, const float* lval1, const int n1) {
+  constexpr int NW = NT / 32;
+  static_assert(kWords % NT == 0, "whole bitmap words per thread");
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = id.n, fc = id.fc, nc = id.nc;
+  const long long out_b = id.out_b;
+  const int32_t* tok_b = id.tok_b;
+  int* misc = ns.misc;
+  float* miscf = reinterpret_cast<float*>(ns.misc);
+  int* nbr_s = ns.nbr_s;
+  const uint32_t mbar_a = smem_u32(ns.mbar);
+  const bool want_nbr = nc > 0 && a.k > 0;
   // ---- union of the two supports, ordered by token: popcount ranks of the OR-ed bitmaps, then
-  // every list entry is scattered to its rank as 2^((z - max) log2 e), or 0 below the threshold
-  int* ut = reinterpret_cast<int*>(s.Z);
-  float* uq = s.Z + kUCap;
-  float* up = uq + kUCap;
+  // every list entry is scattered to its rank
+  int* ut = ns.ut;
+  float* uq = ns.uq;
+  float* up = ns.up;
   int n_u;
   {
-    const int cnt = __popc(s.bm[0][tid] | s.bm[1][tid]);
+    constexpr int WPT = kWords / NT;            // bitmap words per thread
+    int before[WPT], cnt = 0;
+#pragma unroll
+    for (int j = 0; j < WPT; ++j) {
+      before[j] = cnt;
+      cnt += __popc(ns.bm[0][tid * WPT + j] | ns.bm[1][tid * WPT + j]);
+    }
     int incl = cnt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int t = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += t;
     }
-    if (lane == 31) s.wtot[warp] = incl;
+    if (lane == 31) ns.wtot[warp] = incl;
     __syncthreads();
-    int wt = lane < SW ? static_cast<int>(s.wtot[lane]) : 0, wincl = wt;
+    int wt = lane < NW ? static_cast<int>(ns.wtot[lane]) : 0, wincl = wt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int t = __shfl_up_sync(0xffffffffu, wincl, o);
       if (lane >= o) wincl += t;
     }
-    s.rk[tid] = static_cast<uint32_t>(__shfl_sync(0xffffffffu, wincl - wt, warp) + incl - cnt);
-    n_u = __shfl_sync(0xffffffffu, wincl, SW - 1);
+    const int base = __shfl_sync(0xffffffffu, wincl - wt, warp) + incl - cnt;
+#pragma unroll
+    for (int j = 0; j < WPT; ++j) ns.rk[tid * WPT + j] = static_cast<uint32_t>(base + before[j]);
+    n_u = __shfl_sync(0xffffffffu, wincl, NW - 1);
   }
   // ---- neighbour rows must have landed
   if (bulk_issued) {
@@ -462,7 +435,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
       for (int ci = 0; ci < nc; ++ci) {
         int code = tok_b[fc + ci] - a.code_offset;
         if (code >= 0 && code < a.n_codes)
-          for (int r = tid; r < a.k; r += ST)
+          for (int r = tid; r < a.k; r += NT)
             nbr_s[ci * a.kpad + r] = a.nbr[static_cast<long long>(code) * a.k_table + r];
       }
     }
@@ -470,20 +443,21 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
   __syncthreads();
   // position of token t in the union arrays, or -1
   auto uidx = [&](int t) -> int {
-    const uint32_t w = s.bm[0][t >> 5] | s.bm[1][t >> 5], bit = 1u << (t & 31);
-    return (w & bit) ? static_cast<int>(s.rk[t >> 5]) + __popc(w & (bit - 1u)) : -1;
+    const uint32_t w = ns.bm[0][t >> 5] | ns.bm[1][t >> 5], bit = 1u << (t & 31);
+    return (w & bit) ? static_cast<int>(ns.rk[t >> 5]) + __popc(w & (bit - 1u)) : -1;
   };
 #pragma unroll
   for (int side = 0; side < 2; ++side) {
-    const float c0 = -mxs[side] * kLog2e;
     float* mine = side ? up : uq;
     float* other = side ? uq : up;
-    const uint32_t* obm = s.bm[side ^ 1];
-    for (int i = tid; i < n_list[side]; i += ST) {
-      const int t = s.ltok[side][i], u = uidx(t);
-      const float z = s.lval[side][i];
+    const uint32_t* obm = ns.bm[side ^ 1];
+    const int* lt = side ? ltok1 : ltok0;
+    const float* lv = side ? lval1 : lval0;
+    const int nl = side ? n1 : n0;
+    for (int i = tid; i < nl; i += NT) {
+      const int t = lt[i], u = uidx(t);
       ut[u] = t;
-      mine[u] = z >= theta[side] ? ex2_approx(fmaf(z, kLog2e, c0)) : 0.f;
+      mine[u] = lv[i];
       if (!((obm[t >> 5] >> (t & 31)) & 1u)) other[u] = 0.f;
     }
   }
@@ -494,7 +468,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     misc[28 + tid] = (x >= 0 && x < a.V) ? uidx(x) : -1;
   }
   if (want_nbr) {
-    for (int i = tid; i < nc * a.k; i += ST) {
+    for (int i = tid; i < nc * a.k; i += NT) {
       const int ci = i / a.k, r = i - ci * a.k;
       const int t = a.code_offset + nbr_s[ci * a.kpad + r];
       nbr_s[ci * a.kpad + r] = (t >= 0 && t < a.V) ? uidx(t) : -2;
@@ -504,11 +478,11 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
   // From here on thread t owns the union entries [t*per, t*per + per) in every sweep, so that a
   // thread re-reads only what it wrote itself and the per-warp partial sums of a reduction are
   // sums over consecutive tokens.  per is odd: consecutive threads hit different banks.
-  const int per = ((n_u + ST - 1) / ST) | 1;
+  const int per = ((n_u + NT - 1) / NT) | 1;
   const int i0 = min(tid * per, n_u), i1 = min(i0 + per, n_u);
   float tot[2] = {0.f, 0.f};
   for (int i = i0; i < i1; ++i) { tot[0] += uq[i]; tot[1] += up[i]; }
-  block_reduce2<false>(c, tot);
+  block_reduce2<false, NW>(c, tot);
   float qtot = tot[0];
   float qs = qtot > 0.f ? 1.f / qtot : 0.f;
   float psum = tot[1];
@@ -615,7 +589,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
       if (i == ix) { up[i] = 0.f; p = 0.f; }
       if (resum) zs[1] += p;
     }
-    block_reduce2<false>(c, zs);
+    block_reduce2<false, NW>(c, zs);
     const float ps_old = ps;
     psum = resum ? zs[1] : psum - pxraw;
     if (zs[0] > 0.f) {
@@ -629,7 +603,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
         uq[i] = p;
         s2[0] += p;
       }
-      block_reduce2<false>(c, s2);
+      block_reduce2<false, NW>(c, s2);
       qtot = s2[0];
       qs = ps_old;
     }
@@ -648,7 +622,7 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     float sc = 0.f;
     for (int i = i0; i < i1; ++i) sc += uq[i];
     const float incl = warp_incl_scan(sc, lane);
-    const float wt = lane < SW ? c.last_red[lane * 2] : 0.f;
+    const float wt = lane < NW ? c.last_red[lane * 2] : 0.f;
     const float wincl = warp_incl_scan(wt, lane);
     float run = __shfl_sync(0xffffffffu, wincl - wt, warp) + (incl - sc);
     int cand = 0x7fffffff, lastp = -1;
@@ -665,8 +639,8 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
     if (lane == 0) { misc[64 + warp] = cand; misc[80 + warp] = lastp; }
     __syncthreads();
     if (warp == 0) {
-      cand = __reduce_min_sync(0xffffffffu, lane < SW ? misc[64 + lane] : 0x7fffffff);
-      lastp = __reduce_max_sync(0xffffffffu, lane < SW ? misc[80 + lane] : -1);
+      cand = __reduce_min_sync(0xffffffffu, lane < NW ? misc[64 + lane] : 0x7fffffff);
+      lastp = __reduce_max_sync(0xffffffffu, lane < NW ? misc[80 + lane] : -1);
       if (lane == 0) {
         const int found = cand != 0x7fffffff ? cand : lastp;
         a.node_token[out_b + n] = found >= 0 ? ut[found] : -1;
@@ -676,10 +650,119 @@ __global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a
   } else if (tid == 0) {
     a.node_token[out_b + n] = -1;
   }
-  if (tid == 0) {
-    a.node_next[out_b + n] = accepted;
-    redo[out_b + n] = 0;
+  if (tid == 0) a.node_next[out_b + n] = accepted;
+}
+
+// ------------------------------------------------------------------------------------------------
+// One CTA of 512 threads per node does everything (both rows, then the per-node part).
+// E = row entries per thread (V <= 512 * E).
+// `redo[b*N + n]` is set to 1 when node (b, n) has to be processed by the dense kernel instead, else to 0.
+template <typename T, bool CFG, int E>
+__global__ void __launch_bounds__(ST, 2) verify_sparse_kernel(const VerifyArgs a, int32_t* __restrict__ redo, const int chunk) {
+  grid_dependency_sync();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Smem s;
+  s.Z = reinterpret_cast<float*>(smem_raw);
+  s.ltok[0] = reinterpret_cast<int*>(s.Z + z_floats(E));
+  s.lval[0] = reinterpret_cast<float*>(s.ltok[0] + kCap);
+  s.ltok[1] = reinterpret_cast<int*>(s.lval[0] + kCap);
+  s.lval[1] = reinterpret_cast<float*>(s.ltok[1] + kCap);
+  s.bins = reinterpret_cast<uint32_t*>(s.lval[1] + kCap);
+  s.bm[0] = s.bins + kBins;
+  s.bm[1] = s.bm[0] + kWords;
+  s.rk = s.bm[1] + kWords;
+  s.cand = reinterpret_cast<float*>(s.rk + kWords);
+  Ctx c;
+  c.red = s.cand + kCand;
+  c.last_red = c.red;
+  c.parity = 0;
+  s.wtot = reinterpret_cast<uint32_t*>(c.red + 2 * SW * 2);
+  s.misc = reinterpret_cast<int*>(s.wtot + SW);
+  NodeSmem ns;
+  ns.ut = reinterpret_cast<int*>(s.Z);          // the union arrays take over the row buffer
+  ns.uq = s.Z + kUCap;
+  ns.up = ns.uq + kUCap;
+  ns.bm[0] = s.bm[0];
+  ns.bm[1] = s.bm[1];
+  ns.rk = s.rk;
+  ns.wtot = s.wtot;
+  ns.misc = s.misc;
+  ns.mbar = reinterpret_cast<uint64_t*>(s.misc + kMisc);
+  ns.nbr_s = reinterpret_cast<int*>(ns.mbar + 2);
+
+  const int tid = threadIdx.x;
+  if (blockIdx.x == 0 && tid == 0 && a.done) *a.done = 0;      // counter of the repair launch that follows
+  // Launch order: blocks of `chunk` CTAs (one per SM) alternate between internal nodes (two rows,
+  // sibling loop) and leaves (one row), so that the two CTAs sharing an SM start in different
+  // phases and one's streaming overlaps the other's on-chip work.  The grid is padded to whole
+  // blocks; CTAs beyond the last node of their kind leave at once.
+  int idx;
+  {
+    const int nI = a.B * a.n_internal, nL = a.B * (a.N - a.n_internal);
+    const int mI = (nI + chunk - 1) / chunk, mL = (nL + chunk - 1) / chunk;
+    const int cb = blockIdx.x / chunk, off = blockIdx.x - cb * chunk;
+    const int both = 2 * min(mI, mL);
+    int kind, k;
+    if (cb < both) {
+      kind = cb & 1;
+      k = (cb >> 1) * chunk + off;
+    } else {
+      kind = mI > mL ? 0 : 1;
+      k = (min(mI, mL) + (cb - both)) * chunk + off;
+    }
+    if (k >= (kind ? nL : nI)) return;
+    idx = kind ? nI + k : k;            // position in the internal-first node order
   }
+  NodeId id;
+  id.b = idx % a.B;
+  id.n = a.order[idx / a.B];
+  id.fc = a.first_child[id.n];
+  id.nc = a.n_child[id.n];
+  id.out_b = static_cast<long long>(id.b) * a.N;
+  id.tok_b = a.tokens + id.out_b;
+  const int len = min(a.V, ST * E);
+  const long long row_off = static_cast<long long>(id.b) * a.seq_stride + static_cast<long long>(id.n) * a.row_stride;
+
+  const bool bulk_issued = node_prologue<ST>(a, ns, id);
+  static_assert(kWords == ST, "one bitmap word per thread");
+  s.bm[0][tid] = 0;
+  s.bm[1][tid] = 0;
+
+  // ---- both rows, one after the other through the same row buffer
+  const bool masked = a.allow_lo > 0 || a.allow_hi < a.V;
+  const int nside = id.nc > 0 ? 2 : 1;
+  int n_list[2] = {0, 0};
+  bool ok = true;
+  for (int side = 0; side < nside && ok; ++side) {
+    const T* cond = static_cast<const T*>(side ? a.dc : a.tc) + row_off;
+    const T* uncond = CFG ? static_cast<const T*>(side ? a.du : a.tu) + row_off : nullptr;
+    for (int i = tid; i < kBins; i += ST) s.bins[i] = 0;
+    float mx[2];
+    mx[0] = load_row<T, CFG, E>(cond, uncond, a.g, a.inv_tau, len, a.allow_lo, a.allow_hi, masked, s.Z);
+    mx[1] = -INFINITY;
+    block_reduce2<true>(c, mx);
+    if (mx[0] == -INFINITY) { ok = false; break; }           // no finite logit: the dense kernel reports it
+    float theta;
+    ok = compact_topk<E>(s, side, mx[0], side ? a.topk_d : a.topk_t, n_list[side], theta);
+    if (ok) {
+      // list values become 2^((z - max) log2 e), or 0 below the threshold; the same thread reads
+      // them back when the lists are merged
+      const float c0 = -mx[0] * kLog2e;
+      float* lv = s.lval[side];
+      for (int i = tid; i < n_list[side]; i += ST) {
+        const float z = lv[i];
+        lv[i] = z >= theta ? ex2_approx(fmaf(z, kLog2e, c0)) : 0.f;
+      }
+    }
+  }
+  if (!ok) {
+    // finish the outstanding bulk copy before leaving (bounded), then hand the node over
+    if (bulk_issued) mbar_wait_bounded(smem_u32(ns.mbar), 0);
+    if (tid == 0) redo[id.out_b + id.n] = 1;
+    return;
+  }
+  node_tail<ST>(a, c, ns, id, bulk_issued, s.ltok[0], s.lval[0], n_list[0], s.ltok[1], s.lval[1], n_list[1]);
+  if (tid == 0) redo[id.out_b + id.n] = 0;
 }
 
 }  // namespace sparse
