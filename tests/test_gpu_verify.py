@@ -92,6 +92,43 @@ def test_topk_with_massive_ties_is_repaired_by_the_dense_kernel(L):
     _run(L, case)
 
 
+def test_path_queries_and_graph_replay_match_eager_calls(L):
+    """The library says which kernels a call runs; a captured and replayed call (the way the
+    benchmark launches) gives the results of the eager call bit for bit."""
+    case = Case(small_config(vocab=3001, codebook_size=3001, top_k=200, k=12), seed=17, pad=3)
+    g, par, nbr, tok = case.gpu_inputs(L)
+    tree = L.Tree(case.parent)
+    assert L.verify_tree_path(par, tree) == 1 and L.sample_draft_tree_path(par) == 1
+    par_dense = L.Params(**{**par.__dict__, "top_k_target": 0, "top_k_draft": 0})
+    assert L.verify_tree_path(par_dense, tree) == 0 and L.sample_draft_tree_path(par_dense) == 0
+    old = L.set_cluster_size(1)
+    try:
+        assert L.verify_tree_path(par, tree) == 0
+    finally:
+        L.set_cluster_size(old)
+    ua, ur = case.u_accept.cuda(), case.u_resample.cuda()
+    eager = {k: v.clone() for k, v in L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"],
+                                                    g["draft_cond"], g["draft_uncond"], tok, ua, ur, debug=True).items()}
+    out = {}
+    ws = torch.empty(L.lib.lantern_verify_tree_workspace(tree.handle, case.B), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):      # warm-up outside the capture (function attributes are set here)
+        L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"],
+                      tok, ua, ur, debug=True, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(2):               # two dependent calls: the second overwrites the first's results
+            L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"],
+                          tok, ua, ur, debug=True, out=out, workspace=ws)
+    for v in out.values():
+        v.fill_(-3)
+    graph.replay()
+    torch.cuda.synchronize()
+    for k, v in eager.items():
+        assert torch.equal(out[k], v), k
+
+
 def test_allowed_range_and_topk_counts_only_allowed(L):
     case = Case(small_config(vocab=2048, codebook_size=512, code_offset=256, k=6, top_k=40), seed=3,
                 allowed=(256, 768))
