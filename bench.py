@@ -158,7 +158,7 @@ def oracle_run_nodes(cfg, parent, lg, b, gum, ua, ur, nbr, n_nodes):
     return done
 
 
-def cpu_baseline(cfg, parent, lg_cpu, budget_s=15.0):
+def cpu_baseline(cfg, parent, lg_cpu, budget_s=12.0):
     """The oracle, as it stands, on whole sequences of the workload until about budget_s."""
     N = len(parent)
     B = lg_cpu["target_cond"].shape[0]
@@ -170,7 +170,7 @@ def cpu_baseline(cfg, parent, lg_cpu, budget_s=15.0):
         b = seqs % B
         nodes += oracle_run_nodes(cfg, parent, lg_cpu, b, gum[b], ua[b], ur[b], nbr, N)
         seqs += 1
-        if time.perf_counter() - t0 > budget_s or seqs >= 4 * B:
+        if time.perf_counter() - t0 > budget_s or seqs >= 256 * B:
             break
     dt = time.perf_counter() - t0
     return {"value": nodes / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
