@@ -129,6 +129,26 @@ def test_path_queries_and_graph_replay_match_eager_calls(L):
         assert torch.equal(out[k], v), k
 
 
+def test_topk_rows_without_workspace_take_the_dense_kernel(L):
+    # node_next / node_token are given and the workspace is too small for the repair flags: the
+    # call is still valid (the dense kernel and the separate walk launch run) and gives the same results
+    case = Case(small_config(top_k=50), seed=18)
+    g, par, nbr, tok = case.gpu_inputs(L)
+    tree = L.Tree(case.parent)
+    ua, ur = case.u_accept.cuda(), case.u_resample.cuda()
+    full = L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"],
+                         tok, ua, ur, debug=True)
+    tiny = L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"],
+                         tok, ua, ur, debug=True, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    torch.cuda.synchronize()
+    for k in ("accept_len", "out_tokens", "out_nodes", "node_next", "node_token"):
+        assert torch.equal(full[k], tiny[k]), k
+    for k in ("node_mass", "node_thresh"):
+        assert torch.allclose(full[k], tiny[k], atol=1e-5), k
+    res = {k: v.cpu().numpy() for k, v in tiny.items()}
+    compare_verify(res, case.oracle_verify(), case.parent, case.u_accept.numpy(), case.seqs)
+
+
 def test_allowed_range_and_topk_counts_only_allowed(L):
     case = Case(small_config(vocab=2048, codebook_size=512, code_offset=256, k=6, top_k=40), seed=3,
                 allowed=(256, 768))
