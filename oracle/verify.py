@@ -14,6 +14,9 @@ Readings where the paper is silent:
    positive part of q~ - p (Eq. 2), and the drafter is renormalised without x
  * the token drawn when no child is accepted (or at a leaf) uses inverse-CDF
    sampling in token-id order
+ * additive variant (Sec. 2.2, LANTERN's bound, delta > 0): neighbours join A
+   while the mass they add to x, i.e. the total-variation distance between q
+   and q~, stays strictly below delta; q(x) itself does not count against delta
 """
 
 import numpy as np
@@ -22,13 +25,15 @@ from .postprocess import postprocess_row
 from .tree import tree_children
 
 
-def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None):
+def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None, delta=0.0):
     """Sec. 4: m = sum of q over A_{k,lambda}(x) and the members of A besides x.
+    With delta > 0 the additive bound of Sec. 2.2 replaces the multiplicative one:
+    the neighbours' own running sum stays below delta (A_{k,delta}); lam is unused.
 
     If `margins` is a list, |running sum - bound| of every comparison made is
     appended to it (diagnostic for near-tie accounting; no effect on the result)."""
     cum = q_cur[x]
-    bound = lam * q_cur[x]
+    bound = q_cur[x] + delta if delta > 0 else lam * q_cur[x]
     members = []
     code = x - code_offset
     if 0 <= code < n_codes:
@@ -53,7 +58,7 @@ def moved_mass(q_cur, x, m, members):
     return q_t
 
 
-def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset, n_codes):
+def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset, n_codes, delta=0.0):
     """Test the children of one node in stored order (Sec. 4; App. A.2 Eq. 1-2).
 
     Returns (accepted child or -1, q_cur, {child: (m, thr, cut_margin)}): q_cur
@@ -67,7 +72,7 @@ def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset
         if x < 0:
             continue
         margins = []
-        m, members = relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins)
+        m, members = relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins, delta)
         if p_cur[x] > 0:
             thr = min(1.0, m / p_cur[x])          # Sec. 4, final accept probability
         else:
@@ -98,7 +103,7 @@ def inverse_cdf(dist, u, return_margin=False):
 
 
 def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
-                code_offset, n_codes):
+                code_offset, n_codes, delta=0.0):
     """Process one tree node.
 
     q: target distribution of the node; p: drafter distribution (None at a leaf)
@@ -108,7 +113,7 @@ def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
     tested["resample_margin"] is set when a token was drawn.
     """
     nxt, q_cur, tested = sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam,
-                                      code_offset, n_codes)
+                                      code_offset, n_codes, delta)
     if nxt >= 0:
         return nxt, -1, tested
     j, margin = inverse_cdf(q_cur, u_resample, return_margin=True)
@@ -135,7 +140,7 @@ def walk(node_next, node_token, tokens):
 def verify_sequence(parent, target_cond, target_uncond, draft_cond, draft_uncond, tokens,
                     u_accept, u_resample, nbr_idx, *, cfg_scale=1.0, temperature=1.0,
                     top_k_target=0, top_k_draft=0, lam=1.0, k=0, code_offset=0, n_codes=0,
-                    allowed_begin=0, allowed_end=None):
+                    allowed_begin=0, allowed_end=None, delta=0.0):
     """Verify one sequence's tree.  Logit arrays are [N][V]; uncond may be None.
 
     Returns a dict with node_next, node_token (int arrays [N]), node_mass,
@@ -158,7 +163,7 @@ def verify_sequence(parent, target_cond, target_uncond, draft_cond, draft_uncond
             p, _ = postprocess_row(draft_cond[n], None if draft_uncond is None else draft_uncond[n],
                                    cfg_scale, temperature, top_k_draft, allowed_begin, allowed_end)
         nxt, tok, tested = verify_node(q, p, children[n], tokens, u_accept, u_resample[n],
-                                       nbr_idx, k, lam, code_offset, n_codes)
+                                       nbr_idx, k, lam, code_offset, n_codes, delta)
         node_next[n], node_token[n] = nxt, tok
         resample_margin[n] = tested.pop("resample_margin", np.inf)
         for c, (m, thr, cm) in tested.items():

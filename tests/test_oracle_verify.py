@@ -83,6 +83,45 @@ def test_bound_on_accept_probability_and_monotonicity():
             prev = row
 
 
+def test_additive_bound_is_a_bound_on_the_total_variation_distance():
+    """Sec. 2.2 (LANTERN's rule, delta > 0): A = longest prefix of the neighbour list whose own
+    running sum stays strictly below delta, computed via cumsum; the distortion TVD(q, q~) is the
+    moved mass and therefore < delta; delta -> 0 gives Eq. 1, delta > 1 takes all k neighbours;
+    with delta = (lambda - 1) q(x) both rules draw the same set."""
+    rng = np.random.default_rng(33)
+    V, k = 32, 12
+    nbr = _table(rng, V, k)
+    for trial in range(300):
+        q, p = _dists(rng, V, conc=0.3)
+        x = int(rng.integers(V))
+        kk = int(rng.integers(0, k + 1))
+        delta = float(rng.choice([1e-9, 0.01, 0.05, 0.2, 0.5, 2.0]))
+        m, members = oracle.relaxed_mass(q, x, nbr, kk, 1.0, 0, V, delta=delta)
+        run = np.cumsum(q[nbr[x][:kk]])
+        ok = run < delta
+        n_take = kk if ok.all() else int(np.argmin(ok))
+        assert members == [int(a) for a in nbr[x][:n_take]]
+        assert np.isclose(m, q[x] + q[nbr[x][:n_take]].sum(), rtol=1e-14)
+        qt = oracle.moved_mass(q, x, m, members)
+        tvd = 0.5 * np.abs(qt - q).sum()
+        assert abs(tvd - (m - q[x])) < 1e-13 and (tvd < delta or n_take == 0)
+        if delta == 2.0:
+            assert n_take == kk
+        if delta == 1e-9:
+            assert all(q[a] < 1e-9 for a in members)
+        # the accept probability uses m exactly as in the multiplicative rule
+        _, _, tested = oracle.sibling_loop(q, p, [1], [0, x], [0, 1.0], nbr, kk, 1.0, 0, V, delta=delta)
+        assert tested[1][0] == m and tested[1][1] == (min(1.0, m / p[x]) if p[x] > 0 else float(m > 0))
+        # same bound, written either way
+        lam = float(rng.choice([1.5, 3.0, 8.0]))
+        if q[x] > 0:
+            m_l, mem_l = oracle.relaxed_mass(q, x, nbr, kk, lam, 0, V)
+            m_d, mem_d = oracle.relaxed_mass(q, x, nbr, kk, 1.0, 0, V, delta=(lam - 1.0) * q[x])
+            bound = lam * q[x]
+            near = np.abs(q[x] + np.cumsum(q[nbr[x][:kk]]) - bound).min() < 1e-12 if kk else False
+            assert near or (mem_l == mem_d and np.isclose(m_l, m_d, rtol=1e-14))
+
+
 def test_moved_mass_is_a_distribution_with_tvd_equal_to_moved_mass():
     rng = np.random.default_rng(3)
     V, k = 20, 8
