@@ -84,6 +84,10 @@ typedef struct {
   int32_t allowed_end;     /* 0 means V                                                         */
   uint64_t seed;           /* Philox-4x32-10 key; used only where uniforms are not supplied     */
   uint64_t step;           /* counter base, < 2^62: change it every decode step                 */
+  float delta;             /* 0: multiplicative bound lambda (Sec. 4).  > 0: additive bound of
+                              Sec. 2.2 instead (lambda unused): neighbours join A while their own
+                              running sum of q stays < delta, i.e. TVD(q, q~) < delta            */
+  int32_t reserved;        /* set to 0 */
 } lantern_params;
 
 /* ---- (1) latent-neighbour table -------------------------------------------------------------
@@ -131,6 +135,7 @@ lantern_status lantern_sample_draft_tree(const lantern_params* params, const lan
  *   for each child c with token x:
  *     A = {x} + longest prefix of x's neighbour list (first k entries of the table row) whose
  *         running sum of q_cur, q_cur(x) included, stays < lambda * q_cur(x);   m = sum_A q_cur
+ *         (params->delta > 0, Sec. 2.2: ... whose own running sum stays < delta instead)
  *     accept c iff u_accept[c] < min(1, m / p_cur(x))
  *     on rejection: move A's mass onto x, q_cur = normalise([q~ - p_cur]_+), drop x from p_cur
  *   if no child was accepted (or n is a leaf): node_token[n] = inverse-CDF sample of q_cur with

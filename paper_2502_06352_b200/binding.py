@@ -30,6 +30,7 @@ class _CParams(ctypes.Structure):
         ("code_offset", ctypes.c_int32), ("n_codes", ctypes.c_int32),
         ("allowed_begin", ctypes.c_int32), ("allowed_end", ctypes.c_int32),
         ("seed", ctypes.c_uint64), ("step", ctypes.c_uint64),
+        ("delta", ctypes.c_float), ("reserved", ctypes.c_int32),
     ]
 
 
@@ -49,11 +50,12 @@ class Params:
     allowed_end: int = 0
     seed: int = 0
     step: int = 0
+    delta: float = 0.0
 
     def c(self):
         return _CParams(self.cfg_scale, self.temperature, self.top_k_target, self.top_k_draft,
                         self.lam, self.k, self.vocab, self.code_offset, self.n_codes,
-                        self.allowed_begin, self.allowed_end, self.seed, self.step)
+                        self.allowed_begin, self.allowed_end, self.seed, self.step, self.delta, 0)
 
 
 def _load():

@@ -164,7 +164,7 @@ struct VerifyArgs {
   int k_table, use_bulk;
   const int32_t *first_child, *n_child, *order;
   int B, N, V, kpad, n_internal;
-  float g, inv_tau, lambda;
+  float g, inv_tau, lambda, delta;
   int topk_t, topk_d, k, code_offset, n_codes, allow_lo, allow_hi;
   unsigned long long seed, step;
   int32_t *node_next, *node_token;

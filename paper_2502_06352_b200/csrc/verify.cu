@@ -127,6 +127,7 @@ extern "C" lantern_status lantern_verify_tree(
   if (t->n_internal > 0 && !draft_cond) return LANTERN_ERR_INVALID_ARG;
   if ((target_uncond != nullptr) != (draft_uncond != nullptr) && t->n_internal > 0) return LANTERN_ERR_INVALID_ARG;
   if (p->k < 0 || p->top_k_target < 0 || p->top_k_draft < 0) return LANTERN_ERR_INVALID_ARG;
+  if (!(p->delta >= 0.f) || p->delta > 4.f) return LANTERN_ERR_INVALID_ARG;      // also rejects NaN
   if (p->k > 0 && (!nbr_idx || p->k > k_table || p->n_codes <= 0 || k_table > p->n_codes - 1)) return LANTERN_ERR_INVALID_ARG;
   if (p->k > 1024) return LANTERN_ERR_UNSUPPORTED;
   const int V = p->vocab;
@@ -162,7 +163,7 @@ extern "C" lantern_status lantern_verify_tree(
   a.first_child = t->d_first_child; a.n_child = t->d_n_child; a.order = t->d_order;
   a.B = batch; a.N = t->n_nodes; a.V = V; a.n_internal = t->n_internal;
   a.kpad = (p->k + 3) & ~3;
-  a.g = p->cfg_scale; a.inv_tau = 1.0f / p->temperature; a.lambda = p->lambda;
+  a.g = p->cfg_scale; a.inv_tau = 1.0f / p->temperature; a.lambda = p->lambda; a.delta = p->delta;
   a.topk_t = p->top_k_target; a.topk_d = p->top_k_draft; a.k = p->k;
   a.code_offset = p->code_offset; a.n_codes = p->n_codes; a.allow_lo = allow_lo; a.allow_hi = allow_hi;
   a.seed = p->seed; a.step = p->step;

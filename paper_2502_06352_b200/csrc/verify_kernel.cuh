@@ -652,7 +652,7 @@ __device__ __forceinline__ void verify_node(const VerifyArgs& a, const int idx, 
       const float qx = row_at(Q, q_base, x) * qs;
       const float pxraw = row_at(P, p_base, x);
       const float px = pxraw * ps;
-      const float bound = a.lambda * qx;
+      const float bound = a.delta > 0.f ? qx + a.delta : a.lambda * qx;      // Sec. 2.2 / Sec. 4
       float cum = qx;
       int nA = 0;
       bool bad = false, open = has_code;

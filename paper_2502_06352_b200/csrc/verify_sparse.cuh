@@ -516,7 +516,7 @@ __device__ __forceinline__ void node_tail(const VerifyArgs& a, Ctx& c, const Nod
       const float qx = ix >= 0 ? uq[ix] * qs : 0.f;
       const float pxraw = ix >= 0 ? up[ix] : 0.f;
       const float px = pxraw * ps;
-      const float bound = a.lambda * qx;
+      const float bound = a.delta > 0.f ? qx + a.delta : a.lambda * qx;      // Sec. 2.2 / Sec. 4
       float cum = qx;
       int nA = 0;
       bool bad = false, open = has_code;

@@ -24,7 +24,7 @@ class Case:
     """Inputs of one call (CPU tensors) and everything the oracle says about them."""
 
     def __init__(self, cfg, parent=None, seed=0, allowed=(0, 0), k_table=None, temperature=None,
-                 top_k_target=None, top_k_draft=None, pad=0, oracle_seqs=None, tokens="oracle"):
+                 top_k_target=None, top_k_draft=None, pad=0, oracle_seqs=None, tokens="oracle", delta=0.0):
         self.cfg = cfg
         self.parent = W.static_tree(cfg.n_nodes) if parent is None else parent
         N, B, V = len(self.parent), cfg.batch, cfg.vocab
@@ -46,7 +46,7 @@ class Case:
             top_k_target=cfg.top_k if top_k_target is None else top_k_target,
             top_k_draft=cfg.top_k if top_k_draft is None else top_k_draft,
             lam=cfg.lam, k=cfg.k, code_offset=cfg.code_offset, n_codes=cfg.codebook_size,
-            allowed_begin=allowed[0], allowed_end=allowed[1] if allowed[1] else V)
+            allowed_begin=allowed[0], allowed_end=allowed[1] if allowed[1] else V, delta=delta)
         self.seqs = list(range(B)) if oracle_seqs is None else list(oracle_seqs)
         # draft tokens: oracle sampler on the checked sequences, uniform random elsewhere
         lo, hi = self.params["allowed_begin"], self.params["allowed_end"]
@@ -90,7 +90,7 @@ class Case:
         par = L.Params(vocab=self.V, cfg_scale=p["cfg_scale"], temperature=p["temperature"],
                        top_k_target=p["top_k_target"], top_k_draft=p["top_k_draft"], lam=p["lam"], k=p["k"],
                        code_offset=p["code_offset"], n_codes=p["n_codes"], allowed_begin=p["allowed_begin"],
-                       allowed_end=p["allowed_end"])
+                       allowed_end=p["allowed_end"], delta=p["delta"])
         nbr = None if self.nbr is None else torch.from_numpy(self.nbr).to(dev)
         tok = torch.from_numpy(self.tokens.astype(np.int32)).to(dev)
         return g, par, nbr, tok

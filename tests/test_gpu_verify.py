@@ -149,6 +149,18 @@ def test_topk_rows_without_workspace_take_the_dense_kernel(L):
     compare_verify(res, case.oracle_verify(), case.parent, case.u_accept.numpy(), case.seqs)
 
 
+@pytest.mark.parametrize("delta", [0.02, 0.3, 2.0])
+@pytest.mark.parametrize("kw", [dict(k=10), dict(k=16, top_k=100, vocab=3001, codebook_size=3001)])
+def test_additive_bound_variant(L, delta, kw):
+    # Sec. 2.2: neighbours are aggregated while their own mass stays below delta (lambda unused);
+    # dense kernel (first case) and list kernel (second case)
+    case = Case(small_config(lam=1.0, **kw), seed=19, delta=delta, pad=3 if "vocab" in kw else 0)
+    res, stats = _run(L, case)
+    if delta == 2.0:        # every neighbour joins: m = q(x) + sum over all k neighbours
+        orc = case.oracle_verify()
+        assert all(np.all(o["cut_margin"][np.isfinite(o["cut_margin"])] > 0.5) for o in orc)
+
+
 def test_allowed_range_and_topk_counts_only_allowed(L):
     case = Case(small_config(vocab=2048, codebook_size=512, code_offset=256, k=6, top_k=40), seed=3,
                 allowed=(256, 768))
