@@ -87,7 +87,12 @@ typedef struct {
   float delta;             /* 0: multiplicative bound lambda (Sec. 4).  > 0: additive bound of
                               Sec. 2.2 instead (lambda unused): neighbours join A while their own
                               running sum of q stays < delta, i.e. TVD(q, q~) < delta            */
-  int32_t reserved;        /* set to 0 */
+  int32_t lazy_walk;       /* lantern_verify_tree only.  0: every node of the tree is verified
+                              (one launch over B*N nodes), then the walk.  1: path walk (Sec. 2.1):
+                              one thread-block cluster per sequence verifies the root, moves to
+                              the accepted child and so on, reading only the rows on the accepted
+                              path; accept_len / out_tokens / out_nodes are the same, the per-node
+                              outputs are written for the nodes on the path only                */
 } lantern_params;
 
 /* ---- (1) latent-neighbour table -------------------------------------------------------------

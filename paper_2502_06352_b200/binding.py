@@ -30,7 +30,7 @@ class _CParams(ctypes.Structure):
         ("code_offset", ctypes.c_int32), ("n_codes", ctypes.c_int32),
         ("allowed_begin", ctypes.c_int32), ("allowed_end", ctypes.c_int32),
         ("seed", ctypes.c_uint64), ("step", ctypes.c_uint64),
-        ("delta", ctypes.c_float), ("reserved", ctypes.c_int32),
+        ("delta", ctypes.c_float), ("lazy_walk", ctypes.c_int32),
     ]
 
 
@@ -51,11 +51,12 @@ class Params:
     seed: int = 0
     step: int = 0
     delta: float = 0.0
+    lazy_walk: int = 0
 
     def c(self):
         return _CParams(self.cfg_scale, self.temperature, self.top_k_target, self.top_k_draft,
                         self.lam, self.k, self.vocab, self.code_offset, self.n_codes,
-                        self.allowed_begin, self.allowed_end, self.seed, self.step, self.delta, 0)
+                        self.allowed_begin, self.allowed_end, self.seed, self.step, self.delta, self.lazy_walk)
 
 
 def _load():

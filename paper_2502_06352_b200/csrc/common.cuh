@@ -172,6 +172,7 @@ struct VerifyArgs {
   int32_t* status;
   const int32_t* only;     // [B*N] or NULL: process only the nodes whose entry is non-zero
   // set together with `only`: the last CTA to finish also walks the trees (no separate launch)
+  int lazy;                // non-zero: one cluster per sequence walks the accepted path (no `only`, no `done`)
   int32_t* done;           // one counter, zero before the launch and again after it
   int32_t *accept_len, *out_tokens, *out_nodes;
   int D1;

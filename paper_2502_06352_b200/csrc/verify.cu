@@ -95,7 +95,7 @@ constexpr int kWsTailInts = 64;
 bool verify_uses_lists(const lantern_params* p, const TreeDev* t) {
   const int V = p->vocab;
   auto topk_fits = [&](int k) { return k > 0 && k < V && k <= sparse::kMaxTopK; };
-  return g_cluster_override == 0 && V <= sparse::kMaxV && topk_fits(p->top_k_target) &&
+  return !p->lazy_walk && g_cluster_override == 0 && V <= sparse::kMaxV && topk_fits(p->top_k_target) &&
          (t->n_internal == 0 || topk_fits(p->top_k_draft)) && t->max_children <= 8;
 }
 }  // namespace
@@ -171,16 +171,17 @@ extern "C" lantern_status lantern_verify_tree(
   a.status = device_status;
   a.only = nullptr;
   a.done = nullptr;
+  a.lazy = p->lazy_walk ? 1 : 0;
   const int D1 = t->max_depth + 1;
   a.accept_len = accept_len; a.out_tokens = out_tokens; a.out_nodes = out_nodes; a.D1 = D1;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = target_uncond != nullptr;
   const bool f32 = dt == LANTERN_F32;
-  const int min_e = f32 ? 4 : 8, rows = batch * t->n_nodes;
+  const int min_e = f32 ? 4 : 8, rows = a.lazy ? batch : batch * t->n_nodes;
   cudaError_t e;
   // Rows truncated to a moderate top-k on every side that is read take the sparse kernel; the
   // dense kernel then repairs the nodes it could not hold (a.only) and usually finds none.
-  const bool use_sparse = redo && verify_uses_lists(p, t);
+  const bool use_sparse = redo && !a.lazy && verify_uses_lists(p, t);
   if (use_sparse) {
     const int se = V <= sparse::ST * 8 ? 8 : (V <= sparse::ST * 16 ? 16 : 32);
     a.done = redo + static_cast<size_t>(batch) * t->n_nodes;       // the sparse kernel clears it
@@ -205,7 +206,7 @@ extern "C" lantern_status lantern_verify_tree(
     }
   }
   if (e != cudaSuccess) return LANTERN_ERR_CUDA;
-  if (!a.done) {      // otherwise the repair launch has walked the trees
+  if (!a.done && !a.lazy) {      // otherwise the repair launch, or the path walk itself, has walked the trees
     const int seqs = std::max(1, std::min(16, 6144 / t->n_nodes));      // 2 * seqs * N ints <= 48 KB
     if (launch_after_previous(walk_kernel, static_cast<unsigned>((batch + seqs - 1) / seqs), kWalkThreads,
                               sizeof(int32_t) * 2 * seqs * t->n_nodes, st, 1, node_next, node_token, tokens, batch,

@@ -451,16 +451,15 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
 }
 
 
-// One tree node: rows into shared memory, post-processing, sibling loop, resampling.
+// One tree node (sequence b, node n): rows into shared memory, post-processing, sibling loop,
+// resampling.  Returns the accepted child or -1 (the same value in every thread of the row's CTAs).
 template <typename T, bool CFG, int E>
-__device__ __forceinline__ void verify_node(const VerifyArgs& a, const int idx, VCtx& c, const TopkSmem& tk,
+__device__ __forceinline__ int verify_node(const VerifyArgs& a, const int b, const int n, VCtx& c, const TopkSmem& tk,
                                             float* __restrict__ Q, float* __restrict__ P, float* __restrict__ U,
                                             int* misc, const uint32_t mbar_a, uint32_t& mphase, int* nbr_s) {
   constexpr int SL = VT * E;
   constexpr int NV4 = E / 4;                 // float4 per thread in a shared-memory sweep
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b = idx % a.B;
-  const int n = a.order[idx / a.B];
   const int fc = a.first_child[n], nc = a.n_child[n];
   const int lo = c.rank * SL;
   const int len = max(0, min(a.V - lo, SL));
@@ -847,6 +846,7 @@ __device__ __forceinline__ void verify_node(const VerifyArgs& a, const int idx, 
     a.node_token[out_b + n] = -1;
   }
   if (c.rank == 0 && tid == 0) a.node_next[out_b + n] = accepted;
+  return accepted;
 }
 
 // E = row entries per thread; the CTA's slice holds SL = 1024 * E entries.
@@ -897,6 +897,31 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
   // cluster g of G takes the flagged nodes idx = g (mod G) one after another, and leaves at once
   // when none of them is flagged.
   const int rows = a.B * a.N, G = gridDim.x / c.nrank, g0 = blockIdx.x / c.nrank;
+  if (a.lazy) {
+    // Path walk (Sec. 2.1) instead of verifying every node: one cluster per sequence verifies the
+    // root, moves to the accepted child and so on, so only the rows on the accepted path are
+    // read.  The per-node results of the other nodes are not written.
+    const int b = g0;
+    const bool writer = c.rank == 0 && tid == 0;
+    int32_t* ot = a.out_tokens + static_cast<long long>(b) * a.D1;
+    int32_t* on = a.out_nodes + static_cast<long long>(b) * a.D1;
+    int cur = 0, len = 0;
+    for (;;) {
+      const int acc = verify_node<T, CFG, E>(a, b, cur, c, tk, Q, P, U, misc, mbar_a, mphase, nbr_s);
+      csync(c);     // also orders the owner CTA's store of node_token before the read below
+      if (acc <= cur || acc >= a.N || len >= a.D1 - 1) break;      // -1, or anything that is not a forward edge
+      cur = acc;
+      if (writer) { ot[len] = a.tokens[static_cast<long long>(b) * a.N + cur]; on[len] = cur; }
+      ++len;
+    }
+    if (writer) {
+      ot[len] = __ldcg(a.node_token + static_cast<long long>(b) * a.N + cur);
+      on[len] = cur;
+      a.accept_len[b] = len;
+      for (int i = len + 1; i < a.D1; ++i) { ot[i] = -1; on[i] = -1; }
+    }
+    return;
+  }
   bool work = true;
   if (a.only) {
     bool any = false;
@@ -907,7 +932,7 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
   if (work) {
     for (int idx = g0; idx < rows; idx += G) {
       if (a.only && a.only[idx] == 0) continue;
-      verify_node<T, CFG, E>(a, idx, c, tk, Q, P, U, misc, mbar_a, mphase, nbr_s);
+      verify_node<T, CFG, E>(a, idx % a.B, a.order[idx / a.B], c, tk, Q, P, U, misc, mbar_a, mphase, nbr_s);
       csync(c);     // peers may still be reading this CTA's shared memory; the next node overwrites it
     }
   }

@@ -48,6 +48,7 @@ static cudaError_t launch_verify_e(const VerifyArgs& a, const LaunchShape& sh, c
   // one cluster per node; a repair launch (a.only) gets about one cluster per SM and lets each
   // walk its share of the flagged nodes
   unsigned clusters = static_cast<unsigned>(a.B) * a.N;
+  if (a.lazy) clusters = static_cast<unsigned>(a.B);       // path walk: one cluster per sequence
   if (a.only) {
     const unsigned per_wave = static_cast<unsigned>(sm_count() / sh.cs > 0 ? sm_count() / sh.cs : 1);
     if (clusters > per_wave) clusters = per_wave;

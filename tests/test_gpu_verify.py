@@ -161,6 +161,46 @@ def test_additive_bound_variant(L, delta, kw):
         assert all(np.all(o["cut_margin"][np.isfinite(o["cut_margin"])] > 0.5) for o in orc)
 
 
+@pytest.mark.parametrize("cs", [0, 1, 4])
+@pytest.mark.parametrize("kw", [dict(batch=5, n_nodes=60), dict(top_k=80, dtype="bf16", cfg_scale=None, batch=3),
+                                dict(draft_noise=0.05, batch=4)])
+def test_path_walk_gives_the_results_of_verifying_every_node(L, cs, kw):
+    """lazy_walk = 1 (Sec. 2.1 read as a walk from the root): same accepted path and emitted tokens
+    as the launch over all nodes, and the per-node results on the path agree with the oracle."""
+    case = Case(small_config(**kw), seed=20)
+    g, par, nbr, tok = case.gpu_inputs(L)
+    tree = L.Tree(case.parent)
+    ua, ur = case.u_accept.cuda(), case.u_resample.cuda()
+    old = L.set_cluster_size(cs)
+    try:
+        eager = L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"],
+                              g["draft_uncond"], tok, ua, ur, debug=True)
+        par.lazy_walk = 1
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = {k: torch.full_like(v, -5) for k, v in eager.items()}
+        lazy = L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"],
+                             g["draft_uncond"], tok, ua, ur, debug=True, out=out, device_status=status)
+        torch.cuda.synchronize()
+    finally:
+        L.set_cluster_size(old)
+    assert int(status.item()) == 0
+    for k in ("accept_len", "out_tokens", "out_nodes"):
+        assert torch.equal(lazy[k], eager[k]), k
+    orc = case.oracle_verify()
+    for b in range(case.B):
+        path = [0] + [int(n) for n in lazy["out_nodes"][b, : int(lazy["accept_len"][b])].cpu()]
+        for n in path:               # nodes on the path carry the same per-node results
+            assert int(lazy["node_next"][b, n]) == int(eager["node_next"][b, n])
+            assert int(lazy["node_token"][b, n]) == int(eager["node_token"][b, n])
+        assert int(lazy["accept_len"][b]) == orc[b]["accept_len"] or b in _dirty(case, eager, orc)
+    assert int(lazy["accept_len"].max()) >= 1 or kw.get("draft_noise") is None
+
+
+def _dirty(case, eager, orc):
+    res = {k: v.cpu().numpy() for k, v in eager.items()}
+    return compare_verify(res, orc, case.parent, case.u_accept.numpy(), case.seqs)["dirty_sequences"]
+
+
 def test_allowed_range_and_topk_counts_only_allowed(L):
     case = Case(small_config(vocab=2048, codebook_size=512, code_offset=256, k=6, top_k=40), seed=3,
                 allowed=(256, 768))
