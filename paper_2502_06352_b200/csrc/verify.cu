@@ -177,7 +177,9 @@ extern "C" lantern_status lantern_verify_tree(
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = target_uncond != nullptr;
   const bool f32 = dt == LANTERN_F32;
-  const int min_e = f32 ? 4 : 8, rows = a.lazy ? batch : batch * t->n_nodes;
+  const int min_e = f32 ? 4 : 8;
+  // (the path walk is a chain of nodes per sequence: rows are not split over more CTAs than they need)
+  const int rows = a.lazy ? (1 << 20) : batch * t->n_nodes;
   cudaError_t e;
   // Rows truncated to a moderate top-k on every side that is read take the sparse kernel; the
   // dense kernel then repairs the nodes it could not hold (a.only) and usually finds none.
