@@ -75,14 +75,36 @@ __device__ __forceinline__ double exact_dist(const T* __restrict__ cb, int d, in
   return s;
 }
 
+// The same sum, in the same order, for a bfloat16 query row held in shared memory and a candidate
+// row read from global memory with 16-byte loads (d a multiple of 8, both rows 16-byte aligned).
+__device__ __forceinline__ double exact_dist_bf16x8(const __nv_bfloat16* a, const __nv_bfloat16* __restrict__ b, int d) {
+  double s = 0.0;
+  for (int t = 0; t < d; t += 8) {
+    const uint4 av = *reinterpret_cast<const uint4*>(a + t);
+    const uint4 bv = __ldg(reinterpret_cast<const uint4*>(b + t));
+    const uint32_t aw[4] = {av.x, av.y, av.z, av.w}, bw[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const double d0 = static_cast<double>(__uint_as_float(aw[i] << 16)) - static_cast<double>(__uint_as_float(bw[i] << 16));
+      s = fma(d0, d0, s);
+      const double d1 = static_cast<double>(__uint_as_float(aw[i] & 0xffff0000u)) -
+                        static_cast<double>(__uint_as_float(bw[i] & 0xffff0000u));
+      s = fma(d1, d1, s);
+    }
+  }
+  return s;
+}
+
 // Exact ranking of one query's surviving candidates (keys carry the candidate index in their
 // low 32 bits): distances re-evaluated in double, sorted by (distance, index), first k written.
 // With `overflow` the buffer is ignored and k rounds of an exact arg-min over all rows are run.
+// `q_row`, if given, is the query's bfloat16 row in shared memory (d a multiple of 8): the distances
+// then come from exact_dist_bf16x8.
 template <typename T>
 __device__ __forceinline__ void rank_query(const T* __restrict__ cb, int L, int d, int k, int qi,
                                            const unsigned long long* bq, int n_in, bool overflow, int CAP,
                                            double* sortd, int* sorti, double* redd, int* redi,
-                                           int32_t* out_i, float* out_d) {
+                                           int32_t* out_i, float* out_d, const __nv_bfloat16* q_row = nullptr) {
   const int tid = threadIdx.x;
     if (!overflow) {
     const int n = min(n_in, CAP);
@@ -90,7 +112,10 @@ __device__ __forceinline__ void rank_query(const T* __restrict__ cb, int L, int 
       if (i < n) {
         int j = static_cast<int>(bq[i] & 0xffffffffu);
         sorti[i] = j;
-        sortd[i] = exact_dist<T>(cb, d, qi, j);
+        if (sizeof(T) == 2 && q_row)
+          sortd[i] = exact_dist_bf16x8(q_row, reinterpret_cast<const __nv_bfloat16*>(cb) + static_cast<long long>(j) * d, d);
+        else
+          sortd[i] = exact_dist<T>(cb, d, qi, j);
       } else {
         sorti[i] = 0x7fffffff;
         sortd[i] = INFINITY;

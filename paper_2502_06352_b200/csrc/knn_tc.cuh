@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(kKnnThreads) knn_tc_kernel(const KnnTcArgs a) 
     if (qi >= L) break;
     rank_query<__nv_bfloat16>(cb, L, d, k, qi, buf + static_cast<size_t>(q) * CAP, cnt[q], ovf[q] != 0, CAP, sortd, sorti,
                               redd, redi, a.nbr_idx + static_cast<long long>(qi) * k,
-                              a.nbr_dist ? a.nbr_dist + static_cast<long long>(qi) * k : nullptr);
+                              a.nbr_dist ? a.nbr_dist + static_cast<long long>(qi) * k : nullptr, As + q * ld);
   }
 }
 
