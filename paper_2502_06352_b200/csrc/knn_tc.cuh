@@ -60,12 +60,27 @@ __device__ __forceinline__ void stage_rows(const __nv_bfloat16* __restrict__ cb,
                                            __nv_bfloat16* dst) {
   const int chunks = d / 8;                   // 16-byte chunks per row
   const int ld = d + kTcPad;
-  for (int i = threadIdx.x; i < rows * chunks; i += kKnnThreads) {
-    const int r = i / chunks, ch = i - r * chunks;
+  // thread i starts at chunk i and advances by the thread count: (row, chunk) follow by addition
+  int r = static_cast<int>(threadIdx.x) / chunks, ch = static_cast<int>(threadIdx.x) - r * chunks;
+  const int dr = kKnnThreads / chunks, dch = kKnnThreads - dr * chunks;
+  while (r < rows) {
     const int row = row0 + r;
     const bool in = row < L;
     const __nv_bfloat16* src = cb + static_cast<long long>(in ? row : 0) * d + ch * 8;
     cp_async16(smem_u32(dst + r * ld + ch * 8), src, in ? 16u : 0u);
+    r += dr;
+    ch += dch;
+    if (ch >= chunks) { ch -= chunks; ++r; }
+  }
+}
+
+// squared norms of the candidate rows [row0, row0 + kTcCT) into shared memory (zero beyond L)
+__device__ __forceinline__ void stage_norms(const float* __restrict__ nrm, int L, int row0, float* dst) {
+  if (threadIdx.x < kTcCT) {
+    const int j = row0 + threadIdx.x;
+    const bool in = j < L;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst + threadIdx.x)),
+                 "l"(nrm + (in ? j : 0)), "r"(in ? 4u : 0u) : "memory");
   }
 }
 
@@ -96,8 +111,8 @@ __global__ void __launch_bounds__(kKnnThreads) knn_tc_kernel(const KnnTcArgs a) 
 
   stage_rows(cb, L, d, q0, kTcQT, As);
   stage_rows(cb, L, d, 0, kTcCT, Bs);
+  stage_norms(a.nrm, L, 0, ncs);
   cp_async_commit();
-  if (tid < kTcCT) ncs[tid] = tid < L ? a.nrm[tid] : 0.f;
   if (tid < kTcQT) {
     const float n = q0 + tid < L ? a.nrm[q0 + tid] : 0.f;
     nq[tid] = n;
@@ -115,11 +130,8 @@ __global__ void __launch_bounds__(kKnnThreads) knn_tc_kernel(const KnnTcArgs a) 
     const int cur = t & 1;
     if (t + 1 < ntiles) {
       stage_rows(cb, L, d, (t + 1) * kTcCT, kTcCT, Bs + (cur ^ 1) * kTcCT * ld);
+      stage_norms(a.nrm, L, (t + 1) * kTcCT, ncs + (cur ^ 1) * kTcCT);
       cp_async_commit();
-      if (tid < kTcCT) {
-        const int j = (t + 1) * kTcCT + tid;
-        ncs[(cur ^ 1) * kTcCT + tid] = j < L ? a.nrm[j] : 0.f;
-      }
       cp_async_wait<1>();
     } else {
       cp_async_wait<0>();
@@ -159,8 +171,10 @@ __global__ void __launch_bounds__(kKnnThreads) knn_tc_kernel(const KnnTcArgs a) 
         }
       }
     }
-    __syncthreads();
-    // cut back buffers that might overflow during the next tile
+    __syncthreads();                                   // this tile's appends are counted
+    // cut back buffers that might overflow during the next tile (usually none: one vote)
+    const bool near_full = tid < kTcQT && cnt[tid] > CAP - kTcCT && !ovf[tid];
+    if (!__syncthreads_or(near_full)) continue;
     for (int q = 0; q < kTcQT; ++q) {
       const int n = cnt[q];
       if (n <= CAP - kTcCT || ovf[q]) continue;            // uniform: shared values
