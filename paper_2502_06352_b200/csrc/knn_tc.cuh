@@ -55,6 +55,12 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// four 8 x 8 bf16 matrices from shared memory: lane l supplies the address of row l % 8 of matrix l / 8
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const __nv_bfloat16* row_ptr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(row_ptr)) : "memory");
+}
+
 // stage rows [row0, row0 + rows) of the codebook into padded shared-memory rows (zero beyond L)
 __device__ __forceinline__ void stage_rows(const __nv_bfloat16* __restrict__ cb, int L, int d, int row0, int rows,
                                            __nv_bfloat16* dst) {
@@ -139,19 +145,17 @@ __global__ void __launch_bounds__(kKnnThreads) knn_tc_kernel(const KnnTcArgs a) 
     __syncthreads();
     const __nv_bfloat16* Bt = Bs + cur * kTcCT * ld;
     float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    // fragments by ldmatrix: A = query rows (matrices: rows 0-7 / 8-15 x k 0-7 / 8-15), B = candidate
+    // rows of two 8-wide column tiles (matrices: tile 0 k 0-7, tile 0 k 8-15, tile 1 k 0-7, tile 1 k 8-15)
+    const int mi = lane >> 3, mr = lane & 7;
+    const __nv_bfloat16* a_ptr = As + (wq * 16 + (mi & 1) * 8 + mr) * ld + (mi >> 1) * 8;
+    const __nv_bfloat16* b_ptr = Bt + (wc * 16 + (mi >> 1) * 8 + mr) * ld + (mi & 1) * 8;
     for (int kb = 0; kb < d; kb += 16) {
-      uint32_t af[4];
-      af[0] = *reinterpret_cast<const uint32_t*>(As + r0 * ld + kb + kc);
-      af[1] = *reinterpret_cast<const uint32_t*>(As + r1 * ld + kb + kc);
-      af[2] = *reinterpret_cast<const uint32_t*>(As + r0 * ld + kb + kc + 8);
-      af[3] = *reinterpret_cast<const uint32_t*>(As + r1 * ld + kb + kc + 8);
-#pragma unroll
-      for (int nt = 0; nt < 2; ++nt) {
-        const __nv_bfloat16* bp = Bt + (wc * 16 + nt * 8 + (lane >> 2)) * ld + kb + kc;
-        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(bp);
-        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(bp + 8);
-        mma_bf16_16816(acc[nt], af, b0, b1);
-      }
+      uint32_t af[4], bf[4];
+      ldmatrix_x4(af, a_ptr + kb);
+      ldmatrix_x4(bf, b_ptr + kb);
+      mma_bf16_16816(acc[0], af, bf[0], bf[1]);
+      mma_bf16_16816(acc[1], af, bf[2], bf[3]);
     }
     // epilogue: approximate distances, filter, append
     const float thr0 = thr[r0], thr1 = thr[r1], nq0 = nq[r0], nq1 = nq[r1];
