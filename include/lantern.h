@@ -188,6 +188,7 @@ lantern_status lantern_verify_tree(const lantern_params* params, const lantern_t
  * (dense + walk, or lists + repair launch that also walks).  Returns -1 on NULL arguments.       */
 #define LANTERN_PATH_DENSE 0
 #define LANTERN_PATH_LISTS 1
+#define LANTERN_PATH_STREAM 2
 int32_t lantern_verify_tree_path(const lantern_params* params, const lantern_tree* tree);
 int32_t lantern_sample_draft_tree_path(const lantern_params* params);
 

@@ -269,7 +269,8 @@ def philox_raw(seed, first, c1, c2, c3, n, device="cuda"):
 
 
 def verify_tree_path(params: "Params", tree: "Tree") -> int:
-    """lantern_verify_tree_path: 0 = dense kernels, 1 = list-based kernels + repair launch."""
+    """lantern_verify_tree_path: 0 = dense kernels, 1 = list-based kernels + repair launch,
+    2 = streaming kernel (rows without top-k)."""
     cp = params.c()
     return lib.lantern_verify_tree_path(ctypes.byref(cp), tree.handle)
 

@@ -163,7 +163,7 @@ struct VerifyArgs {
   const int32_t* nbr;
   int k_table, use_bulk;
   const int32_t *first_child, *n_child, *order;
-  int B, N, V, kpad, n_internal;
+  int B, N, V, kpad, n_internal, max_children;
   float g, inv_tau, lambda, delta;
   int topk_t, topk_d, k, code_offset, n_codes, allow_lo, allow_hi;
   unsigned long long seed, step;

@@ -34,6 +34,7 @@ static int sm_count() {
 #undef LANTERN_VT
 #undef LANTERN_VNS
 #include "verify_sparse.cuh"
+#include "verify_stream.cuh"
 
 namespace lantern {
 
@@ -61,6 +62,38 @@ static cudaError_t launch_sparse_any(const VerifyArgs& a, int32_t* redo, int e, 
              : launch_sparse<__nv_bfloat16, false>(a, redo, e, smem, st);
 }
 
+// ---- launch of the streaming kernel (rows without top-k): one CTA, or a cluster of cs CTAs, per node
+template <typename T, bool CFG, bool TAU1>
+static cudaError_t launch_stream_t(const VerifyArgs& a, int cs, size_t smem, cudaStream_t st) {
+  auto kern = stream::verify_stream_kernel<T, CFG, TAU1>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  if (cs > 8) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+  }
+  return launch_after_previous(kern, static_cast<unsigned>(a.B) * a.N * cs, stream::ST, smem, st, cs, a);
+}
+static cudaError_t launch_stream_any(const VerifyArgs& a, int cs, size_t smem, bool f32, bool cfg, cudaStream_t st) {
+  const bool tau1 = a.inv_tau == 1.0f;
+  if (f32) {
+    if (cfg) return launch_stream_t<float, true, false>(a, cs, smem, st);
+    return tau1 ? launch_stream_t<float, false, true>(a, cs, smem, st) : launch_stream_t<float, false, false>(a, cs, smem, st);
+  }
+  if (cfg) return launch_stream_t<__nv_bfloat16, true, false>(a, cs, smem, st);
+  return tau1 ? launch_stream_t<__nv_bfloat16, false, true>(a, cs, smem, st)
+              : launch_stream_t<__nv_bfloat16, false, false>(a, cs, smem, st);
+}
+// CTAs per node: one when the nodes alone fill the machine, else the smallest power of two that
+// does, as long as every warp keeps at least one full 512-byte step of the row
+static int stream_cluster_size(int nodes, int V, bool f32) {
+  if (g_cluster_override > 0) return g_cluster_override;
+  const int nvec = V / (f32 ? 4 : 8);
+  int cs = 1;
+  while (cs < 16 && static_cast<long long>(nodes) * cs < 4 * sm_count() && nvec / (2 * cs * stream::SW) >= 32) cs *= 2;
+  return cs;
+}
+
 // ---- walk (Sec. 2.1) as a launch of its own: a CTA stages the per-node results of `seqs`
 // sequences in shared memory (at most 48 KB) and walks them
 constexpr int kWalkThreads = 128;
@@ -75,6 +108,18 @@ __global__ void __launch_bounds__(kWalkThreads) walk_kernel(const int32_t* __res
   const int b0 = blockIdx.x * seqs;
   walk_staged(node_next, node_token, tokens, b0, min(seqs, B - b0), N, D1, accept_len, out_tokens, out_nodes,
               walk_stage);
+}
+
+
+static lantern_status launch_walk(const TreeDev* t, int batch, const int32_t* node_next, const int32_t* node_token,
+                                  const int32_t* tokens, int32_t* accept_len, int32_t* out_tokens, int32_t* out_nodes,
+                                  int D1, cudaStream_t st) {
+  const int seqs = std::max(1, std::min(16, 6144 / t->n_nodes));      // 2 * seqs * N ints <= 48 KB
+  if (launch_after_previous(walk_kernel, static_cast<unsigned>((batch + seqs - 1) / seqs), kWalkThreads,
+                            sizeof(int32_t) * 2 * seqs * t->n_nodes, st, 1, node_next, node_token, tokens, batch,
+                            t->n_nodes, D1, seqs, accept_len, out_tokens, out_nodes) != cudaSuccess)
+    return LANTERN_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
 }
 
 }  // namespace lantern
@@ -98,11 +143,22 @@ bool verify_uses_lists(const lantern_params* p, const TreeDev* t) {
   return !p->lazy_walk && g_cluster_override == 0 && V <= sparse::kMaxV && topk_fits(p->top_k_target) &&
          (t->n_internal == 0 || topk_fits(p->top_k_draft)) && t->max_children <= 8;
 }
+// Rows that no top-k truncates take the streaming kernel (unless the path walk is asked for).
+bool verify_uses_stream(const lantern_params* p, const TreeDev* t) {
+  const int V = p->vocab;
+  const bool tk_t = p->top_k_target > 0 && p->top_k_target < V;
+  const bool tk_d = t->n_internal > 0 && p->top_k_draft > 0 && p->top_k_draft < V;
+  const bool cfg4 = true;      // the larger layout decides
+  return !p->lazy_walk && !tk_t && !tk_d && V <= stream::kMaxV &&
+         stream::smem_bytes(V, t->max_children, p->k + 1, cfg4) <= 227 * 1024;
+}
 }  // namespace
 
 extern "C" int32_t lantern_verify_tree_path(const lantern_params* p, const lantern_tree* tree) {
   if (!p || !tree) return -1;
-  return verify_uses_lists(p, reinterpret_cast<const TreeDev*>(tree)) ? LANTERN_PATH_LISTS : LANTERN_PATH_DENSE;
+  const TreeDev* t = reinterpret_cast<const TreeDev*>(tree);
+  if (verify_uses_stream(p, t)) return LANTERN_PATH_STREAM;
+  return verify_uses_lists(p, t) ? LANTERN_PATH_LISTS : LANTERN_PATH_DENSE;
 }
 
 extern "C" size_t lantern_verify_tree_workspace(const lantern_tree* tree, int32_t batch) {
@@ -161,7 +217,7 @@ extern "C" lantern_status lantern_verify_tree(
   a.nbr = nbr_idx; a.k_table = k_table;
   a.use_bulk = (p->k > 0 && k_table % 4 == 0 && reinterpret_cast<uintptr_t>(nbr_idx) % 16 == 0) ? 1 : 0;
   a.first_child = t->d_first_child; a.n_child = t->d_n_child; a.order = t->d_order;
-  a.B = batch; a.N = t->n_nodes; a.V = V; a.n_internal = t->n_internal;
+  a.B = batch; a.N = t->n_nodes; a.V = V; a.n_internal = t->n_internal; a.max_children = t->max_children;
   a.kpad = (p->k + 3) & ~3;
   a.g = p->cfg_scale; a.inv_tau = 1.0f / p->temperature; a.lambda = p->lambda; a.delta = p->delta;
   a.topk_t = p->top_k_target; a.topk_d = p->top_k_draft; a.k = p->k;
@@ -191,6 +247,12 @@ extern "C" lantern_status lantern_verify_tree(
     if (e != cudaSuccess) return LANTERN_ERR_CUDA;
     a.only = redo;
   }
+  if (!use_sparse && verify_uses_stream(p, t)) {
+    const int cs = stream_cluster_size(batch * t->n_nodes, allow_hi - allow_lo, f32);
+    e = launch_stream_any(a, cs, stream::smem_bytes(V, t->max_children, p->k + 1, cfg), f32, cfg, st);
+    if (e != cudaSuccess) return LANTERN_ERR_CUDA;
+    return launch_walk(t, batch, node_next, node_token, tokens, accept_len, out_tokens, out_nodes, D1, st);
+  }
   // rows that fit one CTA run the 1024-thread build; rows split over a cluster run the
   // 512-thread build (cheaper barriers, half the per-thread fixed work per entry)
   v1024::LaunchShape s1;
@@ -208,14 +270,8 @@ extern "C" lantern_status lantern_verify_tree(
     }
   }
   if (e != cudaSuccess) return LANTERN_ERR_CUDA;
-  if (!a.done && !a.lazy) {      // otherwise the repair launch, or the path walk itself, has walked the trees
-    const int seqs = std::max(1, std::min(16, 6144 / t->n_nodes));      // 2 * seqs * N ints <= 48 KB
-    if (launch_after_previous(walk_kernel, static_cast<unsigned>((batch + seqs - 1) / seqs), kWalkThreads,
-                              sizeof(int32_t) * 2 * seqs * t->n_nodes, st, 1, node_next, node_token, tokens, batch,
-                              t->n_nodes, D1, seqs, accept_len, out_tokens, out_nodes) != cudaSuccess)
-      return LANTERN_ERR_CUDA;
-    if (cudaGetLastError() != cudaSuccess) return LANTERN_ERR_CUDA;
-  }
+  if (!a.done && !a.lazy)        // otherwise the repair launch, or the path walk itself, has walked the trees
+    return launch_walk(t, batch, node_next, node_token, tokens, accept_len, out_tokens, out_nodes, D1, st);
   return LANTERN_OK;
 }
 
