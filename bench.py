@@ -1,16 +1,20 @@
 """Benchmark of the relaxed tree-verification hot path.
 
 One step = one pass of the path over one batch of synthetic input: the draft sampler over
-every internal node, the relaxed verification of every node and the walk (three kernel
-launches).  The neighbour table is built once per codebook and is timed separately.
+every internal node, then the relaxed verification of every node and the walk.  The
+neighbour table is built once per codebook and is timed separately.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
-Prints one JSON line (rank 0).  Under torchrun every rank verifies its own batch of
-sequences (no data-path collective); the value is all ranks' nodes over the slowest rank's
-device time.
+Prints one JSON line (rank 0).  The headline numbers (value, roofline, e2e, cpu_baseline) are
+those of --workload (default: the largest single-GPU configuration, c4_batch64); the `configs`
+object of the same line carries the verify / sampler timings and roofline fractions of every
+other configuration (c1..c3, c3 restricted to its image tokens, and the neighbour-table sweep).
+Under torchrun every rank verifies its own batch of sequences (no data-path collective); the
+value is all ranks' nodes over the slowest rank's device time.
 """
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -23,17 +27,21 @@ sys.path.insert(0, ROOT)
 METRIC = "verified tree nodes/sec"
 UNIT = "nodes/s"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+MIN_TIMED_MS = 50.0
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="c2_llamagen512")
+    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c4_batch64")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--ring", type=int, default=0, help="input buffer sets cycled through (0 = enough to exceed L2)")
-    ap.add_argument("--e2e-steps", type=int, default=100)
+    ap.add_argument("--e2e-steps", type=int, default=8)
+    ap.add_argument("--configs", default="all", choices=["all", "none"],
+                    help="all: also time the other configurations and report them under `configs`")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of CUDA-graph replays")
     ap.add_argument("--walk", default="eager", choices=["eager", "lazy"],
@@ -42,29 +50,32 @@ def parse_args():
     return ap.parse_args()
 
 
-def algorithmic_bytes(cfg, parent, batch):
-    """Bytes one verify launch must move: every target row and every internal node's drafter
-    row once, the neighbour rows of the draft tokens, and the per-node outputs."""
+def algorithmic_bytes(cfg, parent, batch, allowed=None):
+    """(verify bytes, sampler bytes) one call must move: every target row and every internal
+    node's drafter row once (only the allowed slice of a row when the tokens are restricted),
+    the neighbour rows of the draft tokens, and the per-node inputs / outputs."""
     N = len(parent)
     I = len(set(parent[1:]))
     c = 2 if cfg.cfg_scale is not None else 1
     e = 4 if cfg.dtype == "f32" else 2
-    rows = batch * (N + I) * c * cfg.vocab * e
+    width = cfg.vocab if allowed is None else allowed[1] - allowed[0]
+    rows = batch * (N + I) * c * width * e
     table = batch * (N - 1) * cfg.k * 4
     outs = batch * N * (4 + 4 + 4 + 4 + 4)      # tokens, two uniforms in; next, token out
-    return rows + table + outs, batch * I * c * cfg.vocab * e
+    return rows + table + outs, batch * I * c * width * e
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (mean of the two
-# captured launches), from the ncu capture summarised under profiles/; valid only for the kernel
-# source it was taken from
-TRAFFIC = {"c2_llamagen512": {"kernel_sha256": "d16142fbf6a4b272", "bytes": 105080000}}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (taken on a smaller batch and scaled by the number of rows,
+# as stated there); valid only for the kernel source it was taken from
+TRAFFIC = {}
 
 
 def kernel_sha256():
     import hashlib
     h = hashlib.sha256()
-    for f in ("verify_sparse.cuh", "verify_kernel.cuh", "verify_launch.cuh", "verify.cu", "rowops.cuh", "common.cuh"):
+    for f in ("verify_stream.cuh", "verify_sparse.cuh", "verify_kernel.cuh", "verify_launch.cuh", "verify.cu",
+              "rowops.cuh", "common.cuh"):
         with open(os.path.join(ROOT, "paper_2502_06352_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -131,18 +142,20 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def oracle_step_inputs(cfg, parent, logits_cpu, seqs, seed):
+# ------------------------------------------------------------------------------------------------
+# CPU oracle baseline (the reference arm and the cpu_baseline leg)
+
+def oracle_step_inputs(cfg, parent, n_seqs, seed):
     import workloads as W
     N, V = len(parent), cfg.vocab
-    gum = W.make_gumbel_uniforms(len(seqs), N, V, seed).numpy()
-    ua, ur = W.make_uniforms(len(seqs), N, seed + 1)
+    gum = W.make_gumbel_uniforms(n_seqs, N, V, seed).numpy()
+    ua, ur = W.make_uniforms(n_seqs, N, seed + 1)
     nbr = W.random_neighbor_table(cfg.codebook_size, cfg.k, seed + 2).numpy()
     return gum, ua.numpy(), ur.numpy(), nbr
 
 
 def oracle_run_nodes(cfg, parent, lg, b, gum, ua, ur, nbr, n_nodes):
     """Oracle sampler + verifier on the first n_nodes nodes of sequence b (bounded sample)."""
-    import numpy as np
     import oracle
     f = lambda t: None if t is None else t[b].float().numpy()
     kw = dict(cfg_scale=cfg.cfg_scale if cfg.cfg_scale is not None else 1.0, temperature=cfg.temperature)
@@ -161,24 +174,47 @@ def oracle_run_nodes(cfg, parent, lg, b, gum, ua, ur, nbr, n_nodes):
     return done
 
 
-def cpu_baseline(cfg, parent, lg_cpu, budget_s=12.0):
-    """The oracle, as it stands, on whole sequences of the workload until about budget_s."""
-    N = len(parent)
-    B = lg_cpu["target_cond"].shape[0]
-    gum, ua, ur, nbr = oracle_step_inputs(cfg, parent, lg_cpu, list(range(B)), 4242)
+def _oracle_worker(job):
+    """One process of the all-cores baseline: whole sequences of the workload (its own seeded
+    inputs) until the time budget is spent.  Returns (nodes, seconds)."""
+    name, worker, budget_s = job
+    import torch
+    torch.set_num_threads(1)
+    import workloads as W
+    cfg = W.CONFIGS[name]
+    parent = W.static_tree(cfg.n_nodes)
+    lg = W.make_logits(cfg, step=7000 + worker, device="cpu", batch=1)
+    gum, ua, ur, nbr = oracle_step_inputs(cfg, parent, 1, 4242 + worker)
     t0 = time.perf_counter()
     nodes = 0
-    seqs = 0
     while True:
-        b = seqs % B
-        nodes += oracle_run_nodes(cfg, parent, lg_cpu, b, gum[b], ua[b], ur[b], nbr, N)
-        seqs += 1
-        if time.perf_counter() - t0 > budget_s or seqs >= 256 * B:
+        nodes += oracle_run_nodes(cfg, parent, lg, 0, gum[0], ua[0], ur[0], nbr, len(parent))
+        if time.perf_counter() - t0 > budget_s:
             break
-    dt = time.perf_counter() - t0
-    return {"value": nodes / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": "%d whole sequences (%d nodes: draft sampling + relaxed verification of every node) of %s, %.1f s"
-                      % (seqs, nodes, cfg.name, dt)}
+    return nodes, time.perf_counter() - t0
+
+
+def cpu_baseline(cfg, parent, budget_s=10.0):
+    """The oracle, as it stands, on whole sequences of the workload: one process for about
+    budget_s, then one process per host core for about budget_s (each on its own sequence)."""
+    import multiprocessing as mp
+    n1, t1 = _oracle_worker((cfg.name, 0, budget_s))
+    cores = os.cpu_count() or 1
+    value_all, used = None, 1
+    if cores > 1:
+        try:
+            ctx = mp.get_context("spawn")
+            with ctx.Pool(cores) as pool:
+                res = pool.map(_oracle_worker, [(cfg.name, w, budget_s) for w in range(cores)])
+            value_all = sum(n / t for n, t in res)
+            used = cores
+        except Exception as exc:          # no process pool on this host: the one-core figure stands
+            sys.stderr.write("all-cores oracle baseline not run: %r\n" % (exc,))
+    value = value_all if value_all is not None else n1 / t1
+    return {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "value_one_core": n1 / t1,
+            "sample": "whole sequences of %s (draft sampling + relaxed verification of every node), about %.0f s "
+                      "per process; one process: %d nodes in %.1f s; %d processes, one sequence each, run "
+                      "together" % (cfg.name, budget_s, n1, t1, used)}
 
 
 def run_reference(args, cfg, parent):
@@ -189,7 +225,7 @@ def run_reference(args, cfg, parent):
         return
     N = len(parent)
     lg = W.make_logits(cfg, step=0, device="cpu", batch=1)
-    gum, ua, ur, nbr = oracle_step_inputs(cfg, parent, lg, [0], 4242)
+    gum, ua, ur, nbr = oracle_step_inputs(cfg, parent, 1, 4242)
     t0 = time.perf_counter()
     oracle_run_nodes(cfg, parent, lg, 0, gum[0], ua[0], ur[0], nbr, 4)
     t_node = (time.perf_counter() - t0) / 4
@@ -213,23 +249,24 @@ def run_reference(args, cfg, parent):
         "gpu_launches": 0}))
 
 
-def run_table_sweep(args):
-    """--workload c5_table_sweep: every (L, d, k) neighbour-table build of the sweep, timed with
-    CUDA events (best of 3 after a warm-up), plus the oracle timed on a few rows of each shape."""
-    import numpy as np
+# ------------------------------------------------------------------------------------------------
+# neighbour-table sweep (config 5)
+
+def table_sweep(with_oracle):
+    """Every (L, d, k) neighbour-table build of the sweep, timed with CUDA events (best of 3 after
+    a warm-up); with_oracle also times the oracle on a few rows of each shape."""
     import torch
     import workloads as W
     from workloads.configs import SWEEP_L, SWEEP_D, SWEEP_K, SWEEP_DUP_FRAC
     import paper_2502_06352_b200 as L
-    import oracle
-    torch.cuda.set_device(0)
     rows = []
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for n in SWEEP_L:
         for d in SWEEP_D:
             cb = W.make_codebook(n, d, "bf16", seed=5, dup_frac=SWEEP_DUP_FRAC, device="cuda")
             t_or = None
-            if not args.no_cpu_baseline:
+            if with_oracle:
+                import oracle
                 cb64 = cb.cpu().to(torch.float64).numpy()
                 t0 = time.perf_counter()
                 oracle.neighbor_table(cb64, max(SWEEP_K), rows=list(range(0, n, max(1, n // 8)))[:8])
@@ -247,15 +284,207 @@ def run_table_sweep(args):
                 alg = n * d * 2 + n * k * 4
                 rows.append({"L": n, "d": d, "k": k, "ms": round(best, 3), "rows_per_s": n / (best * 1e-3),
                              "gbs": alg / (best * 1e-3) / 1e9, "contraction_tflops": 2.0 * n * n * d / (best * 1e-3) / 1e12,
+                             "candidates_per_s": float(n) * n / (best * 1e-3),
                              "path": "tensor" if (d % 16 == 0 and 32 <= d <= 256 and k <= 320) else "brute",
                              "oracle_rows_per_s": None if t_or is None else 1.0 / t_or})
+    return rows, SWEEP_DUP_FRAC
+
+
+def run_table_sweep(args):
+    """--workload c5_table_sweep: the sweep as the headline of its own JSON line."""
+    import torch
+    torch.cuda.set_device(0)
+    rows, dup = table_sweep(not args.no_cpu_baseline)
     total_rows = sum(r["L"] for r in rows)
     total_ms = sum(r["ms"] for r in rows)
     print(json.dumps({"metric": "neighbour-table rows/sec", "value": total_rows / (total_ms * 1e-3), "unit": "rows/s",
                       "n_gpus": 1, "steps": 3, "warmup": 1, "ms_per_step": total_ms, "higher_is_better": True,
                       "scaling": "weak", "vs_baseline": None, "dtype": "bf16 mma + f64 re-rank", "data": "synthetic",
-                      "config": {"workload": "c5_table_sweep", "dup_frac": SWEEP_DUP_FRAC}, "builds": rows,
+                      "config": {"workload": "c5_table_sweep", "dup_frac": dup}, "builds": rows,
                       "gpu_launches": 4 * 2 * len(rows)}))
+
+
+# ------------------------------------------------------------------------------------------------
+# one configuration on the device
+
+class Workload:
+    """Inputs of one configuration resident on the device: a ring of step buffers larger than
+    L2, the neighbour table, parameters and output buffers; step / verify / sampler calls."""
+
+    def __init__(self, L, W, cfg, dev, rank=0, ring=0, allowed=None, walk="eager", build_table=True, max_ring_bytes=40e9):
+        import torch
+        self.L, self.cfg, self.dev, self.allowed = L, cfg, dev, allowed
+        self.parent = W.static_tree(cfg.n_nodes)
+        self.N, self.B, self.V = len(self.parent), cfg.batch, cfg.vocab
+        self.tree = L.Tree(self.parent)
+        n_ops = 4 if cfg.cfg_scale is not None else 2
+        self.set_bytes = n_ops * self.B * self.N * self.V * (4 if cfg.dtype == "f32" else 2)
+        r = ring if ring > 0 else max(2, -(-3 * 126 * 2 ** 20 // self.set_bytes))
+        self.ring = min(r, max(2, int(max_ring_bytes // self.set_bytes)))
+        self.table_ms = None
+        if build_table:
+            codebook = W.make_codebook(cfg.codebook_size, cfg.codebook_dim, cfg.codebook_dtype, seed=cfg.index, device=dev)
+            self.nbr = L.build_neighbors(codebook, cfg.k)
+            torch.cuda.synchronize()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            tb = []
+            for _ in range(3):
+                ev0.record()
+                self.nbr = L.build_neighbors(codebook, cfg.k)
+                ev1.record()
+                torch.cuda.synchronize()
+                tb.append(ev0.elapsed_time(ev1))
+            self.table_ms = min(tb)
+        else:
+            self.nbr = W.random_neighbor_table(cfg.codebook_size, cfg.k, 7, device=dev)
+        self.bufs = [W.make_logits(cfg, step=1000 * rank + s, device=dev) for s in range(self.ring)]
+        self.params = L.Params(vocab=self.V, cfg_scale=cfg.cfg_scale if cfg.cfg_scale is not None else 1.0,
+                               temperature=cfg.temperature, top_k_target=cfg.top_k, top_k_draft=cfg.top_k, lam=cfg.lam,
+                               k=cfg.k, code_offset=cfg.code_offset, n_codes=cfg.codebook_size, seed=0x1A27E2 + rank,
+                               allowed_begin=0 if allowed is None else allowed[0],
+                               allowed_end=0 if allowed is None else allowed[1], lazy_walk=1 if walk == "lazy" else 0)
+        self.tokens = [torch.zeros((self.B, self.N), dtype=torch.int32, device=dev) for _ in range(self.ring)]
+        self.out = {}
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        need = L.lib.lantern_verify_tree_workspace(self.tree.handle, self.B)
+        self.workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        self.alg_bytes, self.sampler_bytes = algorithmic_bytes(cfg, self.parent, self.B, allowed)
+        for i in range(self.ring):                       # draft tokens for the verify-only timing
+            self.sample(i, i)
+        torch.cuda.synchronize()
+
+    def sample(self, i, step, lg=None):
+        lg = self.bufs[i % self.ring] if lg is None else lg
+        self.params.step = step
+        self.L.sample_draft_tree(self.params, self.tree, lg["draft_cond"], lg["draft_uncond"],
+                                 tokens=self.tokens[i % self.ring], device_status=self.status)
+
+    def verify(self, i, step, lg=None):
+        lg = self.bufs[i % self.ring] if lg is None else lg
+        self.params.step = step
+        self.L.verify_tree(self.params, self.tree, self.nbr, lg["target_cond"], lg["target_uncond"], lg["draft_cond"],
+                           lg["draft_uncond"], self.tokens[i % self.ring], None, None, out=self.out,
+                           device_status=self.status, workspace=self.workspace)
+
+    def step(self, i, step, lg=None):
+        self.sample(i, step, lg)
+        self.verify(i, step, lg)
+
+    def kernels(self):
+        """Which kernels the library runs for these parameters (it decides; this only reports)."""
+        pv = self.L.verify_tree_path(self.params, self.tree)
+        ps = self.L.sample_draft_tree_path(self.params)
+        v = {0: ("verify_nodes_kernel + walk_kernel", 2),
+             1: ("verify_sparse_kernel + verify_nodes_kernel (repair launch, walks the trees)", 2),
+             2: ("verify_stream_kernel + walk_kernel", 2)}[pv]
+        if self.params.lazy_walk:
+            v = ("verify_nodes_kernel (path walk: one cluster per sequence)", 1)
+        s = {0: ("sample_children_kernel", 1), 1: ("sample_sparse_kernel + sample_children_kernel (repair launch)", 2),
+             2: ("sample_stream_kernel", 1)}[ps]
+        return v, s
+
+
+def time_calls(torch, call, ring, use_graph=True, min_ms=MIN_TIMED_MS, min_reps=20, max_reps=2000):
+    """Device time per call: `ring` consecutive calls (one per input set) are captured in a CUDA
+    graph and replayed; every replay is timed on its own with CUDA events on the launching
+    stream, until min_reps replays and min_ms of device time.  Returns the per-call times in ms
+    (sorted) of the replays."""
+    for i in range(min(ring, 3)):
+        call(i)
+    torch.cuda.synchronize()
+    g = None
+    if use_graph:
+        try:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(ring):
+                    call(i)
+            g.replay()
+            torch.cuda.synchronize()
+        except Exception as exc:
+            sys.stderr.write("graph capture failed, timing eager launches: %r\n" % (exc,))
+            g = None
+            torch.cuda.synchronize()
+    times, total, reps = [], 0.0, 0
+    while reps < max_reps and (reps < min_reps or total < min_ms):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        if g is not None:
+            g.replay()
+        else:
+            for i in range(ring):
+                call(i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        times.append(ms / ring)
+        total += ms
+        reps += 1
+    times.sort()
+    return times
+
+
+def summarize(times, nbytes, peak):
+    med = times[len(times) // 2]
+    gbs = nbytes / (med * 1e-3) / 1e9
+    return {"us_median": round(1e3 * med, 2), "us_min": round(1e3 * times[0], 2), "replays": len(times),
+            "gbs": round(gbs, 1), "frac_measured": round(gbs / peak, 4), "frac_nominal_8tbs": round(gbs / NOMINAL_HBM_GBS, 4)}
+
+
+def config_entry(torch, L, W, cfg, dev, peak, allowed=None, use_graph=True, ring=0, note=None):
+    """Verify / sampler / step timings of one configuration for the `configs` object."""
+    w = Workload(L, W, cfg, dev, allowed=allowed, build_table=False, ring=ring)
+    tv = time_calls(torch, lambda i: w.verify(i, 100000 + i), w.ring, use_graph)
+    ts = time_calls(torch, lambda i: w.sample(i, 100000 + i), w.ring, use_graph)
+    tt = time_calls(torch, lambda i: w.step(i, 100000 + i), w.ring, use_graph)
+    (vk, _), (sk, _) = w.kernels()
+    med = tt[len(tt) // 2]
+    ent = {"batch": w.B, "tree_nodes": w.N, "vocab": w.V, "logits": cfg.dtype, "allowed": allowed,
+           "ring": "%d input sets, %.0f MB (> 126 MB L2)" % (w.ring, w.ring * w.set_bytes / 1e6),
+           "verify_bytes": w.alg_bytes, "sampler_bytes": w.sampler_bytes,
+           "verify": dict(summarize(tv, w.alg_bytes, peak), kernel=vk),
+           "sampler": dict(summarize(ts, w.sampler_bytes, peak), kernel=sk),
+           "step_us_median": round(1e3 * med, 2), "nodes_per_s": round(w.B * w.N / (med * 1e-3)),
+           "mean_accept_len": float(w.out["accept_len"].float().mean().item()), "device_status": int(w.status.item())}
+    if note:
+        ent["note"] = note
+    del w
+    torch.cuda.empty_cache()
+    return ent
+
+
+def c1_three_numbers(torch, L, W, dev, peak, use_graph=True):
+    """Config 1 is smaller than a launch: (i) latency of a single eager verify call on an idle
+    stream, (ii) 256 decode steps over 256 distinct input sets replayed back to back in one CUDA
+    graph, (iii) the 256 steps' 256 x 26 rows verified by one launch through the batch dimension."""
+    cfg = W.CONFIGS["c1_tiny"]
+    w = Workload(L, W, cfg, dev, build_table=False, ring=256)
+    lat = []
+    for i in range(60):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        w.verify(i, 300000 + i)
+        e1.record()
+        torch.cuda.synchronize()
+        lat.append(e0.elapsed_time(e1))
+    lat = sorted(lat[10:])
+    tv = time_calls(torch, lambda i: w.verify(i, 100000 + i), w.ring, use_graph)
+    tt = time_calls(torch, lambda i: w.step(i, 100000 + i), w.ring, use_graph)
+    out = {"single_call_verify_us_median": round(1e3 * lat[len(lat) // 2], 2),
+           "graph_256_steps_verify": summarize(tv, w.alg_bytes, peak),
+           "graph_256_steps_step_us_median": round(1e3 * tt[len(tt) // 2], 2)}
+    del w
+    torch.cuda.empty_cache()
+    big = dataclasses.replace(cfg, batch=256)
+    wb = Workload(L, W, big, dev, build_table=False, ring=2)
+    tb = time_calls(torch, lambda i: wb.verify(i, 100000 + i), wb.ring, use_graph)
+    sb = time_calls(torch, lambda i: wb.sample(i, 100000 + i), wb.ring, use_graph)
+    out["steps_batched_256x26_rows_verify"] = summarize(tb, wb.alg_bytes, peak)
+    out["steps_batched_256x26_rows_sampler"] = summarize(sb, wb.sampler_bytes, peak)
+    del wb
+    torch.cuda.empty_cache()
+    return out
 
 
 def main():
@@ -281,45 +510,11 @@ def main():
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    use_graph = not args.no_graph
+    peak, peak_kind = peak_hbm()
 
-    N, B, V = len(parent), cfg.batch, cfg.vocab
-    tree = L.Tree(parent)
-    alg_bytes, sampler_bytes = algorithmic_bytes(cfg, parent, B)
-    set_bytes = sum(B * N * V * (4 if cfg.dtype == "f32" else 2) for _ in range(4 if cfg.cfg_scale is not None else 2))
-    ring = args.ring if args.ring > 0 else max(2, -(-3 * 126 * 2 ** 20 // set_bytes))
-    ring = min(ring, max(2, int(60e9 // set_bytes)))
-
-    # ---- neighbour table: built once per codebook by the library (timed on its own)
-    codebook = W.make_codebook(cfg.codebook_size, cfg.codebook_dim, cfg.codebook_dtype, seed=cfg.index, device=dev)
-    nbr = L.build_neighbors(codebook, cfg.k)
-    torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    tb = []
-    for _ in range(3):
-        ev0.record()
-        nbr = L.build_neighbors(codebook, cfg.k)
-        ev1.record()
-        torch.cuda.synchronize()
-        tb.append(ev0.elapsed_time(ev1))
-    table_ms = min(tb)
-
-    # ---- inputs: a ring of independent step buffers, together larger than L2
-    bufs = [W.make_logits(cfg, step=1000 * rank + s, device=dev) for s in range(ring)]
-    params = L.Params(vocab=V, cfg_scale=cfg.cfg_scale if cfg.cfg_scale is not None else 1.0,
-                      temperature=cfg.temperature, top_k_target=cfg.top_k, top_k_draft=cfg.top_k, lam=cfg.lam,
-                      k=cfg.k, code_offset=cfg.code_offset, n_codes=cfg.codebook_size, seed=0x1A27E2 + rank,
-                      lazy_walk=1 if args.walk == "lazy" else 0)
-    tokens = torch.zeros((B, N), dtype=torch.int32, device=dev)
-    out = {}
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-    need = L.lib.lantern_verify_tree_workspace(tree.handle, B)
-    workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
-
-    def step(i, lg):
-        params.step = i
-        L.sample_draft_tree(params, tree, lg["draft_cond"], lg["draft_uncond"], tokens=tokens, device_status=status)
-        L.verify_tree(params, tree, nbr, lg["target_cond"], lg["target_uncond"], lg["draft_cond"], lg["draft_uncond"],
-                      tokens, None, None, out=out, device_status=status, workspace=workspace)
+    w = Workload(L, W, cfg, dev, rank=rank, ring=args.ring, walk=args.walk)
+    N, B, V, ring = w.N, w.B, w.V, w.ring
 
     def sync_all():
         torch.cuda.synchronize()
@@ -327,94 +522,74 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    for i in range(max(3, args.warmup)):
-        step(i, bufs[i % ring])
+    warm = max(3, args.warmup)
+    for i in range(warm):
+        w.step(i, i)
     sync_all()
 
-    # ---- timed region: exactly K steps, device-resident inputs.  The launches of `ring`
-    # consecutive steps are captured once in a CUDA graph and replayed (the step is three small
+    # ---- timed region: exactly K steps on device-resident inputs.  The launches of `ring`
+    # consecutive steps are captured once in a CUDA graph and replayed (a step is a few short
     # launches: without a graph the host, not the GPU, sets the pace of the small workloads).
+    # The K-step region is repeated until MIN_TIMED_MS of device time has been timed; the
+    # median repetition is reported.
     K = args.steps
-
-    def verify_only(i, lg):
-        params.step = 100000 + i
-        L.verify_tree(params, tree, nbr, lg["target_cond"], lg["target_uncond"], lg["draft_cond"], lg["draft_uncond"],
-                      tokens, None, None, out=out, device_status=status, workspace=workspace)
-
-    def full_step(i, lg):
-        params.step = 100000 + i
-        L.sample_draft_tree(params, tree, lg["draft_cond"], lg["draft_uncond"], tokens=tokens, device_status=status)
-        verify_only(i, lg)
-
     per_graph = min(ring, max(1, K))
-    g_step = g_verify = None
-    if not args.no_graph:
+    g_step = None
+    if use_graph:
         try:
             g_step = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g_step):
                 for i in range(per_graph):
-                    full_step(i, bufs[i % ring])
-            g_verify = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g_verify):
-                for i in range(per_graph):
-                    verify_only(i, bufs[i % ring])
+                    w.step(i, 100000 + i)
             g_step.replay()
-            g_verify.replay()
             torch.cuda.synchronize()
         except Exception as exc:                    # capture not possible: time eager launches
             sys.stderr.write("graph capture failed, timing eager launches: %r\n" % (exc,))
-            g_step = g_verify = None
+            g_step = None
             torch.cuda.synchronize()
     clocks = ClockSampler(local)
     time.sleep(0.3)
-    sync_all()
-    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    done = 0
-    if g_step is not None:
-        while done + per_graph <= K:
-            g_step.replay()
-            done += per_graph
-    while done < K:
-        full_step(done, bufs[done % ring])
-        done += 1
-    t_end.record()
-    sync_all()
-    elapsed_ms = t_start.elapsed_time(t_end)
-    # the dominant kernel on its own (same stream, same buffers, measured live)
-    v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n_verify = 0
-    v0.record()
-    if g_verify is not None:
-        while n_verify < min(K, 512):
-            g_verify.replay()
-            n_verify += per_graph
-    else:
-        while n_verify < min(K, 256):
-            verify_only(n_verify, bufs[n_verify % ring])
-            n_verify += 1
-    v1.record()
-    sync_all()
+    regions, total_ms = [], 0.0
+    while len(regions) < 3 or (total_ms < MIN_TIMED_MS and len(regions) < 200):
+        sync_all()
+        t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_start.record()
+        done = 0
+        if g_step is not None:
+            while done + per_graph <= K:
+                g_step.replay()
+                done += per_graph
+        while done < K:
+            w.step(done, 100000 + done)
+            done += 1
+        t_end.record()
+        sync_all()
+        ms = t_start.elapsed_time(t_end)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        regions.append(ms)
+        total_ms += ms
+    regions.sort()
+    elapsed_ms = regions[len(regions) // 2]
+    # the dominant kernel on its own, and the sampler (same stream, same buffers, measured live)
+    tv = time_calls(torch, lambda i: w.verify(i, 100000 + i), ring, use_graph)
+    ts = time_calls(torch, lambda i: w.sample(i, 100000 + i), ring, use_graph)
     clk = clocks.stop()
-    verify_avg_ms = v0.elapsed_time(v1) / n_verify
-    verify_ms = [verify_avg_ms]
-    accept_mean = float(out["accept_len"].float().mean().item())
-    dev_status = int(status.item())
-
-    if world > 1:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    verify_med_ms = tv[len(tv) // 2]
+    accept_mean = float(w.out["accept_len"].float().mean().item())
+    dev_status = int(w.status.item())
     total_nodes = world * B * N * K
     value = total_nodes / (elapsed_ms * 1e-3)
 
     # ---- end to end: per step, inputs come from pinned host memory and results go back
     KE = max(1, min(args.e2e_steps, K))
     host = {k: (None if v is None else torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v))
-            for k, v in bufs[0].items()}
-    stage = {k: (None if v is None else torch.empty_like(v)) for k, v in bufs[0].items()}
+            for k, v in w.bufs[0].items()}
+    stage = {k: (None if v is None else torch.empty_like(v)) for k, v in w.bufs[0].items()}
     h_len = torch.empty((B,), dtype=torch.int32, pin_memory=True)
-    h_tok = torch.empty((B, tree.max_depth + 1), dtype=torch.int32, pin_memory=True)
+    h_tok = torch.empty((B, w.tree.max_depth + 1), dtype=torch.int32, pin_memory=True)
     h2d = sum(v.numel() * v.element_size() for v in host.values() if v is not None)
     d2h = h_len.numel() * 4 + h_tok.numel() * 4
 
@@ -422,15 +597,16 @@ def main():
         for k_, v in host.items():
             if v is not None:
                 stage[k_].copy_(v, non_blocking=True)
-        step(200000 + i, stage)
-        h_len.copy_(out["accept_len"], non_blocking=True)
-        h_tok.copy_(out["out_tokens"], non_blocking=True)
+        w.step(0, 200000 + i, stage)
+        h_len.copy_(w.out["accept_len"], non_blocking=True)
+        h_tok.copy_(w.out["out_tokens"], non_blocking=True)
         torch.cuda.synchronize()
 
     for i in range(3):
         e2e_step(i)
     sync_all()
     w0 = time.perf_counter()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record()
     for i in range(KE):
         e2e_step(i)
@@ -442,7 +618,9 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
     e2e_value = world * B * N * KE / (e2e_ms * 1e-3)
+    del host, stage
 
+    alg_bytes = w.alg_bytes
     if args.walk == "lazy":
         # the path walk reads only the rows of the nodes it visits: count them for the same calls
         # the verify-only timing made (each input set of the ring once)
@@ -454,54 +632,75 @@ def main():
         e_sz = 4 if cfg.dtype == "f32" else 2
         total = 0
         for i in range(ring):
-            verify_only(i, bufs[i % ring])
+            w.verify(i, 100000 + i)
             torch.cuda.synchronize()
-            al = out["accept_len"].cpu().numpy()
-            on = out["out_nodes"].cpu().numpy()
+            al = w.out["accept_len"].cpu().numpy()
+            on = w.out["out_nodes"].cpu().numpy()
             for b in range(B):
                 for n in [0] + [int(x) for x in on[b, : int(al[b])]]:
                     total += (2 if n in kids else 1) * c_ops * V * e_sz
         alg_bytes = total // ring
-    # which kernels ran (the library decides from the parameters; this only reports it)
-    lists_v = L.verify_tree_path(params, tree) == 1
-    lists_s = L.sample_draft_tree_path(params) == 1
-    verify_kernels = ("verify_sparse_kernel + verify_nodes_kernel (repair launch, walks the trees)" if lists_v
-                      else "verify_nodes_kernel + walk_kernel")
-    launches_per_step = (2 if lists_s else 1) + 2
-    if args.walk == "lazy":
-        verify_kernels = "verify_nodes_kernel (path walk: one cluster per sequence)"
-        launches_per_step = (2 if lists_s else 1) + 1
+    (vk, vl), (sk, sl) = w.kernels()
+    launches_per_step = vl + sl
+    table = {"ms": w.table_ms, "L": cfg.codebook_size, "d": cfg.codebook_dim, "k": cfg.k, "dtype": cfg.codebook_dtype}
+    set_bytes = w.set_bytes
+    del w
+    torch.cuda.empty_cache()
+
     if rank == 0:
-        peak, peak_kind = peak_hbm()
-        achieved = alg_bytes / (verify_avg_ms * 1e-3) / 1e9
+        achieved = alg_bytes / (verify_med_ms * 1e-3) / 1e9
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": warm,
             "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
+            "dtype": cfg.dtype, "data": "synthetic",
             "config": {"workload": cfg.name, "batch_per_gpu": B, "tree_nodes": N, "vocab": V, "logits": cfg.dtype,
+                       "arithmetic": "f32 (exact re-ranking steps in f64)",
                        "cfg_scale": cfg.cfg_scale, "top_k": cfg.top_k, "neighbours_k": cfg.k, "lambda": cfg.lam,
                        "codebook": [cfg.codebook_size, cfg.codebook_dim], "parallelism": "dp%d" % world,
                        "l2_policy": "ring of %d input sets, %.0f MB in total (> 126 MB L2)" % (ring, ring * set_bytes / 1e6),
                        "step": "sample_draft_tree + verify_tree (incl. walk), %d kernel launches" % launches_per_step,
                        "walk": args.walk + (" (only the rows on the accepted paths are read; algorithmic_bytes counts those)"
                                             if args.walk == "lazy" else ""),
-                       "launch": "cuda graph of %d steps, replayed" % per_graph if g_step is not None else "eager"},
-            "roofline": {"bound": "hbm", "kernel": verify_kernels, "achieved": achieved, "peak": peak,
-                         "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": measured_traffic(cfg.name) if args.walk == "eager" else None,
-                         "algorithmic_bytes": alg_bytes, "launch_ms_avg": verify_avg_ms,
-                         "launch_ms_median": verify_ms[len(verify_ms) // 2],
-                         "step_bytes_incl_sampler": alg_bytes + sampler_bytes,
-                         "step_gbs": (alg_bytes + sampler_bytes) / (elapsed_ms / K * 1e-3) / 1e9},
+                       "launch": "cuda graph of %d steps, replayed" % per_graph if g_step is not None else "eager",
+                       "timed": "region of exactly %d steps, repeated %d times (%.0f ms of device time); median region"
+                                % (K, len(regions), total_ms)},
+            "roofline": {"bound": "hbm", "kernel": vk, "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
+                         "frac_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+                         "traffic": measured_traffic(cfg.name) if args.walk == "eager" else None,
+                         "algorithmic_bytes": alg_bytes, "launch_ms_median": verify_med_ms, "launch_ms_min": tv[0],
+                         "replays": len(tv),
+                         "sampler": dict(summarize(ts, algorithmic_bytes(cfg, parent, B)[1], peak), kernel=sk),
+                         "step_bytes_incl_sampler": alg_bytes + algorithmic_bytes(cfg, parent, B)[1],
+                         "step_gbs": (alg_bytes + algorithmic_bytes(cfg, parent, B)[1]) / (elapsed_ms / K * 1e-3) / 1e9},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": KE},
             "gpu_launches": launches_per_step * K,
             "clocks": clk,
-            "table_build": {"ms": table_ms, "L": cfg.codebook_size, "d": cfg.codebook_dim, "k": cfg.k,
-                            "dtype": cfg.codebook_dtype},
+            "table_build": table,
             "stats": {"mean_accept_len": accept_mean, "tokens_per_step": accept_mean + 1.0, "device_status": dev_status},
         }
+        if world == 1 and args.configs == "all" and args.walk == "eager":
+            cfgs = {}
+            for name in ("c1_tiny", "c2_llamagen512", "c3_lumina", "c4_batch64"):
+                if name == cfg.name:
+                    cfgs[name] = {"see": "headline of this line", "verify": dict(summarize(tv, alg_bytes, peak), kernel=vk),
+                                  "sampler": line["roofline"]["sampler"], "step_us_median": round(1e3 * elapsed_ms / K, 2),
+                                  "nodes_per_s": round(value)}
+                    continue
+                cfgs[name] = config_entry(torch, L, W, W.CONFIGS[name], dev, peak, use_graph=use_graph)
+            c3 = W.CONFIGS["c3_lumina"]
+            cfgs["c3_lumina_image_tokens_only"] = config_entry(
+                torch, L, W, c3, dev, peak, allowed=(c3.code_offset, c3.code_offset + c3.codebook_size), use_graph=use_graph,
+                ring=16, note="tokens restricted to the 8192 image codes; bytes counted for that slice of every row")
+            cfgs["c1_tiny"]["three_numbers"] = c1_three_numbers(torch, L, W, dev, peak, use_graph)
+            rows, dup = table_sweep(False)
+            cfgs["c5_table_sweep"] = {
+                "dup_frac": dup, "total_ms": round(sum(r["ms"] for r in rows), 2),
+                "builds": [[r["L"], r["d"], r["k"], r["ms"], round(r["contraction_tflops"], 2), r["path"]] for r in rows],
+                "columns": ["L", "d", "k", "ms", "contraction TFLOP/s (2 L^2 d / time)", "path"]}
+            line["configs"] = cfgs
         if world == 1 and not args.no_cpu_baseline:
-            lg_cpu = {k: (None if v is None else v.cpu()) for k, v in bufs[0].items()}
-            line["cpu_baseline"] = cpu_baseline(cfg, parent, lg_cpu)
+            line["cpu_baseline"] = cpu_baseline(cfg, parent)
         print(json.dumps(line))
     if world > 1:
         dist.barrier()

@@ -43,7 +43,10 @@ enum {
                                    treated as probability 0                                     */
   LANTERN_DEV_TIMEOUT = 2,      /* a bounded on-chip wait expired; the data was re-read with
                                    plain loads                                                  */
-  LANTERN_DEV_EMPTY_ROW = 4     /* a row had no finite logit                                    */
+  LANTERN_DEV_EMPTY_ROW = 4,    /* a row had no finite logit                                    */
+  LANTERN_DEV_KEY_TIES = 8      /* draft sampling: more Gumbel keys than the kernel ranks exactly
+                                   lay within 2.5e-4 of the last child's key; the children are
+                                   distinct draws, their order may differ from an exact ranking */
 };
 
 const char* lantern_status_string(lantern_status s);

@@ -34,6 +34,7 @@ struct SampleArgs {
 
 }  // namespace lantern
 #include "sampler_sparse.cuh"
+#include "sampler_stream.cuh"
 namespace lantern {
 
 __device__ __forceinline__ bool better(float ka, int ia, float kb, int ib) {   // a beats b
@@ -306,6 +307,31 @@ static cudaError_t launch_sample_sparse(const SampleArgs& a, int V, cudaStream_t
   return launch_sample_sparse_e<T, CFG, 32>(a, st);
 }
 
+
+// ---- launch of the streaming kernel (rows without top-k): one CTA, or a cluster, per parent
+template <typename T, bool CFG, bool TAU1>
+static cudaError_t launch_sample_stream_t(const SampleArgs& a, int cs, cudaStream_t st) {
+  auto kern = stream::sample_stream_kernel<T, CFG, TAU1>;
+  const size_t smem = stream::sampler_stream_smem();
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  if (cs > 8) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+  }
+  return launch_after_previous(kern, static_cast<unsigned>(a.B) * a.n_parents * cs, stream::ST, smem, st, cs, a);
+}
+static cudaError_t launch_sample_stream(const SampleArgs& a, int cs, bool f32, bool cfg, cudaStream_t st) {
+  const bool tau1 = a.inv_tau == 1.0f;
+  if (f32) {
+    if (cfg) return launch_sample_stream_t<float, true, false>(a, cs, st);
+    return tau1 ? launch_sample_stream_t<float, false, true>(a, cs, st) : launch_sample_stream_t<float, false, false>(a, cs, st);
+  }
+  if (cfg) return launch_sample_stream_t<__nv_bfloat16, true, false>(a, cs, st);
+  return tau1 ? launch_sample_stream_t<__nv_bfloat16, false, true>(a, cs, st)
+              : launch_sample_stream_t<__nv_bfloat16, false, false>(a, cs, st);
+}
+
 }  // namespace lantern
 
 using namespace lantern;
@@ -321,8 +347,14 @@ bool sampler_uses_lists(const lantern_params* p) {
 }
 }  // namespace
 
+// Rows that no top-k truncates take the streaming kernel.
+static bool sampler_uses_stream(const lantern_params* p) {
+  return !(p->top_k_draft > 0 && p->top_k_draft < p->vocab) && p->vocab <= stream::kMaxV;
+}
+
 extern "C" int32_t lantern_sample_draft_tree_path(const lantern_params* p) {
   if (!p) return -1;
+  if (sampler_uses_stream(p)) return LANTERN_PATH_STREAM;
   return sampler_uses_lists(p) ? LANTERN_PATH_LISTS : LANTERN_PATH_DENSE;
 }
 
@@ -366,12 +398,26 @@ extern "C" lantern_status lantern_sample_draft_tree(
   a.tokens = tokens; a.draft_prob = draft_prob; a.status = device_status;
   a.n_parents = i1 - i0;
   a.repair = 0;
-  int cs, e;
-  size_t smem;
-  const int ov = lantern_set_cluster_size(-1);     // -1 is not a valid size: reads the current value
-  if (!sampler_shape(V, batch * (i1 - i0), dt == LANTERN_F32 ? 4 : 8, ov, &cs, &e, &smem)) return LANTERN_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = draft_uncond != nullptr;
+  const int ov = lantern_set_cluster_size(-1);     // -1 is not a valid size: reads the current value
+  if (sampler_uses_stream(p)) {
+    // CTAs per parent: one when the parents alone fill the machine
+    int cs = ov;
+    if (cs <= 0) {
+      int dev = 0, sms = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+      const int nvec = (allow_hi - allow_lo) / (dt == LANTERN_F32 ? 4 : 8);
+      cs = 1;
+      while (cs < 16 && static_cast<long long>(batch) * (i1 - i0) * cs < 4 * sms && nvec / (2 * cs * stream::SW) >= 32) cs *= 2;
+    }
+    return launch_sample_stream(a, cs, dt == LANTERN_F32, cfg, st) == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
+  }
+  int cs, e;
+  size_t smem;
+  if (!sampler_shape(V, batch * (i1 - i0), dt == LANTERN_F32 ? 4 : 8, ov, &cs, &e, &smem)) return LANTERN_ERR_UNSUPPORTED;
   cudaError_t err;
   // Rows truncated to a moderate top-k take the list-based kernel; the dense kernel then draws
   // the parents it marked as not fitting (usually none).

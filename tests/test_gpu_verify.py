@@ -100,7 +100,7 @@ def test_path_queries_and_graph_replay_match_eager_calls(L):
     tree = L.Tree(case.parent)
     assert L.verify_tree_path(par, tree) == 1 and L.sample_draft_tree_path(par) == 1
     par_dense = L.Params(**{**par.__dict__, "top_k_target": 0, "top_k_draft": 0})
-    assert L.verify_tree_path(par_dense, tree) == 2 and L.sample_draft_tree_path(par_dense) == 0      # streaming kernel
+    assert L.verify_tree_path(par_dense, tree) == 2 and L.sample_draft_tree_path(par_dense) == 2      # streaming kernels
     par_walk = L.Params(**{**par_dense.__dict__, "lazy_walk": 1})
     assert L.verify_tree_path(par_walk, tree) == 0
     old = L.set_cluster_size(1)
