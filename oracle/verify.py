@@ -25,13 +25,16 @@ from .postprocess import postprocess_row
 from .tree import tree_children
 
 
-def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None, delta=0.0):
+def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None, delta=0.0, force_members=None):
     """Sec. 4: m = sum of q over A_{k,lambda}(x) and the members of A besides x.
     With delta > 0 the additive bound of Sec. 2.2 replaces the multiplicative one:
     the neighbours' own running sum stays below delta (A_{k,delta}); lam is unused.
 
     If `margins` is a list, |running sum - bound| of every comparison made is
-    appended to it (diagnostic for near-tie accounting; no effect on the result)."""
+    appended to it (diagnostic for near-tie accounting; no effect on the result).
+    `force_members` (diagnostic, used only when a comparison with another
+    implementation continues past a near-tie): take exactly that many list entries
+    instead of applying the bound."""
     cum = q_cur[x]
     bound = q_cur[x] + delta if delta > 0 else lam * q_cur[x]
     members = []
@@ -41,7 +44,8 @@ def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None, 
             a = code_offset + int(nbr_idx[code][r])
             if margins is not None:
                 margins.append(abs(cum + q_cur[a] - bound))
-            if cum + q_cur[a] < bound:
+            take = cum + q_cur[a] < bound if force_members is None else r < force_members
+            if take:
                 cum = cum + q_cur[a]
                 members.append(a)
             else:
@@ -58,10 +62,14 @@ def moved_mass(q_cur, x, m, members):
     return q_t
 
 
-def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset, n_codes, delta=0.0):
+def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset, n_codes, delta=0.0, forced=None):
     """Test the children of one node in stored order (Sec. 4; App. A.2 Eq. 1-2).
 
-    Returns (accepted child or -1, q_cur, {child: (m, thr, cut_margin)}): q_cur
+    `forced` (diagnostic): {child: {"accept": bool, "n_members": int}} overrides the
+    accept decision and / or the size of A of that child, so that a comparison can go
+    on after a floating-point near-tie with the other side's decision imposed.
+
+    Returns (accepted child or -1, q_cur, {child: (m, thr, cut_margin, |A| - 1)}): q_cur
     is the target distribution left after the rejections (q itself at a leaf);
     cut_margin is the smallest |running sum - bound| met while forming A."""
     q_cur = np.array(q, dtype=np.float64)
@@ -72,13 +80,18 @@ def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset
         if x < 0:
             continue
         margins = []
-        m, members = relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins, delta)
+        f = (forced or {}).get(c, {})
+        m, members = relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins, delta,
+                                  force_members=f.get("n_members"))
         if p_cur[x] > 0:
             thr = min(1.0, m / p_cur[x])          # Sec. 4, final accept probability
         else:
             thr = 1.0 if m > 0 else 0.0
-        tested[c] = (m, thr, min(margins) if margins else np.inf)
-        if float(u_accept[c]) < thr:
+        tested[c] = (m, thr, min(margins) if margins else np.inf, len(members))
+        accept = float(u_accept[c]) < thr
+        if "accept" in f:
+            accept = bool(f["accept"])
+        if accept:
             return c, q_cur, tested
         q_t = moved_mass(q_cur, x, m, members)
         r = np.maximum(q_t - p_cur, 0.0)           # Eq. 2
@@ -103,17 +116,17 @@ def inverse_cdf(dist, u, return_margin=False):
 
 
 def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
-                code_offset, n_codes, delta=0.0):
+                code_offset, n_codes, delta=0.0, forced=None):
     """Process one tree node.
 
     q: target distribution of the node; p: drafter distribution (None at a leaf)
     child_ids: its children in stored order; tokens[c]: draft token of node c
     (a negative token means "no draft" and is skipped).
-    Returns (next_child or -1, sampled token or -1, {child: (m, thr, cut_margin)});
+    Returns (next_child or -1, sampled token or -1, {child: (m, thr, cut_margin, |A| - 1)});
     tested["resample_margin"] is set when a token was drawn.
     """
     nxt, q_cur, tested = sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam,
-                                      code_offset, n_codes, delta)
+                                      code_offset, n_codes, delta, forced)
     if nxt >= 0:
         return nxt, -1, tested
     j, margin = inverse_cdf(q_cur, u_resample, return_margin=True)
@@ -166,7 +179,7 @@ def verify_sequence(parent, target_cond, target_uncond, draft_cond, draft_uncond
                                        nbr_idx, k, lam, code_offset, n_codes, delta)
         node_next[n], node_token[n] = nxt, tok
         resample_margin[n] = tested.pop("resample_margin", np.inf)
-        for c, (m, thr, cm) in tested.items():
+        for c, (m, thr, cm, _) in tested.items():
             node_mass[c], node_thresh[c], cut_margin[c] = m, thr, cm
     accept_len, out_tokens, out_nodes = walk(node_next, node_token, tokens)
     return dict(node_next=node_next, node_token=node_token, node_mass=node_mass,

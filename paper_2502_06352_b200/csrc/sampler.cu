@@ -37,6 +37,8 @@ struct SampleArgs {
 #include "sampler_stream.cuh"
 namespace lantern {
 
+constexpr float kDenseKeyErr = 2e-5f;     // bound on |float32 key - exact key| (|key| < 64)
+
 __device__ __forceinline__ bool better(float ka, int ia, float kb, int ib) {   // a beats b
   return ka > kb || (ka == kb && ia < ib);
 }
@@ -104,6 +106,12 @@ __device__ __forceinline__ void sample_node(const SampleArgs& a, const int idx, 
   const bool has_topk = kth[0] > 0;
   if (has_topk) topk_thresholds<E>(c, tk, Z, Z, mx, kth, theta);
 
+  // (the top-k routine's candidate scratch is dead from here on: it holds the rounds' winners and
+  // the near-tied tokens of the exact re-ranking)
+  float* fx_key = tk.all;                                   // [8]
+  int* fx_tok = reinterpret_cast<int*>(tk.all + 8);         // [8]
+  int* fx_cand = fx_tok + 8;                                // [32]
+  int* fx_cnt = fx_cand + 32;
   // ---- keys z + G, G = -log(-log U), and the softmax denominator, in one sweep
   const uint32_t row_id = static_cast<uint32_t>(out_b + n);
   const float* gum = a.gumbel ? a.gumbel + (static_cast<long long>(row_id) * a.V + lo) : nullptr;
@@ -164,6 +172,7 @@ __device__ __forceinline__ void sample_node(const SampleArgs& a, const int idx, 
       c.parity ^= 1;
     }
     const bool valid = ck != -INFINITY;
+    if (tid == 0) { fx_key[round] = ck; fx_tok[round] = valid ? ci : -1; }
     if (valid && ci == bi) {                    // exactly one thread of the row owns the winner
       const int jl = ci - lo;
       K[jl] = -INFINITY;
@@ -174,6 +183,78 @@ __device__ __forceinline__ void sample_node(const SampleArgs& a, const int idx, 
     if (!valid && c.rank == 0 && tid == 0) {
       a.tokens[out_b + fc + round] = -1;
       if (a.draft_prob) a.draft_prob[out_b + fc + round] = 0.f;
+    }
+  }
+
+  // ---- exact order.  The rounds ranked float32 keys (error below kDenseKeyErr each).  Where two
+  // of the chosen keys, or a chosen key and one left out, are closer than twice that, the
+  // entries involved are ranked again by keys evaluated in double precision (ties: lower token
+  // id) by CTA 0 of the row, which reads the other CTAs' near-tied tokens through DSMEM.
+  __syncthreads();
+  int nv = 0;
+  while (nv < nc && fx_tok[nv] >= 0) ++nv;
+  const float k_last = nv > 0 ? fx_key[nv - 1] : 0.f;
+  bool need = false;
+  for (int r = 1; r < nv; ++r) need |= fx_key[r - 1] - fx_key[r] <= 2.f * kDenseKeyErr;
+  if (tid == 0) *fx_cnt = 0;
+  __syncthreads();
+  if (nv > 0) {
+#pragma unroll
+    for (int v = 0; v < NV4; ++v) {
+      const int j = warp * 32 * E + v * 128 + lane * 4;
+      const float4 k4 = *reinterpret_cast<const float4*>(K + j);
+      const float kv[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (kv[e] != -INFINITY && kv[e] >= k_last - 2.f * kDenseKeyErr) {
+          const int at = atomicAdd(fx_cnt, 1);
+          if (at < 32) fx_cand[at] = lo + j + e;
+        }
+      }
+    }
+  }
+  csync(c);                                     // every CTA's list of near-tied tokens is complete
+  if (c.rank == 0 && warp == 0 && nv > 0) {
+    int ncand = nv, extra = 0;
+    int t = lane < nv ? fx_tok[lane] : 0x7fffffff;
+    for (uint32_t q = 0; q < c.nrank; ++q) {
+      const int nq = single ? *fx_cnt : static_cast<int>(dsmem_ld_u32(dsmem_addr(smem_u32(fx_cnt), q)));
+      extra += nq;
+      for (int i = 0; i < nq && i < 32; ++i) {
+        const int tq = single ? fx_cand[i] : static_cast<int>(dsmem_ld_u32(dsmem_addr(smem_u32(&fx_cand[i]), q)));
+        if (ncand < 32 && lane == ncand) t = tq;
+        ++ncand;
+      }
+    }
+    if (extra > 0 || need) {
+      if (ncand > 32) {
+        if (lane == 0) vflag(a.status, LANTERN_DEV_KEY_TIES);     // more near-ties than one warp ranks
+      } else {
+        double key = -INFINITY;
+        float z = 0.f;
+        if (lane < ncand) {
+          z = combine<CFG>(Vec<T>::widen(dcp[t]), CFG ? Vec<T>::widen(dup[t]) : 0.f, a.g, a.inv_tau);
+          float u;
+          if (a.gumbel) {
+            u = __ldcs(a.gumbel + static_cast<long long>(row_id) * a.V + t);
+          } else {
+            const Philox4 r = philox_stream(a.seed, a.step, row_id, kStreamGumbel, static_cast<uint32_t>(t >> 2));
+            const uint32_t w = (t & 3) == 0 ? r.x : ((t & 3) == 1 ? r.y : ((t & 3) == 2 ? r.z : r.w));
+            u = uniform_open(w);
+          }
+          key = static_cast<double>(z) - log(-log(static_cast<double>(u)));
+        }
+        int rank = 0;
+        for (int o = 0; o < ncand; ++o) {
+          const double ko = __shfl_sync(0xffffffffu, key, o);
+          const int to = __shfl_sync(0xffffffffu, t, o);
+          rank += (ko > key || (ko == key && to < t)) ? 1 : 0;
+        }
+        if (lane < ncand && rank < nv) {
+          a.tokens[out_b + fc + rank] = t;
+          if (a.draft_prob) a.draft_prob[out_b + fc + rank] = ex2_approx(fmaf(z, kLog2e, c0)) * inv_sum;
+        }
+      }
     }
   }
 }

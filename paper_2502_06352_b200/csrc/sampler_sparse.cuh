@@ -14,10 +14,11 @@ namespace sparse {
 
 constexpr int kRedoToken = -2;
 constexpr int kPerThread = kCap / ST;     // list entries per thread
+constexpr float kKeyErr = 2e-5f;          // bound on |float32 key - exact key| (|key| < 64)
 
 __host__ __device__ constexpr size_t sampler_smem_bytes(int e) {
   return static_cast<size_t>(ST) * e * 4 + 3 * kCap * 4 + kBins * 4 + kWords * 4 + kCand * 4 + 2 * SW * 2 * 4 +
-         SW * 4 + kMisc * 4 + 2 * 2 * SW * 4;
+         SW * 4 + kMisc * 4 + 2 * 2 * SW * 4 + (8 + 8 + 8 + 32 + 4) * 4;
 }
 
 __device__ __forceinline__ bool key_better(float ka, int ia, float kb, int ib) {   // a beats b
@@ -55,6 +56,11 @@ __global__ void __launch_bounds__(ST, 2) sample_sparse_kernel(const SampleArgs a
   s.wtot = reinterpret_cast<uint32_t*>(c.red + 2 * SW * 2);
   s.misc = reinterpret_cast<int*>(s.wtot + SW);
   float* pk = reinterpret_cast<float*>(s.misc + kMisc);    // [2][2*SW] warps' best key and token, two buffers
+  float* wkey = pk + 2 * 2 * SW;                           // [8] keys of the rounds' winners
+  int* wtok = reinterpret_cast<int*>(wkey + 8);            // [8] their tokens (-1: none), [8] their list positions
+  int* wpos = wtok + 8;
+  int* cpos = wpos + 8;                                    // [32] list positions of the entries ranked exactly
+  int* ccnt = cpos + 32;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int idx = blockIdx.x;
@@ -127,7 +133,9 @@ __global__ void __launch_bounds__(ST, 2) sample_sparse_kernel(const SampleArgs a
     int ci = lane < SW ? __float_as_int(buf[SW + lane]) : 0x7fffffff;
     warp_key_best(ck, ci);
     const bool valid = ck != -INFINITY;
+    if (tid == 0) { wkey[round] = ck; wtok[round] = valid ? ci : -1; }
     if (valid && ci == bi) {                    // exactly one thread owns the winner
+      wpos[round] = bpos;
       a.tokens[out_b + fc + round] = ci;
       if (a.draft_prob)
         a.draft_prob[out_b + fc + round] = ex2_approx(fmaf(s.lval[0][bpos], kLog2e, c0)) * inv_sum;
@@ -147,6 +155,72 @@ __global__ void __launch_bounds__(ST, 2) sample_sparse_kernel(const SampleArgs a
     if (!valid && tid == 0) {
       a.tokens[out_b + fc + round] = -1;
       if (a.draft_prob) a.draft_prob[out_b + fc + round] = 0.f;
+    }
+  }
+
+  // ---- exact order.  The rounds ranked float32 keys (error below kKeyErr each).  Where two of
+  // the chosen keys, or a chosen key and one left out, are closer than 2 * kKeyErr, the entries
+  // involved are ranked again by keys evaluated in double precision (ties: lower token id).
+  __syncthreads();
+  int nv = 0;
+  while (nv < nc && wtok[nv] >= 0) ++nv;
+  if (nv == 0) return;
+  const float k_last = wkey[nv - 1];
+  bool close = false;
+  for (int r = 1; r < nv; ++r) close |= wkey[r - 1] - wkey[r] <= 2.f * kKeyErr;
+  bool mine = false;
+#pragma unroll
+  for (int m = 0; m < kPerThread; ++m) {
+    const int i = tid + m * ST;
+    if (i >= n_list) break;
+    mine |= keys[i] != -INFINITY && keys[i] >= k_last - 2.f * kKeyErr;
+  }
+  if (!__syncthreads_or((mine || close) ? 1 : 0)) return;
+  if (tid < nv) { cpos[tid] = wpos[tid]; }
+  if (tid == 0) *ccnt = nv;
+  __syncthreads();
+#pragma unroll
+  for (int m = 0; m < kPerThread; ++m) {
+    const int i = tid + m * ST;
+    if (i >= n_list) break;
+    if (keys[i] != -INFINITY && keys[i] >= k_last - 2.f * kKeyErr) {
+      const int at = atomicAdd(ccnt, 1);
+      if (at < 32) cpos[at] = i;
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int ncand = *ccnt;
+    if (ncand > 32) {                             // more near-ties than one warp ranks
+      if (lane == 0) vflag(a.status, LANTERN_DEV_KEY_TIES);
+      return;
+    }
+    double key = -INFINITY;
+    int t = 0x7fffffff;
+    float z = 0.f;
+    if (lane < ncand) {
+      const int i = cpos[lane];
+      t = s.ltok[0][i];
+      z = s.lval[0][i];
+      float u;
+      if (gum) {
+        u = __ldcs(gum + t);
+      } else {
+        const Philox4 r = philox_stream(a.seed, a.step, row_id, kStreamGumbel, static_cast<uint32_t>(t >> 2));
+        const uint32_t w = (t & 3) == 0 ? r.x : ((t & 3) == 1 ? r.y : ((t & 3) == 2 ? r.z : r.w));
+        u = uniform_open(w);
+      }
+      key = static_cast<double>(z) - log(-log(static_cast<double>(u)));
+    }
+    int rank = 0;
+    for (int o = 0; o < ncand; ++o) {
+      const double ko = __shfl_sync(0xffffffffu, key, o);
+      const int to = __shfl_sync(0xffffffffu, t, o);
+      rank += (ko > key || (ko == key && to < t)) ? 1 : 0;
+    }
+    if (lane < ncand && rank < nv) {
+      a.tokens[out_b + fc + rank] = t;
+      if (a.draft_prob) a.draft_prob[out_b + fc + rank] = ex2_approx(fmaf(z, kLog2e, c0)) * inv_sum;
     }
   }
 }

@@ -25,10 +25,19 @@
 namespace lantern {
 namespace stream {
 
-constexpr int ST = 256;            // threads per CTA
+#ifndef LANTERN_STREAM_THREADS
+#define LANTERN_STREAM_THREADS 256
+#endif
+#ifndef LANTERN_STREAM_MINB
+#define LANTERN_STREAM_MINB 4
+#endif
+#ifndef LANTERN_STREAM_PAD
+#define LANTERN_STREAM_PAD 0
+#endif
+constexpr int ST = LANTERN_STREAM_THREADS;            // threads per CTA
 constexpr int SW = ST / 32;        // warps per CTA
 constexpr int kMaxV = 1 << 20;     // bitmap: V / 8 bytes of shared memory
-constexpr int kSmallBytes = 1024;  // reductions, per-warp sums, scalars
+constexpr int kSmallBytes = 2048 + LANTERN_STREAM_PAD;  // reductions, per-warp sums, scalars
 
 // shared-memory bytes of one CTA
 __host__ __device__ constexpr size_t smem_bytes(int V, int max_children, int kp1, bool cfg) {
@@ -709,7 +718,7 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
 }
 
 template <typename T, bool CFG, bool TAU1>
-__global__ void __launch_bounds__(ST, 4) verify_stream_kernel(const VerifyArgs a) {
+__global__ void __launch_bounds__(ST, LANTERN_STREAM_MINB) verify_stream_kernel(const VerifyArgs a) {
   grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char stream_smem[];
   constexpr int NOPS = CFG ? 4 : 2;

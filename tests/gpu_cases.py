@@ -24,7 +24,8 @@ class Case:
     """Inputs of one call (CPU tensors) and everything the oracle says about them."""
 
     def __init__(self, cfg, parent=None, seed=0, allowed=(0, 0), k_table=None, temperature=None,
-                 top_k_target=None, top_k_draft=None, pad=0, oracle_seqs=None, tokens="oracle", delta=0.0):
+                 top_k_target=None, top_k_draft=None, pad=0, oracle_seqs=None, tokens="oracle", delta=0.0,
+                 library_table=False):
         self.cfg = cfg
         self.parent = W.static_tree(cfg.n_nodes) if parent is None else parent
         N, B, V = len(self.parent), cfg.batch, cfg.vocab
@@ -62,6 +63,16 @@ class Case:
                 tok[b, 1:] = t[1:]
         self.tokens = tok
         self._orc = None
+        # library_table: the device side verifies with the table lantern_build_neighbors makes of
+        # the codebook; the oracle gets its own brute-force rows for the codes the checked
+        # sequences draft (the other rows are never read)
+        self.library_table = library_table
+        if library_table:
+            codes = sorted({int(t) - cfg.code_offset for b in self.seqs for t in tok[b, 1:]
+                            if 0 <= int(t) - cfg.code_offset < cfg.codebook_size})
+            rows, _ = oracle.neighbor_table(cb.to(torch.float64).numpy(), self.k_table, rows=codes)
+            self.nbr = np.zeros((cfg.codebook_size, self.k_table), dtype=np.int32)
+            self.nbr[codes] = rows
 
     def _sampler_kw(self):
         p = self.params
@@ -82,6 +93,21 @@ class Case:
                     **self.params))
         return self._orc
 
+    def oracle_node(self, b, n, forced):
+        """oracle.verify_node of node n of sequence b with decisions imposed (near-tie rule)."""
+        lg, p = self.logits, self.params
+        children = oracle.tree_children(self.parent)
+        row = lambda t: None if t is None else f64(t[b][n])
+        q, _ = oracle.postprocess_row(row(lg["target_cond"]), row(lg["target_uncond"]), p["cfg_scale"], p["temperature"],
+                                      p["top_k_target"], p["allowed_begin"], p["allowed_end"])
+        pd = None
+        if children[n]:
+            pd, _ = oracle.postprocess_row(row(lg["draft_cond"]), row(lg["draft_uncond"]), p["cfg_scale"],
+                                           p["temperature"], p["top_k_draft"], p["allowed_begin"], p["allowed_end"])
+        return oracle.verify_node(q, pd, children[n], self.tokens[b], self.u_accept[b].numpy(),
+                                  self.u_resample[b].numpy()[n], self.nbr, p["k"], p["lam"], p["code_offset"],
+                                  p["n_codes"], p["delta"], forced=forced)
+
     # ---- device side
     def gpu_inputs(self, L):
         dev = "cuda"
@@ -92,6 +118,8 @@ class Case:
                        code_offset=p["code_offset"], n_codes=p["n_codes"], allowed_begin=p["allowed_begin"],
                        allowed_end=p["allowed_end"], delta=p["delta"])
         nbr = None if self.nbr is None else torch.from_numpy(self.nbr).to(dev)
+        if self.library_table:
+            nbr = L.build_neighbors(self.codebook.to(dev), self.k_table)
         tok = torch.from_numpy(self.tokens.astype(np.int32)).to(dev)
         return g, par, nbr, tok
 

@@ -82,8 +82,14 @@ def test_config_codebooks_sampled_rows(L, n, d, k, dt):
     assert np.all(s[:, 1:] != s[:, :-1]) and idx.min() >= 0 and idx.max() < n
 
 
-def test_sweep_largest_shape_sampled_rows(L):
-    n, d, k = 65536, 64, 50
+@pytest.mark.parametrize("n,d,k", [(65536, 64, 50), (65536, 256, 200), (65536, 8, 200)])
+def test_sweep_largest_shapes_sampled_rows(L, n, d, k):
+    """The largest codebooks of the table sweep (bf16, 5 % duplicate rows): sampled rows against
+    the oracle, duplicates among them."""
     cb = W.make_codebook(n, d, "bf16", seed=6, dup_frac=0.05)
     rows = [0, n - 1] + list(np.random.default_rng(1).integers(0, n, 10))
+    # rows that have an exact copy elsewhere (zero distance, tie by index)
+    _, inv, cnt = np.unique(cb.view(torch.int16).numpy(), axis=0, return_inverse=True, return_counts=True)
+    dup_rows = np.nonzero(cnt[inv.ravel()] > 1)[0]
+    rows += [int(x) for x in dup_rows[:3]]
     _check(L, cb, k, rows=rows)

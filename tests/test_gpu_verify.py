@@ -22,8 +22,8 @@ def _run(L, case, **kw):
     assert res["status"] == 0
     orc = case.oracle_verify()
     ua = case.u_accept.numpy()
-    stats = compare_verify(res, orc, case.parent, ua, case.seqs)
-    check_walk(res, case.tokens, res["max_depth"], orc, stats["dirty_sequences"], case.seqs)
+    stats = compare_verify(res, orc, case.parent, ua, case.seqs, rerun=case.oracle_node)
+    check_walk(res, case.tokens, res["max_depth"], orc, stats["dirty_sequences"], case.seqs, stats["patched"])
     assert stats["tie_accept"] + stats["tie_cut"] + stats["tie_resample"] <= max(1, stats["nodes"] // 500)
     return res, stats
 
@@ -306,7 +306,7 @@ def test_invalid_arguments_are_rejected(L):
 def test_named_configs_full_size(L, name):
     case = Case(W.CONFIGS[name], seed=0)
     res, stats = _run(L, case)
-    print(name, {k: v for k, v in stats.items() if k != "dirty_sequences"})
+    print(name, {k: v for k, v in stats.items() if k not in ("dirty_sequences", "patched")})
 
 
 @pytest.mark.parametrize("name,seqs", [("c3_lumina", [0, 3]), ("c4_batch64", [0, 37, 63])])
@@ -319,4 +319,15 @@ def test_large_vocab_configs_sampled_sequences(L, name, seqs):
     assert np.all((nxt >= 0) != (tok >= 0))
     thr = res["node_thresh"]
     assert np.all((thr == -1) | ((thr >= 0) & (thr <= 1)))
-    print(name, {k: v for k, v in stats.items() if k != "dirty_sequences"})
+    print(name, {k: v for k, v in stats.items() if k not in ("dirty_sequences", "patched")})
+
+
+def test_lumina_shape_with_the_table_the_library_built(L):
+    """Config-3 shapes end to end: the verifier reads the neighbour table that
+    lantern_build_neighbors made of the 8192 x 256 bf16 codebook; the oracle uses its own
+    brute-force rows for the drafted codes."""
+    import dataclasses
+    cfg = dataclasses.replace(W.CONFIGS["c3_lumina"], batch=2)
+    case = Case(cfg, seed=4, library_table=True, allowed=(cfg.code_offset, cfg.code_offset + cfg.codebook_size))
+    res, stats = _run(L, case)
+    assert stats["tested"] > 50

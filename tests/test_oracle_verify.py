@@ -281,3 +281,24 @@ def test_identical_models_accept_the_first_child_chain():
     assert list(out["node_mass"][[0, 2, 4]]) == [-1, -1, -1]      # root and later siblings: never tested
     # emitted count = accepted + 1 (step-compression numerator, Sec. 5)
     assert len(out["out_tokens"]) == out["accept_len"] + 1
+
+
+def test_bound_is_strict_at_an_exact_tie():
+    """Sec. 4 displays the bound with "<": a neighbour whose mass brings the running sum exactly
+    to lambda * q(x) stays out (binary fractions, so the tie is exact in floating point), and
+    with lambda = 1 nothing can join."""
+    q = np.array([0.25, 0.25, 0.125, 0.125, 0.25])
+    nbr = np.array([[1, 2, 3, 4], [0, 2, 3, 4], [0, 1, 3, 4], [0, 1, 2, 4], [0, 1, 2, 3]])
+    m, members = oracle.relaxed_mass(q, 0, nbr, 4, 2.0, 0, 5)          # 0.25 + 0.25 == 2 * 0.25: stop
+    assert m == 0.25 and members == []
+    m, members = oracle.relaxed_mass(q, 2, nbr, 4, 3.0, 0, 5)          # bound 0.375: 0.125 + 0.25 == bound
+    assert m == 0.125 and members == []
+    m, members = oracle.relaxed_mass(q, 0, nbr, 4, 2.5, 0, 5)          # bound 0.625: one joins, 0.5 + 0.125 == bound stops
+    assert m == 0.5 and members == [1]
+    m, members = oracle.relaxed_mass(q, 0, nbr, 4, 1.0, 0, 5)
+    assert m == 0.25 and members == []
+    # additive variant (Sec. 2.2): the neighbours' own sum must stay strictly below delta
+    m, members = oracle.relaxed_mass(q, 0, nbr, 4, 1.0, 0, 5, delta=0.25)
+    assert m == 0.25 and members == []
+    m, members = oracle.relaxed_mass(q, 0, nbr, 4, 1.0, 0, 5, delta=0.375)
+    assert m == 0.5 and members == [1]
