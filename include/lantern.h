@@ -16,6 +16,10 @@
  *    OR-ed into *device_status as LANTERN_DEV_* bits; the kernels never trap.
  *  - Same inputs and same uniforms / seed give the same bytes.
  *  - Only lantern_tree_create allocates (a few hundred bytes per tree).
+ *  - Entry points may be called from several host threads at once as long as the calls do not
+ *    share output buffers or a workspace; lantern_set_cluster_size is the exception (see there).
+ *  - The neighbour table must not list a token among its own neighbours and a row's entries
+ *    must be distinct (lantern_build_neighbors guarantees both).
  */
 #ifndef LANTERN_H_
 #define LANTERN_H_
@@ -42,7 +46,8 @@ enum {
   LANTERN_DEV_BAD_INDEX = 1,    /* a token or neighbour index fell outside the vocabulary; it was
                                    treated as probability 0                                     */
   LANTERN_DEV_TIMEOUT = 2,      /* a bounded on-chip wait expired; the data was re-read with
-                                   plain loads                                                  */
+                                   plain loads and the CTA made no further asynchronous copies.
+                                   Never observed; treat the call's results as suspect          */
   LANTERN_DEV_EMPTY_ROW = 4,    /* a row had no finite logit                                    */
   LANTERN_DEV_KEY_TIES = 8      /* draft sampling: more Gumbel keys than the kernel ranks exactly
                                    lay within 2.5e-4 of the last child's key; the children are
@@ -181,14 +186,20 @@ lantern_status lantern_verify_tree(const lantern_params* params, const lantern_t
                                    void* stream);
 
 /* ---- which kernels a call launches ---------------------------------------------------------------
- * Rows that App. B's top-k truncation cuts to at most 1280 entries, in vocabularies of at most
- * 16384 tokens, are handled by list-based kernels (the row is compacted to its survivors; everything
- * after works on those), followed by a launch of the dense kernels that redoes the nodes whose
- * rows did not fit the lists' fixed buffers (massive ties; usually none).  All other calls run the
- * dense kernels alone.  Results are the same either way; these queries only tell which it will be
- * (lantern_verify_tree additionally needs its full workspace for the list path).
- * lantern_sample_draft_tree launches 1 (dense) or 2 (lists) kernels, lantern_verify_tree always 2
- * (dense + walk, or lists + repair launch that also walks).  Returns -1 on NULL arguments.       */
+ * Rows that no top-k truncates are handled by streaming kernels (LANTERN_PATH_STREAM): every row is
+ * read from HBM once and never held on chip; a rejection is one more read-only pass over the
+ * node's two rows, served by L2.  Rows that App. B's top-k truncation cuts to at most 1280 entries,
+ * in vocabularies of at most 16384 tokens, are handled by list-based kernels (LANTERN_PATH_LISTS:
+ * the row is compacted to its survivors; everything after works on those), followed by a launch of
+ * the dense kernels that redoes the nodes whose rows did not fit the lists' fixed buffers (massive
+ * ties; usually none).  All other calls (top-k on wide vocabularies, the path walk) run the dense
+ * kernels alone (LANTERN_PATH_DENSE: rows held in shared memory).  Results are the same either way;
+ * these queries only tell which it will be (lantern_verify_tree additionally needs its full
+ * workspace for the list path).
+ * Launches per call: lantern_sample_draft_tree 1 (streaming, dense) or 2 (lists + repair);
+ * lantern_verify_tree 2 (streaming + walk, dense + walk, or lists + repair launch that also
+ * walks), or 1 with params->lazy_walk (the path-walk kernel walks as it goes).  Returns -1 on NULL
+ * arguments.                                                                                      */
 #define LANTERN_PATH_DENSE 0
 #define LANTERN_PATH_LISTS 1
 #define LANTERN_PATH_STREAM 2
@@ -233,10 +244,14 @@ lantern_status lantern_verify_tree_static(const lantern_params* params, const la
 lantern_status lantern_philox_raw(uint64_t seed, uint32_t first, uint32_t c1, uint32_t c2,
                                   uint32_t c3, int32_t n, uint32_t* out, void* stream);
 
-/* Tuning knob, process-wide: number of CTAs a logit row is split over (a thread-block cluster),
- * 0 = choose automatically.  Returns the previous value.  Results do not depend on it beyond
- * float32 summation order.                                                                      */
+/* Tuning knob: number of CTAs a logit row is split over (a thread-block cluster), 0 = choose
+ * automatically; any value other than 0, 1, 2, 4, 8, 16 is ignored.  Returns the previous value.
+ * Results do not depend on it beyond float32 summation order.  The setting is one unsynchronised
+ * process-wide variable: it is not thread-safe, it applies to every later call of every thread on
+ * every device, and a non-zero value also makes top-k rows take the dense kernels.  Set it once at
+ * start-up, or not at all.                                                                       */
 int32_t lantern_set_cluster_size(int32_t ctas_per_row);
+int32_t lantern_get_cluster_size(void);      /* the current setting */
 
 #ifdef __cplusplus
 }

@@ -96,6 +96,8 @@ def _load():
                                      ctypes.c_uint32, i32, vp, vp]
     L.lantern_set_cluster_size.restype = i32
     L.lantern_set_cluster_size.argtypes = [i32]
+    L.lantern_get_cluster_size.restype = i32
+    L.lantern_get_cluster_size.argtypes = []
     L.lantern_verify_tree_path.restype = i32
     L.lantern_verify_tree_path.argtypes = [ctypes.POINTER(_CParams), vp]
     L.lantern_sample_draft_tree_path.restype = i32
@@ -276,7 +278,8 @@ def verify_tree_path(params: "Params", tree: "Tree") -> int:
 
 
 def sample_draft_tree_path(params: "Params") -> int:
-    """lantern_sample_draft_tree_path: 0 = dense kernel, 1 = list-based kernel + repair launch."""
+    """lantern_sample_draft_tree_path: 0 = dense kernel, 1 = list-based kernel + repair launch,
+    2 = streaming kernel (rows without top-k)."""
     cp = params.c()
     return lib.lantern_sample_draft_tree_path(ctypes.byref(cp))
 

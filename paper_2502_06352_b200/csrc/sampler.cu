@@ -417,13 +417,13 @@ static cudaError_t launch_sample_stream(const SampleArgs& a, int cs, bool f32, b
 
 using namespace lantern;
 
-extern "C" int32_t lantern_set_cluster_size(int32_t);
+extern "C" int32_t lantern_get_cluster_size(void);
 
 namespace {
 // Rows truncated to a moderate top-k can take the list-based kernel.
 bool sampler_uses_lists(const lantern_params* p) {
   const int V = p->vocab;
-  const int ov = lantern_set_cluster_size(-1);     // -1 is not a valid size: reads the current value
+  const int ov = lantern_get_cluster_size();
   return ov == 0 && V <= sparse::kMaxV && p->top_k_draft > 0 && p->top_k_draft < V && p->top_k_draft <= sparse::kMaxTopK;
 }
 }  // namespace
@@ -481,7 +481,7 @@ extern "C" lantern_status lantern_sample_draft_tree(
   a.repair = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = draft_uncond != nullptr;
-  const int ov = lantern_set_cluster_size(-1);     // -1 is not a valid size: reads the current value
+  const int ov = lantern_get_cluster_size();
   if (sampler_uses_stream(p)) {
     // CTAs per parent: one when the parents alone fill the machine
     int cs = ov;

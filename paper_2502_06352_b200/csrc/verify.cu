@@ -6,16 +6,15 @@
 namespace lantern {
 static int g_cluster_override = 0;
 static int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-      n = v;
-    else
-      return 148;
+  // per device: a process may drive GPUs of different sizes
+  static int cached[64] = {};
+  int dev = 0, v = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+    cached[dev] = v;
   }
-  return n;
+  return cached[dev];
 }
 }
 
@@ -133,6 +132,8 @@ extern "C" int32_t lantern_set_cluster_size(int32_t ctas_per_row) {
     g_cluster_override = ctas_per_row;
   return old;
 }
+
+extern "C" int32_t lantern_get_cluster_size(void) { return g_cluster_override; }
 
 namespace {
 constexpr int kWsTailInts = 64;

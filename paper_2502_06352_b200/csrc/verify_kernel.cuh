@@ -456,7 +456,7 @@ __device__ __forceinline__ void topk_thresholds(VCtx& c, const TopkSmem& s, cons
 template <typename T, bool CFG, int E>
 __device__ __forceinline__ int verify_node(const VerifyArgs& a, const int b, const int n, VCtx& c, const TopkSmem& tk,
                                             float* __restrict__ Q, float* __restrict__ P, float* __restrict__ U,
-                                            int* misc, const uint32_t mbar_a, uint32_t& mphase, int* nbr_s) {
+                                            int* misc, const uint32_t mbar_a, uint32_t& mphase, bool& bulk_ok, int* nbr_s) {
   constexpr int SL = VT * E;
   constexpr int NV4 = E / 4;                 // float4 per thread in a shared-memory sweep
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -472,7 +472,7 @@ __device__ __forceinline__ int verify_node(const VerifyArgs& a, const int b, con
   // ---- stage the children's neighbour rows (bulk async copy when rows are 16-byte aligned)
   const bool want_nbr = nc > 0 && a.k > 0;
   bool bulk_issued = false;
-  if (want_nbr && a.use_bulk) {
+  if (want_nbr && a.use_bulk && bulk_ok) {
     if (tid == 0) {
       uint32_t bytes = 0;
       const uint32_t row_bytes = static_cast<uint32_t>(((a.k + 3) & ~3) * 4);
@@ -602,9 +602,16 @@ __device__ __forceinline__ int verify_node(const VerifyArgs& a, const int b, con
 
   // ---- neighbour rows must have landed
   if (bulk_issued) {
-    bool ok = mbar_wait_bounded(mbar_a, mphase);
-    mphase ^= 1u;
-    if (!__syncthreads_and(ok)) {
+    const bool ok = mbar_wait_bounded(mbar_a, mphase);
+    if (__syncthreads_and(ok)) {
+      mphase ^= 1u;
+    } else {
+      // The copy did not complete in time: the barrier's phase is still pending, so the barrier
+      // is not touched again and this CTA stages every later table row with plain loads.  For
+      // this node a late arrival writes the values that are re-read below anyway; if the CTA
+      // goes on to other nodes (repair launch, path walk) a copy arriving that late could still
+      // overwrite their rows, which is why the status bit is raised.
+      bulk_ok = false;
       if (tid == 0) vflag(a.status, LANTERN_DEV_TIMEOUT);
       for (int ci = 0; ci < nc; ++ci) {
         int code = tok_b[fc + ci] - a.code_offset;
@@ -708,11 +715,11 @@ __device__ __forceinline__ int verify_node(const VerifyArgs& a, const int b, con
     }
     // ---- rejection: q~ (mass of A moved onto x), residual, drafter without x
     if (!single) cluster_sync();     // every CTA has finished reading q_cur / p_cur of this round
+    const int xl = x - lo;                                   // position of x in this slice, if any
     for (int r = tid; r < nA; r += VT) {
       const int t = a.code_offset + nrow[r] - lo;
-      if (t >= 0 && t < len) Q[t] = 0.f;
+      if (t >= 0 && t < len && t != xl) Q[t] = 0.f;          // (a row that lists x itself: x is written below)
     }
-    const int xl = x - lo;                                   // position of x in this slice, if any
     if (tid == 0 && xl >= 0 && xl < len) Q[xl] = qs > 0.f ? m / qs : 0.f;
     __syncthreads();
     // One sweep: Q <- [Q * rho - P]_+ with rho = qs * psum, i.e. the residual of Eq. 2 in the
@@ -893,6 +900,7 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   uint32_t mphase = 0;
+  bool bulk_ok = true;        // false after a bounded wait on the table-row copy has expired
   // A regular launch has one CTA (cluster) per node.  A repair launch (a.only given) has fewer:
   // cluster g of G takes the flagged nodes idx = g (mod G) one after another, and leaves at once
   // when none of them is flagged.
@@ -907,7 +915,7 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
     int32_t* on = a.out_nodes + static_cast<long long>(b) * a.D1;
     int cur = 0, len = 0;
     for (;;) {
-      const int acc = verify_node<T, CFG, E>(a, b, cur, c, tk, Q, P, U, misc, mbar_a, mphase, nbr_s);
+      const int acc = verify_node<T, CFG, E>(a, b, cur, c, tk, Q, P, U, misc, mbar_a, mphase, bulk_ok, nbr_s);
       csync(c);     // also orders the owner CTA's store of node_token before the read below
       if (acc <= cur || acc >= a.N || len >= a.D1 - 1) break;      // -1, or anything that is not a forward edge
       cur = acc;
@@ -932,7 +940,7 @@ __global__ void __launch_bounds__(VT, LANTERN_MINB) verify_nodes_kernel(const Ve
   if (work) {
     for (int idx = g0; idx < rows; idx += G) {
       if (a.only && a.only[idx] == 0) continue;
-      verify_node<T, CFG, E>(a, idx % a.B, a.order[idx / a.B], c, tk, Q, P, U, misc, mbar_a, mphase, nbr_s);
+      verify_node<T, CFG, E>(a, idx % a.B, a.order[idx / a.B], c, tk, Q, P, U, misc, mbar_a, mphase, bulk_ok, nbr_s);
       csync(c);     // peers may still be reading this CTA's shared memory; the next node overwrites it
     }
   }
