@@ -38,6 +38,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c4_batch64")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (sequences per call); 0 = as configured")
     ap.add_argument("--ring", type=int, default=0, help="input buffer sets cycled through (0 = enough to exceed L2)")
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--configs", default="all", choices=["all", "none"],
@@ -494,6 +495,8 @@ def main():
         run_table_sweep(args)
         return
     cfg = W.CONFIGS[args.workload]
+    if args.batch > 0:
+        cfg = dataclasses.replace(cfg, batch=args.batch)
     parent = W.static_tree(cfg.n_nodes)
     if args.impl == "reference":
         run_reference(args, cfg, parent)
@@ -653,7 +656,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": warm,
             "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": cfg.dtype, "data": "synthetic",
-            "config": {"workload": cfg.name, "batch_per_gpu": B, "tree_nodes": N, "vocab": V, "logits": cfg.dtype,
+            "config": {"workload": cfg.name + ("" if args.batch <= 0 else " (batch overridden)"), "batch_per_gpu": B, "tree_nodes": N, "vocab": V, "logits": cfg.dtype,
                        "arithmetic": "f32 (exact re-ranking steps in f64)",
                        "cfg_scale": cfg.cfg_scale, "top_k": cfg.top_k, "neighbours_k": cfg.k, "lambda": cfg.lam,
                        "codebook": [cfg.codebook_size, cfg.codebook_dim], "parallelism": "dp%d" % world,

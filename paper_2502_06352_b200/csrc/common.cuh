@@ -125,6 +125,24 @@ __host__ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t 
   }
   return Philox4{c0, c1, c2, c3};
 }
+// The same generator with the ten round keys k + r * W precomputed (kernel arguments: they feed
+// the xor straight from the constant bank, so a round is two wide multiplies and two xors).
+__device__ __forceinline__ Philox4 philox4x32_10_keys(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                      const uint32_t (&rk0)[10], const uint32_t (&rk1)[10]) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = static_cast<uint64_t>(M0) * c0;
+    const uint64_t p1 = static_cast<uint64_t>(M1) * c2;
+    const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ rk0[r];
+    const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ rk1[r];
+    c1 = static_cast<uint32_t>(p1);
+    c3 = static_cast<uint32_t>(p0);
+    c0 = n0;
+    c2 = n2;
+  }
+  return Philox4{c0, c1, c2, c3};
+}
 enum { kStreamGumbel = 0, kStreamAccept = 1, kStreamResample = 2 };
 // counter = (block, row, step_lo, step_hi << 2 | stream), key = seed
 __device__ __forceinline__ Philox4 philox_stream(uint64_t seed, uint64_t step, uint32_t row,

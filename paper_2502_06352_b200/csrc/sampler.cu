@@ -30,6 +30,7 @@ struct SampleArgs {
   int32_t* status;
   int n_parents;       // parents per sequence in this launch
   int repair;          // non-zero: draw only the parents whose first child's token is the redo marker
+  uint32_t rk0[10], rk1[10];   // Philox round keys of `seed`
 };
 
 }  // namespace lantern
@@ -479,6 +480,10 @@ extern "C" lantern_status lantern_sample_draft_tree(
   a.tokens = tokens; a.draft_prob = draft_prob; a.status = device_status;
   a.n_parents = i1 - i0;
   a.repair = 0;
+  for (int r = 0; r < 10; ++r) {
+    a.rk0[r] = static_cast<uint32_t>(p->seed) + static_cast<uint32_t>(r) * 0x9E3779B9u;
+    a.rk1[r] = static_cast<uint32_t>(p->seed >> 32) + static_cast<uint32_t>(r) * 0xBB67AE85u;
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = draft_uncond != nullptr;
   const int ov = lantern_get_cluster_size();

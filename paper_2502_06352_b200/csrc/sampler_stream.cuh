@@ -158,81 +158,107 @@ __global__ void __launch_bounds__(ST, 4) sample_stream_kernel(const SampleArgs a
   if (tid == 0) *s.cnt = 0;
   __syncthreads();
 
-  auto uniforms = [&](int j, float (&U)[VN]) {        // uniforms of tokens j .. j+VN-1 (j a multiple of VN)
+  // Uniforms of tokens j .. j+VN-1 (j a multiple of VN); returns whether one of them exceeds 0.999.
+  // Philox words become floats without an integer conversion: the 23 mantissa bits under the
+  // exponent of 1.0 give 1 + i 2^-23, and subtracting 1 - 2^-24 leaves (i + 1/2) 2^-23 exactly.
+  auto uniforms = [&](int j, float (&U)[VN]) -> bool {
+    bool near_one = false;
     if (gum) {
 #pragma unroll
-      for (int e = 0; e < VN; ++e) U[e] = (j + e < a.V) ? __ldcs(gum + j + e) : 0.5f;
+      for (int e = 0; e < VN; ++e) {
+        U[e] = (j + e < a.V) ? __ldcs(gum + j + e) : 0.5f;
+        near_one |= U[e] > 0.999f;
+      }
     } else {
 #pragma unroll
       for (int q = 0; q < VN / 4; ++q) {
-        const Philox4 r = philox_stream(a.seed, a.step, row_id, kStreamGumbel, static_cast<uint32_t>((j >> 2) + q));
-        U[4 * q] = uniform_open(r.x); U[4 * q + 1] = uniform_open(r.y);
-        U[4 * q + 2] = uniform_open(r.z); U[4 * q + 3] = uniform_open(r.w);
+        const Philox4 r = philox4x32_10_keys(static_cast<uint32_t>((j >> 2) + q), row_id, static_cast<uint32_t>(a.step),
+                                             (static_cast<uint32_t>(a.step >> 32) << 2) | kStreamGumbel, a.rk0, a.rk1);
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          U[4 * q + e] = __uint_as_float(0x3f800000u | (w[e] >> 9)) - 0.99999994f;
+        near_one |= (max(max(r.x, r.y), max(r.z, r.w)) >> 9) > 8380219u;       // 0.999 * 2^23
       }
     }
+    return near_one;
   };
 
+  // Optimistic pass: after the first cut the threshold is high and appends are rare, so the
+  // remaining chunks run without barriers or further cuts; if the list overflows all the same
+  // (keys that keep growing along the row), the row is redone with a check after every chunk.
   float Tk = -INFINITY;                               // every element left out has key <= Tk
   float mx = -INFINITY, sx = 0.f;
   const int iters = (ge.vw + 32 * UV - 1) / (32 * UV);
-  for (int it = 0; it < iters; ++it) {
-    const int base = vbeg + it * 32 * UV;
-    uint4 rc[UV], ru[UV];
+  for (int mode = 0; mode < 2; ++mode) {
+    Tk = -INFINITY;
+    mx = -INFINITY;
+    sx = 0.f;
+    for (int it = 0; it < iters; ++it) {
+      const int base = vbeg + it * 32 * UV;
+      uint4 rc[UV], ru[UV];
 #pragma unroll
-    for (int u = 0; u < UV; ++u) {
-      const int vv = base + 32 * u + lane;
-      if (vv < vend && vv >= ge.vi0 && vv < ge.vi1) io.load(vv, rc[u], ru[u]);
-    }
-#pragma unroll
-    for (int u = 0; u < UV; ++u) {
-      const int vv = base + 32 * u + lane;
-      const bool active = vv < vend;
-      const int j = ge.j0 + vv * VN;
-      float z[VN], key[VN];
-      bool any = false;
-      if (active) {
-        if (vv >= ge.vi0 && vv < ge.vi1) {
-          io.z(rc[u], ru[u], z);
-        } else {                                      // ragged first / last vector of the row
-#pragma unroll
-          for (int e = 0; e < VN; ++e) z[e] = (j + e >= ge.alo && j + e < ge.ahi) ? io.z_at(j + e) : -INFINITY;
-        }
-        float U[VN];
-        uniforms(j, U);
-        bool near_one = false;
-#pragma unroll
-        for (int e = 0; e < VN; ++e) {
-          key[e] = fast_key(z[e], U[e]);
-          near_one |= U[e] > 0.999f;
-        }
-        if (near_one) {                               // rare: one vector in a hundred
-#pragma unroll
-          for (int e = 0; e < VN; ++e)
-            if (U[e] > 0.999f) key[e] = careful_key(z[e], U[e]);
-        }
-#pragma unroll
-        for (int e = 0; e < VN; ++e) any |= key[e] > Tk;
-        if (want_prob) acc_exp<VN>(z, mx, sx);
+      for (int u = 0; u < UV; ++u) {
+        const int vv = base + 32 * u + lane;
+        if (vv < vend && vv >= ge.vi0 && vv < ge.vi1) io.load(vv, rc[u], ru[u]);
       }
-      if (__any_sync(0xffffffffu, any)) {
 #pragma unroll
-        for (int e = 0; e < VN; ++e) {
-          const bool take = active && key[e] > Tk;
-          const uint32_t m = __ballot_sync(0xffffffffu, take);
-          if (m) {
-            int pos0 = 0;
-            if (lane == 0) pos0 = atomicAdd(s.cnt, __popc(m));
-            pos0 = __shfl_sync(0xffffffffu, pos0, 0);
-            const int pos = pos0 + __popc(m & ((1u << lane) - 1u));
-            if (take && pos < kListCap) s.list[pos] = make_uint2(__float_as_uint(key[e]), static_cast<uint32_t>(j + e));
+      for (int u = 0; u < UV; ++u) {
+        const int vv = base + 32 * u + lane;
+        const bool active = vv < vend;
+        const int j = ge.j0 + vv * VN;
+        float z[VN], key[VN];
+        bool any = false;
+        if (active) {
+          if (vv >= ge.vi0 && vv < ge.vi1) {
+            io.z(rc[u], ru[u], z);
+          } else {                                      // ragged first / last vector of the row
+#pragma unroll
+            for (int e = 0; e < VN; ++e) z[e] = (j + e >= ge.alo && j + e < ge.ahi) ? io.z_at(j + e) : -INFINITY;
+          }
+          float U[VN];
+          const bool near_one = uniforms(j, U);
+#pragma unroll
+          for (int e = 0; e < VN; ++e) key[e] = fast_key(z[e], U[e]);
+          if (near_one) {                               // rare: one vector in a hundred
+#pragma unroll
+            for (int e = 0; e < VN; ++e)
+              if (U[e] > 0.999f) key[e] = careful_key(z[e], U[e]);
+          }
+          float best = key[0];
+#pragma unroll
+          for (int e = 1; e < VN; ++e) best = fmaxf(best, key[e]);
+          any = best > Tk;
+          if (want_prob) acc_exp<VN>(z, mx, sx);
+        }
+        if (__any_sync(0xffffffffu, any)) {
+#pragma unroll
+          for (int e = 0; e < VN; ++e) {
+            const bool take = active && key[e] > Tk;
+            const uint32_t m = __ballot_sync(0xffffffffu, take);
+            if (m) {
+              int pos0 = 0;
+              if (lane == 0) pos0 = atomicAdd(s.cnt, __popc(m));
+              pos0 = __shfl_sync(0xffffffffu, pos0, 0);
+              const int pos = pos0 + __popc(m & ((1u << lane) - 1u));
+              if (take && pos < kListCap) s.list[pos] = make_uint2(__float_as_uint(key[e]), static_cast<uint32_t>(j + e));
+            }
           }
         }
       }
+      if (it == 0 || mode == 1) {
+        __syncthreads();
+        const bool full = *s.cnt > kListCap - kIterElems;
+        __syncthreads();                                // everyone has read the count before it moves again
+        if (full) Tk = cut_list(s, R, Tk);
+      }
     }
     __syncthreads();
-    const bool full = *s.cnt > kListCap - kIterElems;
-    __syncthreads();                                  // everyone has read the count before it moves again
-    if (full) Tk = cut_list(s, R, Tk);
+    const bool overflow = *s.cnt > kListCap;
+    if (!overflow) break;
+    __syncthreads();                                    // (mode 1 never overflows: it cuts in time)
+    if (tid == 0) *s.cnt = 0;
+    __syncthreads();
   }
 
   // ---- softmax denominator of the row (for draft_prob)
