@@ -25,7 +25,8 @@ from .postprocess import postprocess_row
 from .tree import tree_children
 
 
-def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None, delta=0.0, force_members=None):
+def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None, delta=0.0, force_members=None,
+                 skip=False):
     """Sec. 4: m = sum of q over A_{k,lambda}(x) and the members of A besides x.
     With delta > 0 the additive bound of Sec. 2.2 replaces the multiplicative one:
     the neighbours' own running sum stays below delta (A_{k,delta}); lam is unused.
@@ -34,7 +35,10 @@ def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None, 
     appended to it (diagnostic for near-tie accounting; no effect on the result).
     `force_members` (diagnostic, used only when a comparison with another
     implementation continues past a near-tie): take exactly that many list entries
-    instead of applying the bound."""
+    instead of applying the bound.
+    `skip` selects the other reading of "a subset of B_k that satisfies the bound"
+    (Sec. 4 gives only the inequality): a neighbour that would break the bound is
+    passed over and the list is searched on, instead of ending the search."""
     cum = q_cur[x]
     bound = q_cur[x] + delta if delta > 0 else lam * q_cur[x]
     members = []
@@ -48,7 +52,7 @@ def relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins=None, 
             if take:
                 cum = cum + q_cur[a]
                 members.append(a)
-            else:
+            elif not skip or force_members is not None:
                 break
     return cum, members
 
@@ -62,8 +66,14 @@ def moved_mass(q_cur, x, m, members):
     return q_t
 
 
-def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset, n_codes, delta=0.0, forced=None):
+def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset, n_codes, delta=0.0, forced=None,
+                 skip=False, det_draft=False):
     """Test the children of one node in stored order (Sec. 4; App. A.2 Eq. 1-2).
+
+    `skip`: greedy-skip reading of the subset (see relaxed_mass).
+    `det_draft`: the draft tokens were chosen deterministically (Sec. 3, what dynamic-tree
+    drafting does): the drafter puts probability 1 on each of them, so the accept probability
+    is min(1, m) = m, p is not used, and the residual after a rejection is q~ without x.
 
     `forced` (diagnostic): {child: {"accept": bool, "n_members": int}} overrides the
     accept decision and / or the size of A of that child, so that a comparison can go
@@ -73,7 +83,7 @@ def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset
     is the target distribution left after the rejections (q itself at a leaf);
     cut_margin is the smallest |running sum - bound| met while forming A."""
     q_cur = np.array(q, dtype=np.float64)
-    p_cur = None if p is None else np.array(p, dtype=np.float64)
+    p_cur = None if (p is None or det_draft) else np.array(p, dtype=np.float64)
     tested = {}
     for c in child_ids:
         x = int(tokens[c])
@@ -82,8 +92,10 @@ def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset
         margins = []
         f = (forced or {}).get(c, {})
         m, members = relaxed_mass(q_cur, x, nbr_idx, k, lam, code_offset, n_codes, margins, delta,
-                                  force_members=f.get("n_members"))
-        if p_cur[x] > 0:
+                                  force_members=f.get("n_members"), skip=skip)
+        if det_draft:
+            thr = min(1.0, m)                     # Sec. 3: p(x) = 1
+        elif p_cur[x] > 0:
             thr = min(1.0, m / p_cur[x])          # Sec. 4, final accept probability
         else:
             thr = 1.0 if m > 0 else 0.0
@@ -94,6 +106,12 @@ def sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam, code_offset
         if accept:
             return c, q_cur, tested
         q_t = moved_mass(q_cur, x, m, members)
+        if det_draft:
+            r = q_t.copy()                         # Eq. 2 with p = the point mass at x
+            r[x] = max(m - 1.0, 0.0)
+            Z = r.sum()
+            q_cur = r / Z if Z > 0 else q_t
+            continue
         r = np.maximum(q_t - p_cur, 0.0)           # Eq. 2
         Z = r.sum()
         q_cur = r / Z if Z > 0 else q_t
@@ -116,7 +134,7 @@ def inverse_cdf(dist, u, return_margin=False):
 
 
 def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
-                code_offset, n_codes, delta=0.0, forced=None):
+                code_offset, n_codes, delta=0.0, forced=None, skip=False, det_draft=False):
     """Process one tree node.
 
     q: target distribution of the node; p: drafter distribution (None at a leaf)
@@ -126,7 +144,7 @@ def verify_node(q, p, child_ids, tokens, u_accept, u_resample, nbr_idx, k, lam,
     tested["resample_margin"] is set when a token was drawn.
     """
     nxt, q_cur, tested = sibling_loop(q, p, child_ids, tokens, u_accept, nbr_idx, k, lam,
-                                      code_offset, n_codes, delta, forced)
+                                      code_offset, n_codes, delta, forced, skip, det_draft)
     if nxt >= 0:
         return nxt, -1, tested
     j, margin = inverse_cdf(q_cur, u_resample, return_margin=True)
@@ -153,7 +171,7 @@ def walk(node_next, node_token, tokens):
 def verify_sequence(parent, target_cond, target_uncond, draft_cond, draft_uncond, tokens,
                     u_accept, u_resample, nbr_idx, *, cfg_scale=1.0, temperature=1.0,
                     top_k_target=0, top_k_draft=0, lam=1.0, k=0, code_offset=0, n_codes=0,
-                    allowed_begin=0, allowed_end=None, delta=0.0):
+                    allowed_begin=0, allowed_end=None, delta=0.0, skip=False, det_draft=False):
     """Verify one sequence's tree.  Logit arrays are [N][V]; uncond may be None.
 
     Returns a dict with node_next, node_token (int arrays [N]), node_mass,
@@ -172,11 +190,11 @@ def verify_sequence(parent, target_cond, target_uncond, draft_cond, draft_uncond
         q, _ = postprocess_row(target_cond[n], None if target_uncond is None else target_uncond[n],
                                cfg_scale, temperature, top_k_target, allowed_begin, allowed_end)
         p = None
-        if children[n]:
+        if children[n] and not det_draft:
             p, _ = postprocess_row(draft_cond[n], None if draft_uncond is None else draft_uncond[n],
                                    cfg_scale, temperature, top_k_draft, allowed_begin, allowed_end)
         nxt, tok, tested = verify_node(q, p, children[n], tokens, u_accept, u_resample[n],
-                                       nbr_idx, k, lam, code_offset, n_codes, delta)
+                                       nbr_idx, k, lam, code_offset, n_codes, delta, skip=skip, det_draft=det_draft)
         node_next[n], node_token[n] = nxt, tok
         resample_margin[n] = tested.pop("resample_margin", np.inf)
         for c, (m, thr, cm, _) in tested.items():
@@ -194,6 +212,6 @@ def verify_batch(parent, target_cond, target_uncond, draft_cond, draft_uncond, t
     for b in range(len(tokens)):
         out.append(verify_sequence(
             parent, target_cond[b], None if target_uncond is None else target_uncond[b],
-            draft_cond[b], None if draft_uncond is None else draft_uncond[b],
+            None if draft_cond is None else draft_cond[b], None if draft_uncond is None else draft_uncond[b],
             tokens[b], u_accept[b], u_resample[b], nbr_idx, **params))
     return out

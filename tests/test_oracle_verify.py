@@ -302,3 +302,65 @@ def test_bound_is_strict_at_an_exact_tie():
     assert m == 0.25 and members == []
     m, members = oracle.relaxed_mass(q, 0, nbr, 4, 1.0, 0, 5, delta=0.375)
     assert m == 0.5 and members == [1]
+
+
+def test_greedy_skip_subset():
+    """The other reading of Sec. 4's subset: a neighbour that would break the bound is passed
+    over.  Checked through the defining property (r joins iff the sum of x and of the earlier
+    members plus q(r) stays below the bound), not through the loop that builds it."""
+    rng = np.random.default_rng(11)
+    V, k = 32, 12
+    nbr = _table(rng, V, k)
+    differs = 0
+    for trial in range(300):
+        q, _ = _dists(rng, V, conc=0.3)
+        lam = float(rng.choice([1.0, 1.5, 2.0, 3.0]))
+        x = int(rng.integers(V))
+        m, members = oracle.relaxed_mass(q, x, nbr, k, lam, 0, V, skip=True)
+        m0, prefix = oracle.relaxed_mass(q, x, nbr, k, lam, 0, V)
+        assert members[: len(prefix)] == prefix and m >= m0           # the prefix comes first
+        assert m < lam * q[x] or (members == [] and m == q[x])
+        assert np.isclose(m, q[x] + sum(q[a] for a in members), rtol=1e-14)
+        inside = set(members)
+        run = q[x]
+        for a in (int(t) for t in nbr[x][:k]):
+            fits = run + q[a] < lam * q[x]
+            assert fits == (a in inside)
+            if fits:
+                run += q[a]
+        differs += members != prefix
+    assert differs > 20          # the two readings really differ on these inputs
+
+
+def test_deterministic_draft_mode():
+    """Sec. 3: a deterministically chosen draft has p(x) = 1, so it is accepted with probability
+    m (= q(x) without relaxation), and the emitted token still follows q exactly when k = 0,
+    whatever the drafts are: enumerate the sibling loop for s = 1, 2, 3."""
+    rng = np.random.default_rng(12)
+    V = 9
+    nbr = _table(rng, V, 4)
+    for trial in range(20):
+        q, _ = _dists(rng, V, conc=0.6)
+        for s in (1, 2, 3):
+            xs = [int(t) for t in rng.choice(V, size=s, replace=False)]
+            tokens = [0] + xs
+            kids = list(range(1, s + 1))
+            # thresholds met along the all-reject path, and the distribution left at its end
+            _, q_fin, tested = oracle.sibling_loop(q, None, kids, tokens, [0.0] + [1.0] * s, nbr, 0, 3.0, 0, V,
+                                                   det_draft=True)
+            law = np.zeros(V)
+            reach = 1.0
+            for c in kids:
+                m, thr = tested[c][:2]
+                assert thr == m
+                law[tokens[c]] += reach * thr
+                reach *= 1.0 - thr
+            law += reach * q_fin
+            assert np.allclose(law, q, atol=1e-14)
+            m1 = tested[1][0]
+            assert m1 == q[xs[0]]
+        # with relaxation the accept probability is the relaxed mass, within the bound
+        x = int(rng.integers(V))
+        _, _, tested = oracle.sibling_loop(q, None, [1], [0, x], [0.0, 1.0], nbr, 4, 2.0, 0, V, det_draft=True)
+        m, thr = tested[1][:2]
+        assert thr == min(1.0, m) and q[x] <= m and (m < 2.0 * q[x] or m == q[x])
