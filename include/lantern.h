@@ -101,7 +101,18 @@ typedef struct {
                               the accepted child and so on, reading only the rows on the accepted
                               path; accept_len / out_tokens / out_nodes are the same, the per-node
                               outputs are written for the nodes on the path only                */
+  int32_t subset_rule;     /* which subset of the neighbour list forms A (Sec. 4 states only the
+                              inequality).  0: the longest prefix of the distance-ordered list that
+                              keeps the bound.  1: greedy skip: a neighbour that would break the
+                              bound is passed over and the search goes on down the list           */
+  int32_t draft_deterministic; /* lantern_verify_tree only.  1: the draft tokens were chosen
+                              deterministically (Sec. 3: what dynamic-tree drafting does), i.e.
+                              p(x) = 1 for each of them: a child is accepted with probability
+                              min(1, m), the residual after a rejection is q~ without x, and the
+                              drafter rows are never read (draft_* may be NULL)                   */
 } lantern_params;
+/* subset_rule = 1 and draft_deterministic = 1 are served by the streaming kernels only: rows that a
+ * top-k truncates return LANTERN_ERR_UNSUPPORTED with either of them.                              */
 
 /* ---- (1) latent-neighbour table -------------------------------------------------------------
  * Sec. 2.2 / Sec. 4: B_k(x) = the k nearest neighbours of codebook vector c_x (App. A.1:

@@ -31,6 +31,7 @@ class _CParams(ctypes.Structure):
         ("allowed_begin", ctypes.c_int32), ("allowed_end", ctypes.c_int32),
         ("seed", ctypes.c_uint64), ("step", ctypes.c_uint64),
         ("delta", ctypes.c_float), ("lazy_walk", ctypes.c_int32),
+        ("subset_rule", ctypes.c_int32), ("draft_deterministic", ctypes.c_int32),
     ]
 
 
@@ -52,11 +53,14 @@ class Params:
     step: int = 0
     delta: float = 0.0
     lazy_walk: int = 0
+    subset_rule: int = 0
+    draft_deterministic: int = 0
 
     def c(self):
         return _CParams(self.cfg_scale, self.temperature, self.top_k_target, self.top_k_draft,
                         self.lam, self.k, self.vocab, self.code_offset, self.n_codes,
-                        self.allowed_begin, self.allowed_end, self.seed, self.step, self.delta, self.lazy_walk)
+                        self.allowed_begin, self.allowed_end, self.seed, self.step, self.delta, self.lazy_walk,
+                        self.subset_rule, self.draft_deterministic)
 
 
 def _load():

@@ -183,6 +183,7 @@ struct VerifyArgs {
   const int32_t *first_child, *n_child, *order;
   int B, N, V, kpad, n_internal, max_children;
   float g, inv_tau, lambda, delta;
+  int skip, det;           // greedy-skip subset rule; deterministic drafts (p(x) = 1, no drafter rows)
   int topk_t, topk_d, k, code_offset, n_codes, allow_lo, allow_hi;
   unsigned long long seed, step;
   int32_t *node_next, *node_token;

@@ -62,16 +62,22 @@ static cudaError_t launch_sparse_any(const VerifyArgs& a, int32_t* redo, int e, 
 }
 
 // ---- launch of the streaming kernel (rows without top-k): one CTA, or a cluster of cs CTAs, per node
-template <typename T, bool CFG, bool TAU1>
-static cudaError_t launch_stream_t(const VerifyArgs& a, int cs, size_t smem, cudaStream_t st) {
-  auto kern = stream::verify_stream_kernel<T, CFG, TAU1>;
+template <typename T, bool CFG, bool TAU1, bool GENERAL>
+static cudaError_t launch_stream_k(const VerifyArgs& a, int cs, size_t smem, cudaStream_t st) {
+  auto kern = stream::verify_stream_kernel<T, CFG, TAU1, GENERAL>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
   if (cs > 8) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
   }
-  return launch_after_previous(kern, static_cast<unsigned>(a.B) * a.N * cs, stream::ST, smem, st, cs, a);
+  const unsigned clusters = a.lazy ? static_cast<unsigned>(a.B) : static_cast<unsigned>(a.B) * a.N;
+  return launch_after_previous(kern, clusters * cs, stream::ST, smem, st, cs, a);
+}
+template <typename T, bool CFG, bool TAU1>
+static cudaError_t launch_stream_t(const VerifyArgs& a, int cs, size_t smem, cudaStream_t st) {
+  return (a.lazy || a.skip || a.det) ? launch_stream_k<T, CFG, TAU1, true>(a, cs, smem, st)
+                                     : launch_stream_k<T, CFG, TAU1, false>(a, cs, smem, st);
 }
 static cudaError_t launch_stream_any(const VerifyArgs& a, int cs, size_t smem, bool f32, bool cfg, cudaStream_t st) {
   const bool tau1 = a.inv_tau == 1.0f;
@@ -141,17 +147,17 @@ constexpr int kWsTailInts = 64;
 bool verify_uses_lists(const lantern_params* p, const TreeDev* t) {
   const int V = p->vocab;
   auto topk_fits = [&](int k) { return k > 0 && k < V && k <= sparse::kMaxTopK; };
-  return !p->lazy_walk && g_cluster_override == 0 && V <= sparse::kMaxV && topk_fits(p->top_k_target) &&
+  return !p->lazy_walk && !p->subset_rule && !p->draft_deterministic && g_cluster_override == 0 &&
+         V <= sparse::kMaxV && topk_fits(p->top_k_target) &&
          (t->n_internal == 0 || topk_fits(p->top_k_draft)) && t->max_children <= 8;
 }
-// Rows that no top-k truncates take the streaming kernel (unless the path walk is asked for).
+// Rows that no top-k truncates take the streaming kernel.
 bool verify_uses_stream(const lantern_params* p, const TreeDev* t) {
   const int V = p->vocab;
   const bool tk_t = p->top_k_target > 0 && p->top_k_target < V;
-  const bool tk_d = t->n_internal > 0 && p->top_k_draft > 0 && p->top_k_draft < V;
-  const bool cfg4 = true;      // the larger layout decides
-  return !p->lazy_walk && !tk_t && !tk_d && V <= stream::kMaxV &&
-         stream::smem_bytes(V, t->max_children, p->k + 1, cfg4) <= 227 * 1024;
+  const bool tk_d = t->n_internal > 0 && !p->draft_deterministic && p->top_k_draft > 0 && p->top_k_draft < V;
+  return !tk_t && !tk_d && V <= stream::kMaxV &&
+         stream::smem_bytes(V, t->max_children, p->k + 1, true) <= 227 * 1024;
 }
 }  // namespace
 
@@ -181,8 +187,11 @@ extern "C" lantern_status lantern_verify_tree(
   const TreeDev* t = reinterpret_cast<const TreeDev*>(tree);
   if (batch <= 0 || p->vocab <= 0 || !(p->temperature > 0.f) || !(p->lambda >= 1.f)) return LANTERN_ERR_INVALID_ARG;
   if (dt != LANTERN_F32 && dt != LANTERN_BF16) return LANTERN_ERR_INVALID_ARG;
-  if (t->n_internal > 0 && !draft_cond) return LANTERN_ERR_INVALID_ARG;
-  if ((target_uncond != nullptr) != (draft_uncond != nullptr) && t->n_internal > 0) return LANTERN_ERR_INVALID_ARG;
+  const bool det = p->draft_deterministic != 0;
+  if (p->subset_rule != 0 && p->subset_rule != 1) return LANTERN_ERR_INVALID_ARG;
+  if (t->n_internal > 0 && !draft_cond && !det) return LANTERN_ERR_INVALID_ARG;
+  if ((target_uncond != nullptr) != (draft_uncond != nullptr) && t->n_internal > 0 && !det) return LANTERN_ERR_INVALID_ARG;
+  if ((det || p->subset_rule) && !verify_uses_stream(p, t)) return LANTERN_ERR_UNSUPPORTED;
   if (p->k < 0 || p->top_k_target < 0 || p->top_k_draft < 0) return LANTERN_ERR_INVALID_ARG;
   if (!(p->delta >= 0.f) || p->delta > 4.f) return LANTERN_ERR_INVALID_ARG;      // also rejects NaN
   if (p->k > 0 && (!nbr_idx || p->k > k_table || p->n_codes <= 0 || k_table > p->n_codes - 1)) return LANTERN_ERR_INVALID_ARG;
@@ -221,6 +230,7 @@ extern "C" lantern_status lantern_verify_tree(
   a.B = batch; a.N = t->n_nodes; a.V = V; a.n_internal = t->n_internal; a.max_children = t->max_children;
   a.kpad = (p->k + 3) & ~3;
   a.g = p->cfg_scale; a.inv_tau = 1.0f / p->temperature; a.lambda = p->lambda; a.delta = p->delta;
+  a.skip = p->subset_rule; a.det = det ? 1 : 0;
   a.topk_t = p->top_k_target; a.topk_d = p->top_k_draft; a.k = p->k;
   a.code_offset = p->code_offset; a.n_codes = p->n_codes; a.allow_lo = allow_lo; a.allow_hi = allow_hi;
   a.seed = p->seed; a.step = p->step;
@@ -249,9 +259,10 @@ extern "C" lantern_status lantern_verify_tree(
     a.only = redo;
   }
   if (!use_sparse && verify_uses_stream(p, t)) {
-    const int cs = stream_cluster_size(batch * t->n_nodes, allow_hi - allow_lo, f32);
+    const int cs = stream_cluster_size(a.lazy ? batch : batch * t->n_nodes, allow_hi - allow_lo, f32);
     e = launch_stream_any(a, cs, stream::smem_bytes(V, t->max_children, p->k + 1, cfg), f32, cfg, st);
     if (e != cudaSuccess) return LANTERN_ERR_CUDA;
+    if (a.lazy) return cudaGetLastError() == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;     // it walks as it goes
     return launch_walk(t, batch, node_next, node_token, tokens, accept_len, out_tokens, out_nodes, D1, st);
   }
   // rows that fit one CTA run the 1024-thread build; rows split over a cluster run the

@@ -205,6 +205,7 @@ struct StreamSmem {
   float* rtot;      // [kMaxCluster] per-CTA sums of the current target (committed)
   float* scan;      // [SW]
   int* misc;        // [32]
+  uint32_t* memb;   // [33] greedy-skip rule: bit r = entry r of the neighbour list joined A
 };
 
 // term of every token of vector vv under the current target (exception and masked tokens: 0)
@@ -240,7 +241,7 @@ __device__ __forceinline__ void vec_terms(const IO& ioq, const IO& iop, const Ge
 // Rejection pass: sum of term_j over this thread's share of warp range [vbeg, vend), skipping
 // the exception tokens; with RESUM also the sum of 2^(zp L + cp) over the tokens not dropped
 // from the drafter.
-template <typename IO, int U, bool RESUM>
+template <typename IO, int U, bool RESUM, bool HASP = true>
 __device__ __forceinline__ void pass_residual(const IO& ioq, const IO& iop, const Geo& ge, int vbeg, int vend, int lane,
                                               const Cur& k, const uint32_t* __restrict__ bits,
                                               const int* __restrict__ dropped, int n_dropped, float& acc, float& accp) {
@@ -252,7 +253,10 @@ __device__ __forceinline__ void pass_residual(const IO& ioq, const IO& iop, cons
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int vv = base + 32 * u + lane;
-      if (vv < he) { ioq.load(vv, qc[u], qu[u]); iop.load(vv, pc[u], pu[u]); }
+      if (vv < he) {
+        ioq.load(vv, qc[u], qu[u]);
+        if (HASP) iop.load(vv, pc[u], pu[u]);
+      }
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -260,16 +264,16 @@ __device__ __forceinline__ void pass_residual(const IO& ioq, const IO& iop, cons
       if (vv < he) {
         float zq[VN], zp[VN];
         ioq.z(qc[u], qu[u], zq);
-        iop.z(pc[u], pu[u], zp);
+        if (HASP) iop.z(pc[u], pu[u], zp);
         const int j = ge.j0 + vv * VN;
         const uint32_t ex = (bits[j >> 5] >> (j & 31)) & ((1u << VN) - 1u);
         if (ex == 0u) {
 #pragma unroll
           for (int e = 0; e < VN; e += 2) {
             const float x0 = ex2_approx(fmaf(zq[e], kLog2e, k.cq)) * k.aq;
-            const float y0 = ex2_approx(fmaf(zp[e], kLog2e, k.cp));
+            const float y0 = HASP ? ex2_approx(fmaf(zp[e], kLog2e, k.cp)) : 0.f;
             const float x1 = ex2_approx(fmaf(zq[e + 1], kLog2e, k.cq)) * k.aq;
-            const float y1 = ex2_approx(fmaf(zp[e + 1], kLog2e, k.cp));
+            const float y1 = HASP ? ex2_approx(fmaf(zp[e + 1], kLog2e, k.cp)) : 0.f;
             a0 += fmaxf(fmaf(-y0, k.ap, x0), 0.f);
             a1 += fmaxf(fmaf(-y1, k.ap, x1), 0.f);
             if (RESUM) { p0 += y0; p1 += y1; }
@@ -277,7 +281,7 @@ __device__ __forceinline__ void pass_residual(const IO& ioq, const IO& iop, cons
         } else {
 #pragma unroll
           for (int e = 0; e < VN; ++e) {
-            const float y = ex2_approx(fmaf(zp[e], kLog2e, k.cp));
+            const float y = HASP ? ex2_approx(fmaf(zp[e], kLog2e, k.cp)) : 0.f;
             if (!((ex >> e) & 1u)) {
               const float x = ex2_approx(fmaf(zq[e], kLog2e, k.cq)) * k.aq;
               a0 += fmaxf(fmaf(-y, k.ap, x), 0.f);
@@ -300,7 +304,7 @@ __device__ __forceinline__ void pass_residual(const IO& ioq, const IO& iop, cons
       for (int e = 0; e < VN; ++e) {
         const int t = ge.j0 + vv * VN + e;
         if (t < ge.alo || t >= ge.ahi) continue;
-        const float y = ex2_approx(fmaf(iop.z_at(t), kLog2e, k.cp));
+        const float y = HASP ? ex2_approx(fmaf(iop.z_at(t), kLog2e, k.cp)) : 0.f;
         const bool ex = (bits[t >> 5] >> (t & 31)) & 1u;
         if (!ex) {
           const float x = ex2_approx(fmaf(ioq.z_at(t), kLog2e, k.cq)) * k.aq;
@@ -320,7 +324,8 @@ __device__ __forceinline__ void pass_residual(const IO& ioq, const IO& iop, cons
 
 // One tree node (sequence b, node n).  Returns the accepted child or -1, the same value in
 // every thread of the node's CTAs.
-template <typename T, bool CFG, bool TAU1>
+// VAR: the acceptance-rule variants (greedy-skip subset, deterministic drafts) are compiled in.
+template <typename T, bool CFG, bool TAU1, bool VAR>
 __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, const int n, SCtx& c, const StreamSmem& sm) {
   using IO = RowIO<T, CFG, TAU1>;
   constexpr int VN = IO::VN;
@@ -334,6 +339,9 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
   const long long out_b = static_cast<long long>(b) * a.N;
   const int kp1 = a.k + 1;
   const bool writer = c.rank == 0 && tid == 0;
+  const bool det = VAR && a.det != 0;       // deterministic drafts (Sec. 3): p(x) = 1, no drafter row
+  const bool skip = VAR && a.skip != 0;     // greedy-skip subset rule
+  const bool has_p = nc > 0 && !det;
   float* fm = reinterpret_cast<float*>(sm.misc);
   int* dropped = sm.misc + 16;          // [LANTERN_MAX_CHILDREN] rejected draft tokens
 
@@ -354,8 +362,8 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
   ioq.u = CFG ? static_cast<const T*>(a.tu) + row_off : nullptr;
   ioq.g = a.g; ioq.it = a.inv_tau; ioq.j0 = ge.j0;
   iop = ioq;
-  iop.c = nc > 0 ? static_cast<const T*>(a.dc) + row_off : nullptr;
-  iop.u = (CFG && nc > 0) ? static_cast<const T*>(a.du) + row_off : nullptr;
+  iop.c = has_p ? static_cast<const T*>(a.dc) + row_off : nullptr;
+  iop.u = (CFG && has_p) ? static_cast<const T*>(a.du) + row_off : nullptr;
 
   // ---- exception bitmap, uniforms
   {
@@ -390,10 +398,10 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
         const int w = sizeof(T) == 4 ? t : (t & ~1);
         const uint32_t dst = smem_u32(sm.ent + e * NOPS);
         cp_async4(dst, ioq.c + w);
-        cp_async4(dst + 4, iop.c + w);
+        if (has_p) cp_async4(dst + 4, iop.c + w);
         if (CFG) {
           cp_async4(dst + 8, ioq.u + w);
-          cp_async4(dst + 12, iop.u + w);
+          if (has_p) cp_async4(dst + 12, iop.u + w);
         }
       }
     }
@@ -405,7 +413,7 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
   float mx[2] = {-INFINITY, -INFINITY}, sx[2] = {0.f, 0.f};
   {
     const int hb = max(vbeg, ge.vi0), he = min(vend, ge.vi1);
-    if (nc > 0) {
+    if (has_p) {
       // the two rows alternate in the instruction stream so that both are in flight
       for (int base = hb; base < he; base += 32 * U2) {
         uint4 qc[U2], qu[U2], pc[U2], pu[U2];
@@ -447,13 +455,13 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
     }
     if (lane == 0) {
       edge_sum(ioq, ge, vbeg, vend, mx[0], sx[0]);
-      if (nc > 0) edge_sum(iop, ge, vbeg, vend, mx[1], sx[1]);
+      if (has_p) edge_sum(iop, ge, vbeg, vend, mx[1], sx[1]);
     }
   }
   // common references, then the sums relative to them
   float gm[2] = {warp_max(mx[0]), warp_max(mx[1])};
   combine<2, true>(c, gm);
-  if (gm[0] == -INFINITY || (nc > 0 && gm[1] == -INFINITY)) {
+  if (gm[0] == -INFINITY || (has_p && gm[1] == -INFINITY)) {
     if (writer) vflag(a.status, LANTERN_DEV_EMPTY_ROW);
   }
   if (gm[0] == -INFINITY) gm[0] = 0.f;
@@ -498,9 +506,8 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
           v[o] = sizeof(T) == 4 ? __uint_as_float(raw) : __uint_as_float((t & 1) ? (raw & 0xffff0000u) : (raw << 16));
         }
         const float zq = ioq.z1(v[0], CFG ? v[2] : 0.f);
-        const float zp = ioq.z1(v[1], CFG ? v[3] : 0.f);
         q0 = ex2_approx(fmaf(zq, kLog2e, cur.cq)) * rq;
-        p0 = ex2_approx(fmaf(zp, kLog2e, cur.cp)) * rp;
+        if (has_p) p0 = ex2_approx(fmaf(ioq.z1(v[1], CFG ? v[3] : 0.f), kLog2e, cur.cp)) * rp;
       }
       sm.ent[e * NOPS] = q0;
       sm.ent[e * NOPS + 1] = p0;
@@ -538,11 +545,28 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
         return fmaxf(fmaf(-alpha, en[r * NOPS + 1], en[r * NOPS]), 0.f) * ibeta;
       };
       const float qx = val(0);
-      const float px = x_dropped ? 0.f : en[1] * iW;
+      const float px = det ? 1.f : (x_dropped ? 0.f : en[1] * iW);
       const float bound = a.delta > 0.f ? qx + a.delta : a.lambda * qx;      // Sec. 2.2 / Sec. 4
       float cum = qx;
       int nA = 0;
       bool open = has_code;
+      if (skip && open) {
+        // greedy-skip rule: a neighbour that would break the bound is passed over and the list
+        // is searched on; the running sum is sequential, 32 entries at a time through shuffles
+        for (int base = 0; base < a.k; base += 32) {
+          const int r = base + lane;
+          const float v = r < a.k ? val(1 + r) : 0.f;
+          uint32_t mask = 0u;
+          const int lim = min(32, a.k - base);
+          for (int i = 0; i < lim; ++i) {
+            const float vi = __shfl_sync(0xffffffffu, v, i);
+            if (cum + vi < bound) { cum += vi; mask |= 1u << i; }
+          }
+          if (lane == 0) sm.memb[base >> 5] = mask;
+          nA += __popc(mask);
+        }
+        open = false;
+      }
       for (int base8 = 0; base8 < a.k && open; base8 += 256) {
         float qa[8];
 #pragma unroll
@@ -588,9 +612,18 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
       continue;
     }
     // ---- rejection: the members of A and x join the exception set; x leaves the drafter
-    for (int r = tid; r < nA; r += ST) {
-      const int t = tk[1 + r];
-      if (t >= 0) atomicOr(&sm.bits[t >> 5], 1u << (t & 31));
+    if (skip) {
+      if (has_code) {
+        for (int r = tid; r < a.k; r += ST) {
+          const int t = tk[1 + r];
+          if (t >= 0 && ((sm.memb[r >> 5] >> (r & 31)) & 1u)) atomicOr(&sm.bits[t >> 5], 1u << (t & 31));
+        }
+      }
+    } else {
+      for (int r = tid; r < nA; r += ST) {
+        const int t = tk[1 + r];
+        if (t >= 0) atomicOr(&sm.bits[t >> 5], 1u << (t & 31));
+      }
     }
     if (tid == 0) {
       atomicOr(&sm.bits[x >> 5], 1u << (x & 31));
@@ -600,19 +633,20 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
     __syncthreads();
     const float alpha_n = fmaf(beta, iW, alpha);
     Cur nx;
-    nx.cq = cur.cq; nx.cp = cur.cp; nx.aq = rq; nx.ap = alpha_n * rp; nx.has_p = true;
-    const bool resum = px > 0.5f;
+    nx.cq = cur.cq; nx.cp = cur.cp; nx.aq = rq; nx.ap = det ? 0.f : alpha_n * rp; nx.has_p = !det;
+    const bool resum = !det && px > 0.5f;
     float zs[2];
     {
       float accq, accp;
-      if (resum) pass_residual<IO, U2, true>(ioq, iop, ge, vbeg, vend, lane, nx, sm.bits, dropped, n_dropped, accq, accp);
+      if (det) pass_residual<IO, U1, false, false>(ioq, iop, ge, vbeg, vend, lane, nx, sm.bits, dropped, n_dropped, accq, accp);
+      else if (resum) pass_residual<IO, U2, true>(ioq, iop, ge, vbeg, vend, lane, nx, sm.bits, dropped, n_dropped, accq, accp);
       else pass_residual<IO, U2, false>(ioq, iop, ge, vbeg, vend, lane, nx, sm.bits, dropped, n_dropped, accq, accp);
       zs[0] = warp_sum(accq);
       zs[1] = warp_sum(accp);
     }
     if (lane == 0) sm.wtmp[warp] = zs[0];
     combine<2, false>(c, zs);
-    const float W_n = resum ? zs[1] * rp : W - en[1] * (x_dropped ? 0.f : 1.f);
+    const float W_n = det ? W : (resum ? zs[1] * rp : W - en[1] * (x_dropped ? 0.f : 1.f));
     if (zs[0] > 0.f) {
       alpha = alpha_n;
       beta = zs[0];
@@ -717,7 +751,9 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
   return accepted;
 }
 
-template <typename T, bool CFG, bool TAU1>
+// GENERAL = false: one node per CTA (cluster), default acceptance rule (the benchmarked launch).
+// GENERAL = true: the same plus what is decided at run time: the path walk and the rule variants.
+template <typename T, bool CFG, bool TAU1, bool GENERAL>
 __global__ void __launch_bounds__(ST, LANTERN_STREAM_MINB) verify_stream_kernel(const VerifyArgs a) {
   grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char stream_smem[];
@@ -734,7 +770,8 @@ __global__ void __launch_bounds__(ST, LANTERN_STREAM_MINB) verify_stream_kernel(
   sm.rtot = sm.wtmp + SW;              // kMaxCluster
   sm.scan = sm.rtot + kMaxCluster;     // SW
   sm.misc = reinterpret_cast<int*>(sm.scan + SW);      // 32
-  static_assert((2 * SW * 4 + 8 + kMaxCluster * 4 + SW + SW + kMaxCluster + SW + 32) * 4 <= kSmallBytes, "small area");
+  sm.memb = reinterpret_cast<uint32_t*>(sm.misc + 32); // 33
+  static_assert((2 * SW * 4 + 8 + kMaxCluster * 4 + SW + SW + kMaxCluster + SW + 32 + 33) * 4 <= kSmallBytes, "small area");
   sm.bits = reinterpret_cast<uint32_t*>(stream_smem + kSmallBytes);
   sm.ent = reinterpret_cast<float*>(sm.bits + (a.V + 127) / 128 * 4);
   sm.tok = reinterpret_cast<int*>(sm.ent + static_cast<size_t>(a.max_children) * kp1 * NOPS);
@@ -742,7 +779,34 @@ __global__ void __launch_bounds__(ST, LANTERN_STREAM_MINB) verify_stream_kernel(
   c.nrank = cluster_nctarank();
   c.parity = 0;
   const int idx = blockIdx.x / c.nrank;
-  stream_node<T, CFG, TAU1>(a, idx % a.B, a.order[idx / a.B], c, sm);
+  // A regular launch verifies one node per CTA (cluster).  With a.lazy the CTA (cluster) owns a
+  // sequence and walks it (Sec. 2.1): it verifies the root, moves to the accepted child and so
+  // on, so only the rows on the accepted path are read and the per-node results of the other
+  // nodes are not written.
+  const bool lazy = GENERAL && a.lazy != 0;
+  const int b = lazy ? idx : idx % a.B;
+  int cur = lazy ? 0 : a.order[idx / a.B];
+  int len = 0;
+  for (;;) {
+    const int acc = stream_node<T, CFG, TAU1, GENERAL>(a, b, cur, c, sm);
+    if (!lazy) break;
+    csync(c);     // the next node reuses the shared memory; also orders the store of node_token before the read below
+    const bool writer = c.rank == 0 && threadIdx.x == 0;
+    int32_t* ot = a.out_tokens + static_cast<long long>(b) * a.D1;
+    int32_t* on = a.out_nodes + static_cast<long long>(b) * a.D1;
+    if (acc <= cur || acc >= a.N || len >= a.D1 - 1) {      // -1, or anything that is not a forward edge
+      if (writer) {
+        ot[len] = __ldcg(a.node_token + static_cast<long long>(b) * a.N + cur);
+        on[len] = cur;
+        a.accept_len[b] = len;
+        for (int i = len + 1; i < a.D1; ++i) { ot[i] = -1; on[i] = -1; }
+      }
+      break;
+    }
+    cur = acc;
+    if (writer) { ot[len] = a.tokens[static_cast<long long>(b) * a.N + cur]; on[len] = cur; }
+    ++len;
+  }
   if (c.nrank > 1) cluster_sync();     // peers may still be reading this CTA's exchange buffer
 }
 

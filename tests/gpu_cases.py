@@ -25,7 +25,7 @@ class Case:
 
     def __init__(self, cfg, parent=None, seed=0, allowed=(0, 0), k_table=None, temperature=None,
                  top_k_target=None, top_k_draft=None, pad=0, oracle_seqs=None, tokens="oracle", delta=0.0,
-                 library_table=False):
+                 library_table=False, skip=False, det_draft=False):
         self.cfg = cfg
         self.parent = W.static_tree(cfg.n_nodes) if parent is None else parent
         N, B, V = len(self.parent), cfg.batch, cfg.vocab
@@ -47,7 +47,8 @@ class Case:
             top_k_target=cfg.top_k if top_k_target is None else top_k_target,
             top_k_draft=cfg.top_k if top_k_draft is None else top_k_draft,
             lam=cfg.lam, k=cfg.k, code_offset=cfg.code_offset, n_codes=cfg.codebook_size,
-            allowed_begin=allowed[0], allowed_end=allowed[1] if allowed[1] else V, delta=delta)
+            allowed_begin=allowed[0], allowed_end=allowed[1] if allowed[1] else V, delta=delta,
+            skip=skip, det_draft=det_draft)
         self.seqs = list(range(B)) if oracle_seqs is None else list(oracle_seqs)
         # draft tokens: oracle sampler on the checked sequences, uniform random elsewhere
         lo, hi = self.params["allowed_begin"], self.params["allowed_end"]
@@ -106,7 +107,7 @@ class Case:
                                            p["temperature"], p["top_k_draft"], p["allowed_begin"], p["allowed_end"])
         return oracle.verify_node(q, pd, children[n], self.tokens[b], self.u_accept[b].numpy(),
                                   self.u_resample[b].numpy()[n], self.nbr, p["k"], p["lam"], p["code_offset"],
-                                  p["n_codes"], p["delta"], forced=forced)
+                                  p["n_codes"], p["delta"], forced=forced, skip=p["skip"], det_draft=p["det_draft"])
 
     # ---- device side
     def gpu_inputs(self, L):
@@ -116,7 +117,8 @@ class Case:
         par = L.Params(vocab=self.V, cfg_scale=p["cfg_scale"], temperature=p["temperature"],
                        top_k_target=p["top_k_target"], top_k_draft=p["top_k_draft"], lam=p["lam"], k=p["k"],
                        code_offset=p["code_offset"], n_codes=p["n_codes"], allowed_begin=p["allowed_begin"],
-                       allowed_end=p["allowed_end"], delta=p["delta"])
+                       allowed_end=p["allowed_end"], delta=p["delta"], subset_rule=int(p["skip"]),
+                       draft_deterministic=int(p["det_draft"]))
         nbr = None if self.nbr is None else torch.from_numpy(self.nbr).to(dev)
         if self.library_table:
             nbr = L.build_neighbors(self.codebook.to(dev), self.k_table)

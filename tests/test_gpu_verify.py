@@ -101,8 +101,8 @@ def test_path_queries_and_graph_replay_match_eager_calls(L):
     assert L.verify_tree_path(par, tree) == 1 and L.sample_draft_tree_path(par) == 1
     par_dense = L.Params(**{**par.__dict__, "top_k_target": 0, "top_k_draft": 0})
     assert L.verify_tree_path(par_dense, tree) == 2 and L.sample_draft_tree_path(par_dense) == 2      # streaming kernels
-    par_walk = L.Params(**{**par_dense.__dict__, "lazy_walk": 1})
-    assert L.verify_tree_path(par_walk, tree) == 0
+    par_walk = L.Params(**{**par.__dict__, "lazy_walk": 1})
+    assert L.verify_tree_path(par_walk, tree) == 0            # top-k rows walk with the dense kernel
     old = L.set_cluster_size(1)
     try:
         assert L.verify_tree_path(par, tree) == 0
@@ -331,3 +331,56 @@ def test_lumina_shape_with_the_table_the_library_built(L):
     case = Case(cfg, seed=4, library_table=True, allowed=(cfg.code_offset, cfg.code_offset + cfg.codebook_size))
     res, stats = _run(L, case)
     assert stats["tested"] > 50
+
+
+@pytest.mark.parametrize("cs", [0, 1, 4])
+@pytest.mark.parametrize("kw", [dict(k=24, lam=1.8), dict(k=24, lam=1.8, dtype="bf16", cfg_scale=None),
+                                dict(vocab=5003, codebook_size=5003, k=40, lam=1.6)])
+def test_greedy_skip_subset_rule(L, cs, kw):
+    """subset_rule = 1 (the other reading of Sec. 4's subset): parity with the oracle's greedy set."""
+    pad = 5 if "vocab" in kw else 0
+    old = L.set_cluster_size(cs)
+    try:
+        case = Case(small_config(**kw), seed=41, skip=True, pad=pad)
+        _run(L, case)
+    finally:
+        L.set_cluster_size(old)
+    # the rule matters on these inputs: the prefix rule gives other masses somewhere
+    plain = Case(small_config(**kw), seed=41, pad=pad).oracle_verify()
+    assert any(not np.allclose(a["node_mass"], b["node_mass"]) for a, b in zip(case.oracle_verify(), plain))
+
+
+@pytest.mark.parametrize("cs", [0, 2])
+@pytest.mark.parametrize("kw", [dict(), dict(dtype="bf16", cfg_scale=None, k=0), dict(n_nodes=60, lam=1.5)])
+def test_deterministic_draft_mode(L, cs, kw):
+    """draft_deterministic = 1 (Sec. 3): accept probability m, drafter rows never read (NULL)."""
+    old = L.set_cluster_size(cs)
+    try:
+        case = Case(small_config(**kw), seed=43, det_draft=True)
+        g, par, nbr, tok = case.gpu_inputs(L)
+        tree = L.Tree(case.parent)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], None, None, tok,
+                            case.u_accept.cuda(), case.u_resample.cuda(), debug=True, device_status=status)
+        torch.cuda.synchronize()
+        res = {k: v.cpu().numpy() for k, v in out.items()}
+        assert int(status.item()) == 0
+        orc = case.oracle_verify()
+        stats = compare_verify(res, orc, case.parent, case.u_accept.numpy(), case.seqs, rerun=case.oracle_node)
+        check_walk(res, case.tokens, tree.max_depth, orc, stats["dirty_sequences"], case.seqs, stats["patched"])
+        thr, mass = res["node_thresh"], res["node_mass"]
+        tested = mass >= 0
+        assert np.allclose(thr[tested], np.minimum(1.0, mass[tested]), atol=1e-6)
+    finally:
+        L.set_cluster_size(old)
+
+
+def test_variants_are_refused_on_topk_rows(L):
+    case = Case(small_config(top_k=50), seed=44)
+    g, par, nbr, tok = case.gpu_inputs(L)
+    tree = L.Tree(case.parent)
+    for kw in (dict(subset_rule=1), dict(draft_deterministic=1)):
+        bad = L.Params(**{**par.__dict__, **kw})
+        with pytest.raises(L.LanternError) as e:
+            L.verify_tree(bad, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"], tok)
+        assert e.value.status == 2
