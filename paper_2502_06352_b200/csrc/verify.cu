@@ -156,6 +156,9 @@ bool verify_uses_stream(const lantern_params* p, const TreeDev* t) {
   const int V = p->vocab;
   const bool tk_t = p->top_k_target > 0 && p->top_k_target < V;
   const bool tk_d = t->n_internal > 0 && !p->draft_deterministic && p->top_k_draft > 0 && p->top_k_draft < V;
+  // (the path walk is a chain of dependent nodes per sequence: the dense kernel, whose rejection
+  // passes read shared memory, walks it faster; the streaming kernel walks only for the variants)
+  if (p->lazy_walk && !p->subset_rule && !p->draft_deterministic) return false;
   return !tk_t && !tk_d && V <= stream::kMaxV &&
          stream::smem_bytes(V, t->max_children, p->k + 1, true) <= 227 * 1024;
 }

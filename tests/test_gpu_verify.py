@@ -375,6 +375,22 @@ def test_deterministic_draft_mode(L, cs, kw):
         L.set_cluster_size(old)
 
 
+def test_path_walk_with_a_rule_variant_runs_on_the_streaming_kernel(L):
+    case = Case(small_config(k=24, lam=1.8, batch=4, n_nodes=60), seed=45, skip=True)
+    g, par, nbr, tok = case.gpu_inputs(L)
+    tree = L.Tree(case.parent)
+    ua, ur = case.u_accept.cuda(), case.u_resample.cuda()
+    eager = L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"],
+                          tok, ua, ur, debug=True)
+    par.lazy_walk = 1
+    assert L.verify_tree_path(par, tree) == 2
+    lazy = L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"],
+                         tok, ua, ur, debug=True)
+    torch.cuda.synchronize()
+    for k in ("accept_len", "out_tokens", "out_nodes"):
+        assert torch.equal(lazy[k], eager[k]), k
+
+
 def test_variants_are_refused_on_topk_rows(L):
     case = Case(small_config(top_k=50), seed=44)
     g, par, nbr, tok = case.gpu_inputs(L)
