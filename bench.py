@@ -373,8 +373,8 @@ class Workload:
 
     def kernels(self):
         """Which kernels the library runs for these parameters (it decides; this only reports)."""
-        pv = self.L.verify_tree_path(self.params, self.tree)
-        ps = self.L.sample_draft_tree_path(self.params)
+        pv = self.L.verify_tree_path(self.params, self.tree, self.B)
+        ps = self.L.sample_draft_tree_path(self.params, self.tree, self.B)
         v = {0: ("verify_nodes_kernel + walk_kernel", 2),
              1: ("verify_sparse_kernel + verify_nodes_kernel (repair launch, walks the trees)", 2),
              2: ("verify_stream_kernel + walk_kernel", 2)}[pv]

@@ -110,6 +110,9 @@ typedef struct {
                               p(x) = 1 for each of them: a child is accepted with probability
                               min(1, m), the residual after a rejection is q~ without x, and the
                               drafter rows are never read (draft_* may be NULL)                   */
+  int32_t kernels;         /* 0: the library chooses between its kernels by size (see "which kernels a
+                              call launches").  1: streaming kernels wherever they apply, whatever
+                              the size.  2: never the streaming kernels.  Results are the same     */
 } lantern_params;
 /* subset_rule = 1 and draft_deterministic = 1 are served by the streaming kernels only: rows that a
  * top-k truncates return LANTERN_ERR_UNSUPPORTED with either of them.                              */
@@ -204,9 +207,12 @@ lantern_status lantern_verify_tree(const lantern_params* params, const lantern_t
  * the row is compacted to its survivors; everything after works on those), followed by a launch of
  * the dense kernels that redoes the nodes whose rows did not fit the lists' fixed buffers (massive
  * ties; usually none).  All other calls (top-k on wide vocabularies, the path walk) run the dense
- * kernels alone (LANTERN_PATH_DENSE: rows held in shared memory).  Results are the same either way;
- * these queries only tell which it will be (lantern_verify_tree additionally needs its full
- * workspace for the list path).
+ * kernels alone (LANTERN_PATH_DENSE: rows held in shared memory).  So do small calls without top-k
+ * (fewer than 128 tree nodes, or 256 expanded parents, in the whole batch) whose rows fit the dense
+ * kernels: a handful of nodes is a chain of dependent steps, which shared-memory rows shorten.
+ * params->kernels overrides the choice by size.  Results are the same either way; these queries
+ * only tell which it will be for a batch of `batch` sequences (lantern_verify_tree additionally
+ * needs its full workspace for the list path).
  * Launches per call: lantern_sample_draft_tree 1 (streaming, dense) or 2 (lists + repair);
  * lantern_verify_tree 2 (streaming + walk, dense + walk, or lists + repair launch that also
  * walks), or 1 with params->lazy_walk (the path-walk kernel walks as it goes).  Returns -1 on NULL
@@ -214,8 +220,8 @@ lantern_status lantern_verify_tree(const lantern_params* params, const lantern_t
 #define LANTERN_PATH_DENSE 0
 #define LANTERN_PATH_LISTS 1
 #define LANTERN_PATH_STREAM 2
-int32_t lantern_verify_tree_path(const lantern_params* params, const lantern_tree* tree);
-int32_t lantern_sample_draft_tree_path(const lantern_params* params);
+int32_t lantern_verify_tree_path(const lantern_params* params, const lantern_tree* tree, int32_t batch);
+int32_t lantern_sample_draft_tree_path(const lantern_params* params, const lantern_tree* tree, int32_t batch);
 
 /* ---- relaxed verification without any allocation ---------------------------------------------
  * The paper has no counterpart to this entry point; it exists for callers that must not, or

@@ -31,7 +31,7 @@ class _CParams(ctypes.Structure):
         ("allowed_begin", ctypes.c_int32), ("allowed_end", ctypes.c_int32),
         ("seed", ctypes.c_uint64), ("step", ctypes.c_uint64),
         ("delta", ctypes.c_float), ("lazy_walk", ctypes.c_int32),
-        ("subset_rule", ctypes.c_int32), ("draft_deterministic", ctypes.c_int32),
+        ("subset_rule", ctypes.c_int32), ("draft_deterministic", ctypes.c_int32), ("kernels", ctypes.c_int32),
     ]
 
 
@@ -55,12 +55,13 @@ class Params:
     lazy_walk: int = 0
     subset_rule: int = 0
     draft_deterministic: int = 0
+    kernels: int = 0
 
     def c(self):
         return _CParams(self.cfg_scale, self.temperature, self.top_k_target, self.top_k_draft,
                         self.lam, self.k, self.vocab, self.code_offset, self.n_codes,
                         self.allowed_begin, self.allowed_end, self.seed, self.step, self.delta, self.lazy_walk,
-                        self.subset_rule, self.draft_deterministic)
+                        self.subset_rule, self.draft_deterministic, self.kernels)
 
 
 def _load():
@@ -103,9 +104,9 @@ def _load():
     L.lantern_get_cluster_size.restype = i32
     L.lantern_get_cluster_size.argtypes = []
     L.lantern_verify_tree_path.restype = i32
-    L.lantern_verify_tree_path.argtypes = [ctypes.POINTER(_CParams), vp]
+    L.lantern_verify_tree_path.argtypes = [ctypes.POINTER(_CParams), vp, i32]
     L.lantern_sample_draft_tree_path.restype = i32
-    L.lantern_sample_draft_tree_path.argtypes = [ctypes.POINTER(_CParams)]
+    L.lantern_sample_draft_tree_path.argtypes = [ctypes.POINTER(_CParams), vp, i32]
     return L
 
 
@@ -274,18 +275,18 @@ def philox_raw(seed, first, c1, c2, c3, n, device="cuda"):
     return out.to(torch.int64) & 0xFFFFFFFF
 
 
-def verify_tree_path(params: "Params", tree: "Tree") -> int:
+def verify_tree_path(params: "Params", tree: "Tree", batch: int) -> int:
     """lantern_verify_tree_path: 0 = dense kernels, 1 = list-based kernels + repair launch,
     2 = streaming kernel (rows without top-k)."""
     cp = params.c()
-    return lib.lantern_verify_tree_path(ctypes.byref(cp), tree.handle)
+    return lib.lantern_verify_tree_path(ctypes.byref(cp), tree.handle, batch)
 
 
-def sample_draft_tree_path(params: "Params") -> int:
+def sample_draft_tree_path(params: "Params", tree: "Tree", batch: int) -> int:
     """lantern_sample_draft_tree_path: 0 = dense kernel, 1 = list-based kernel + repair launch,
     2 = streaming kernel (rows without top-k)."""
     cp = params.c()
-    return lib.lantern_sample_draft_tree_path(ctypes.byref(cp))
+    return lib.lantern_sample_draft_tree_path(ctypes.byref(cp), tree.handle, batch)
 
 
 def set_cluster_size(ctas_per_row: int) -> int:

@@ -429,14 +429,21 @@ bool sampler_uses_lists(const lantern_params* p) {
 }
 }  // namespace
 
-// Rows that no top-k truncates take the streaming kernel.
-static bool sampler_uses_stream(const lantern_params* p) {
-  return !(p->top_k_draft > 0 && p->top_k_draft < p->vocab) && p->vocab <= stream::kMaxV;
+// Rows that no top-k truncates can take the streaming kernel; it does when the call expands at
+// least kStreamMinParents parents (fewer are a chain of dependent steps that the dense kernel's
+// shared-memory row shortens), when the dense kernel cannot hold the row, or when asked to.
+constexpr int kStreamMinParents = 256;
+static bool sampler_uses_stream(const lantern_params* p, long long parents, bool fits_dense) {
+  if ((p->top_k_draft > 0 && p->top_k_draft < p->vocab) || p->vocab > stream::kMaxV) return false;
+  if (p->kernels == 2) return !fits_dense;
+  if (p->kernels == 1) return true;
+  return parents >= kStreamMinParents || !fits_dense;
 }
 
-extern "C" int32_t lantern_sample_draft_tree_path(const lantern_params* p) {
-  if (!p) return -1;
-  if (sampler_uses_stream(p)) return LANTERN_PATH_STREAM;
+extern "C" int32_t lantern_sample_draft_tree_path(const lantern_params* p, const lantern_tree* tree, int32_t batch) {
+  if (!p || !tree || batch <= 0) return -1;
+  const TreeDev* t = reinterpret_cast<const TreeDev*>(tree);
+  if (sampler_uses_stream(p, static_cast<long long>(batch) * t->n_internal, true)) return LANTERN_PATH_STREAM;
   return sampler_uses_lists(p) ? LANTERN_PATH_LISTS : LANTERN_PATH_DENSE;
 }
 
@@ -487,7 +494,11 @@ extern "C" lantern_status lantern_sample_draft_tree(
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool cfg = draft_uncond != nullptr;
   const int ov = lantern_get_cluster_size();
-  if (sampler_uses_stream(p)) {
+  int cs_d, e_d;
+  size_t smem_d;
+  const bool fits_dense = sampler_shape(V, batch * (i1 - i0), dt == LANTERN_F32 ? 4 : 8, ov, &cs_d, &e_d, &smem_d);
+  if (p->kernels < 0 || p->kernels > 2) return LANTERN_ERR_INVALID_ARG;
+  if (sampler_uses_stream(p, static_cast<long long>(batch) * (i1 - i0), fits_dense)) {
     // CTAs per parent: one when the parents alone fill the machine
     int cs = ov;
     if (cs <= 0) {

@@ -151,23 +151,41 @@ bool verify_uses_lists(const lantern_params* p, const TreeDev* t) {
          V <= sparse::kMaxV && topk_fits(p->top_k_target) &&
          (t->n_internal == 0 || topk_fits(p->top_k_draft)) && t->max_children <= 8;
 }
-// Rows that no top-k truncates take the streaming kernel.
-bool verify_uses_stream(const lantern_params* p, const TreeDev* t) {
+// Can the streaming kernel serve these parameters at all (rows that no top-k truncates)?
+bool stream_applies(const lantern_params* p, const TreeDev* t) {
   const int V = p->vocab;
   const bool tk_t = p->top_k_target > 0 && p->top_k_target < V;
   const bool tk_d = t->n_internal > 0 && !p->draft_deterministic && p->top_k_draft > 0 && p->top_k_draft < V;
-  // (the path walk is a chain of dependent nodes per sequence: the dense kernel, whose rejection
-  // passes read shared memory, walks it faster; the streaming kernel walks only for the variants)
-  if (p->lazy_walk && !p->subset_rule && !p->draft_deterministic) return false;
   return !tk_t && !tk_d && V <= stream::kMaxV &&
          stream::smem_bytes(V, t->max_children, p->k + 1, true) <= 227 * 1024;
 }
+// Can the dense kernels hold a row of these parameters (float32 rows in shared memory)?
+bool dense_fits(const lantern_params* p, const TreeDev* t, bool f32, bool cfg) {
+  const int kpad = (p->k + 3) & ~3, min_e = f32 ? 4 : 8;
+  v1024::LaunchShape s1;
+  v512::LaunchShape s5;
+  return v1024::choose_shape(p->vocab, 1 << 20, t->max_children, kpad, min_e, cfg, &s1) ||
+         v512::choose_shape(p->vocab, 1 << 20, t->max_children, kpad, min_e, cfg, &s5);
+}
+constexpr int kStreamMinNodes = 128;     // below this many nodes per call the dense kernels' shorter chain wins
+// Does this call take the streaming kernel?  (`fits_dense`: the answer of dense_fits, or true when
+// the storage type is not known yet, as in the path query.)
+bool verify_uses_stream(const lantern_params* p, const TreeDev* t, int batch, bool fits_dense) {
+  if (!stream_applies(p, t)) return false;
+  if (p->subset_rule || p->draft_deterministic) return true;       // only the streaming kernel has the variants
+  if (p->kernels == 2) return !fits_dense;
+  // the path walk is a chain of dependent nodes per sequence: the dense kernel, whose rejection
+  // passes read shared memory, walks it faster
+  if (p->lazy_walk) return !fits_dense;
+  if (p->kernels == 1) return true;
+  return static_cast<long long>(batch) * t->n_nodes >= kStreamMinNodes || !fits_dense;
+}
 }  // namespace
 
-extern "C" int32_t lantern_verify_tree_path(const lantern_params* p, const lantern_tree* tree) {
-  if (!p || !tree) return -1;
+extern "C" int32_t lantern_verify_tree_path(const lantern_params* p, const lantern_tree* tree, int32_t batch) {
+  if (!p || !tree || batch <= 0) return -1;
   const TreeDev* t = reinterpret_cast<const TreeDev*>(tree);
-  if (verify_uses_stream(p, t)) return LANTERN_PATH_STREAM;
+  if (verify_uses_stream(p, t, batch, true)) return LANTERN_PATH_STREAM;
   return verify_uses_lists(p, t) ? LANTERN_PATH_LISTS : LANTERN_PATH_DENSE;
 }
 
@@ -194,7 +212,8 @@ extern "C" lantern_status lantern_verify_tree(
   if (p->subset_rule != 0 && p->subset_rule != 1) return LANTERN_ERR_INVALID_ARG;
   if (t->n_internal > 0 && !draft_cond && !det) return LANTERN_ERR_INVALID_ARG;
   if ((target_uncond != nullptr) != (draft_uncond != nullptr) && t->n_internal > 0 && !det) return LANTERN_ERR_INVALID_ARG;
-  if ((det || p->subset_rule) && !verify_uses_stream(p, t)) return LANTERN_ERR_UNSUPPORTED;
+  if ((det || p->subset_rule) && !stream_applies(p, t)) return LANTERN_ERR_UNSUPPORTED;
+  if (p->kernels < 0 || p->kernels > 2) return LANTERN_ERR_INVALID_ARG;
   if (p->k < 0 || p->top_k_target < 0 || p->top_k_draft < 0) return LANTERN_ERR_INVALID_ARG;
   if (!(p->delta >= 0.f) || p->delta > 4.f) return LANTERN_ERR_INVALID_ARG;      // also rejects NaN
   if (p->k > 0 && (!nbr_idx || p->k > k_table || p->n_codes <= 0 || k_table > p->n_codes - 1)) return LANTERN_ERR_INVALID_ARG;
@@ -261,7 +280,7 @@ extern "C" lantern_status lantern_verify_tree(
     if (e != cudaSuccess) return LANTERN_ERR_CUDA;
     a.only = redo;
   }
-  if (!use_sparse && verify_uses_stream(p, t)) {
+  if (!use_sparse && verify_uses_stream(p, t, batch, dense_fits(p, t, f32, cfg))) {
     const int cs = stream_cluster_size(a.lazy ? batch : batch * t->n_nodes, allow_hi - allow_lo, f32);
     e = launch_stream_any(a, cs, stream::smem_bytes(V, t->max_children, p->k + 1, cfg), f32, cfg, st);
     if (e != cudaSuccess) return LANTERN_ERR_CUDA;

@@ -25,8 +25,9 @@ class Case:
 
     def __init__(self, cfg, parent=None, seed=0, allowed=(0, 0), k_table=None, temperature=None,
                  top_k_target=None, top_k_draft=None, pad=0, oracle_seqs=None, tokens="oracle", delta=0.0,
-                 library_table=False, skip=False, det_draft=False):
+                 library_table=False, skip=False, det_draft=False, kernels=1):
         self.cfg = cfg
+        self.kernels = kernels      # lantern_params.kernels: 1 = streaming kernels wherever they apply (tests are small)
         self.parent = W.static_tree(cfg.n_nodes) if parent is None else parent
         N, B, V = len(self.parent), cfg.batch, cfg.vocab
         self.N, self.B, self.V = N, B, V
@@ -118,7 +119,7 @@ class Case:
                        top_k_target=p["top_k_target"], top_k_draft=p["top_k_draft"], lam=p["lam"], k=p["k"],
                        code_offset=p["code_offset"], n_codes=p["n_codes"], allowed_begin=p["allowed_begin"],
                        allowed_end=p["allowed_end"], delta=p["delta"], subset_rule=int(p["skip"]),
-                       draft_deterministic=int(p["det_draft"]))
+                       draft_deterministic=int(p["det_draft"]), kernels=self.kernels)
         nbr = None if self.nbr is None else torch.from_numpy(self.nbr).to(dev)
         if self.library_table:
             nbr = L.build_neighbors(self.codebook.to(dev), self.k_table)

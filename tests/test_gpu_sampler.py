@@ -61,9 +61,10 @@ def _compare(case, gum, gtok, gprob):
 
 @pytest.mark.parametrize("kw", [dict(), dict(cfg_scale=None), dict(top_k=20), dict(dtype="bf16", cfg_scale=None),
                                 dict(vocab=1003, codebook_size=1003), dict(n_nodes=60, temperature=0.8)])
-def test_explicit_uniforms(L, kw):
+@pytest.mark.parametrize("kernels", [1, 2])          # streaming kernel forced / excluded
+def test_explicit_uniforms(L, kw, kernels):
     pad = 5 if kw.get("vocab") == 1003 else 0
-    case = Case(small_config(**kw), seed=21, tokens="random", pad=pad)
+    case = Case(small_config(**kw), seed=21, tokens="random", pad=pad, kernels=kernels)
     gum = W.make_gumbel_uniforms(case.B, case.N, case.V, 1234)
     gtok, gprob, _ = _gpu_sample(L, case, gumbel=gum)
     assert _compare(case, gum.numpy(), gtok, gprob) <= 1

@@ -18,14 +18,22 @@ def L():
 
 
 def _run(L, case, **kw):
-    res = case.gpu_verify(L, **kw)
-    assert res["status"] == 0
-    orc = case.oracle_verify()
-    ua = case.u_accept.numpy()
-    stats = compare_verify(res, orc, case.parent, ua, case.seqs, rerun=case.oracle_node)
-    check_walk(res, case.tokens, res["max_depth"], orc, stats["dirty_sequences"], case.seqs, stats["patched"])
-    assert stats["tie_accept"] + stats["tie_cut"] + stats["tie_resample"] <= max(1, stats["nodes"] // 500)
-    return res, stats
+    """Parity of one case; run with the streaming kernels forced and with them excluded, so that
+    every kernel that can serve the parameters is compared with the oracle."""
+    out = None
+    for kernels in (2, 1):
+        case.kernels = kernels
+        res = case.gpu_verify(L, **kw)
+        assert res["status"] == 0
+        orc = case.oracle_verify()
+        ua = case.u_accept.numpy()
+        stats = compare_verify(res, orc, case.parent, ua, case.seqs, rerun=case.oracle_node)
+        check_walk(res, case.tokens, res["max_depth"], orc, stats["dirty_sequences"], case.seqs, stats["patched"])
+        assert stats["tie_accept"] + stats["tie_cut"] + stats["tie_resample"] <= max(1, stats["nodes"] // 500)
+        out = (res, stats)
+        if case.params["skip"] or case.params["det_draft"] or (case.params["top_k_target"] and case.params["top_k_draft"]):
+            break               # one family of kernels serves these parameters
+    return out
 
 
 @pytest.mark.parametrize("cs", [0, 1, 2, 4, 8, 16])
@@ -98,14 +106,18 @@ def test_path_queries_and_graph_replay_match_eager_calls(L):
     case = Case(small_config(vocab=3001, codebook_size=3001, top_k=200, k=12), seed=17, pad=3)
     g, par, nbr, tok = case.gpu_inputs(L)
     tree = L.Tree(case.parent)
-    assert L.verify_tree_path(par, tree) == 1 and L.sample_draft_tree_path(par) == 1
+    B = case.B
+    assert L.verify_tree_path(par, tree, B) == 1 and L.sample_draft_tree_path(par, tree, B) == 1
     par_dense = L.Params(**{**par.__dict__, "top_k_target": 0, "top_k_draft": 0})
-    assert L.verify_tree_path(par_dense, tree) == 2 and L.sample_draft_tree_path(par_dense) == 2      # streaming kernels
+    assert L.verify_tree_path(par_dense, tree, B) == 2 and L.sample_draft_tree_path(par_dense, tree, B) == 2      # streaming kernels (forced)
+    par_auto = L.Params(**{**par_dense.__dict__, "kernels": 0})
+    assert L.verify_tree_path(par_auto, tree, B) == 0 and L.sample_draft_tree_path(par_auto, tree, B) == 0    # a small call
+    assert L.verify_tree_path(par_auto, tree, 64) == 2 and L.sample_draft_tree_path(par_auto, tree, 64) == 2
     par_walk = L.Params(**{**par.__dict__, "lazy_walk": 1})
-    assert L.verify_tree_path(par_walk, tree) == 0            # top-k rows walk with the dense kernel
+    assert L.verify_tree_path(par_walk, tree, B) == 0         # top-k rows walk with the dense kernel
     old = L.set_cluster_size(1)
     try:
-        assert L.verify_tree_path(par, tree) == 0
+        assert L.verify_tree_path(par, tree, B) == 0
     finally:
         L.set_cluster_size(old)
     ua, ur = case.u_accept.cuda(), case.u_resample.cuda()
@@ -383,7 +395,7 @@ def test_path_walk_with_a_rule_variant_runs_on_the_streaming_kernel(L):
     eager = L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"],
                           tok, ua, ur, debug=True)
     par.lazy_walk = 1
-    assert L.verify_tree_path(par, tree) == 2
+    assert L.verify_tree_path(par, tree, case.B) == 2
     lazy = L.verify_tree(par, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"],
                          tok, ua, ur, debug=True)
     torch.cuda.synchronize()
