@@ -218,6 +218,71 @@ def cpu_baseline(cfg, parent, budget_s=10.0):
                       "together" % (cfg.name, budget_s, n1, t1, used)}
 
 
+def parity_sample(L, W, cfg, parent, lg, nbr, seq_ids):
+    """Near-tie accounting on the benchmarked workload (part of the CPU-baseline leg: it runs the
+    oracle): a few sequences of one input set go through the same kernels with explicit uniforms
+    and are compared with the oracle under the near-tie rule.  Returns the counts per class."""
+    import numpy as np
+    import torch
+    import oracle
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from parity_util import KEY_TIE, check_walk, compare_verify
+    N, V, n = len(parent), cfg.vocab, len(seq_ids)
+    dev = lg["target_cond"].device
+    idx = torch.tensor(seq_ids, device=dev)
+    sub = {k: (None if v is None else v.index_select(0, idx).contiguous()) for k, v in lg.items()}
+    cpu = {k: (None if v is None else v.float().cpu().numpy()) for k, v in sub.items()}
+    gum = W.make_gumbel_uniforms(n, N, V, 777)
+    ua, ur = W.make_uniforms(n, N, 778)
+    tree = L.Tree(parent)
+    par = L.Params(vocab=V, cfg_scale=cfg.cfg_scale if cfg.cfg_scale is not None else 1.0, temperature=cfg.temperature,
+                   top_k_target=cfg.top_k, top_k_draft=cfg.top_k, lam=cfg.lam, k=cfg.k, code_offset=cfg.code_offset,
+                   n_codes=cfg.codebook_size, kernels=1)
+    tok = L.sample_draft_tree(par, tree, sub["draft_cond"], sub["draft_uncond"], gumbel_uniforms=gum.to(dev))
+    res = L.verify_tree(par, tree, nbr, sub["target_cond"], sub["target_uncond"], sub["draft_cond"], sub["draft_uncond"],
+                        tok, ua.to(dev), ur.to(dev), debug=True)
+    torch.cuda.synchronize()
+    res = {k: v.cpu().numpy() for k, v in res.items()}
+    gtok = tok.cpu().numpy()
+    nbr_np = nbr.cpu().numpy()
+    kw = dict(cfg_scale=par.cfg_scale, temperature=cfg.temperature)
+    vkw = dict(top_k_target=cfg.top_k, top_k_draft=cfg.top_k, lam=cfg.lam, k=cfg.k, code_offset=cfg.code_offset,
+               n_codes=cfg.codebook_size, **kw)
+    children = oracle.tree_children(parent)
+    sampler_ties, orc = 0, []
+    for i in range(n):
+        g = lambda name: None if cpu[name] is None else cpu[name][i]
+        otok, _ = oracle.sample_draft_tree(parent, g("draft_cond"), g("draft_uncond"), gum[i].numpy(),
+                                           top_k_draft=cfg.top_k, **kw)
+        for node in range(N):
+            kids = children[node]
+            if kids and [int(gtok[i, c]) for c in kids] != [int(otok[c]) for c in kids]:
+                p_row, _ = oracle.postprocess_row(g("draft_cond")[node], None if g("draft_uncond") is None else g("draft_uncond")[node],
+                                                  kw["cfg_scale"], cfg.temperature, cfg.top_k)
+                _, _, gaps = oracle.sample_children(p_row, gum[i][node].numpy(), len(kids), return_gaps=True)
+                if min(gaps) >= KEY_TIE:
+                    raise AssertionError(("draft sampler differs from the oracle", seq_ids[i], node))
+                sampler_ties += 1
+        # the verifier is compared on the device's drafts (they are the oracle's unless a key near-tie was counted)
+        orc.append(oracle.verify_sequence(parent, g("target_cond"), g("target_uncond"), g("draft_cond"), g("draft_uncond"),
+                                          gtok[i].astype(np.int64), ua[i].numpy(), ur[i].numpy(), nbr_np, **vkw))
+
+    def rerun(b, node, forced):
+        g = lambda name: None if cpu[name] is None else cpu[name][b][node]
+        q, _ = oracle.postprocess_row(g("target_cond"), g("target_uncond"), kw["cfg_scale"], cfg.temperature, cfg.top_k)
+        pd = None
+        if children[node]:
+            pd, _ = oracle.postprocess_row(g("draft_cond"), g("draft_uncond"), kw["cfg_scale"], cfg.temperature, cfg.top_k)
+        return oracle.verify_node(q, pd, children[node], gtok[b].astype(np.int64), ua[b].numpy(), ur[b].numpy()[node], nbr_np,
+                                  cfg.k, cfg.lam, cfg.code_offset, cfg.codebook_size, forced=forced)
+
+    stats = compare_verify(res, orc, parent, ua.numpy(), rerun=rerun)
+    check_walk(res, gtok, tree.max_depth, orc, stats["dirty_sequences"], None, stats["patched"])
+    return {"sequences": n, "nodes": stats["nodes"], "tested_children": stats["tested"], "tie_accept": stats["tie_accept"],
+            "tie_cut": stats["tie_cut"], "tie_resample": stats["tie_resample"], "tie_sampler_key": sampler_ties,
+            "rule": "integers exact; a difference counts as a tie only where the oracle's margin is below 1e-6"}
+
+
 def run_reference(args, cfg, parent):
     """--impl reference: the CPU oracle on bounded samples of the same workload."""
     import workloads as W
@@ -647,6 +712,9 @@ def main():
     launches_per_step = vl + sl
     table = {"ms": w.table_ms, "L": cfg.codebook_size, "d": cfg.codebook_dim, "k": cfg.k, "dtype": cfg.codebook_dtype}
     set_bytes = w.set_bytes
+    parity = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.walk == "eager":
+        parity = parity_sample(L, W, cfg, parent, w.bufs[0], w.nbr, sorted({0, B // 2}))
     del w
     torch.cuda.empty_cache()
 
@@ -702,6 +770,8 @@ def main():
                 "builds": [[r["L"], r["d"], r["k"], r["ms"], round(r["contraction_tflops"], 2), r["path"]] for r in rows],
                 "columns": ["L", "d", "k", "ms", "contraction TFLOP/s (2 L^2 d / time)", "path"]}
             line["configs"] = cfgs
+        if parity is not None:
+            line["stats"]["parity_sample"] = parity
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(cfg, parent)
         print(json.dumps(line))

@@ -412,3 +412,57 @@ def test_variants_are_refused_on_topk_rows(L):
         with pytest.raises(L.LanternError) as e:
             L.verify_tree(bad, tree, nbr, g["target_cond"], g["target_uncond"], g["draft_cond"], g["draft_uncond"], tok)
         assert e.value.status == 2
+
+
+@pytest.mark.parametrize("kernels", [1, 2])
+def test_emitted_token_follows_the_relaxed_law_chi_square(L, kernels):
+    """V = 16, a root with two children, the library's own Philox for the drafts, the accept tests
+    and the residual draw: over 2^18 independent sequences the first emitted token follows the law
+    that the sibling loop defines, enumerated exactly with the oracle over all ordered draft pairs
+    (weights p_a p_b / (1 - p_a): sampling without replacement)."""
+    V, B, k, lam = 16, 1 << 18, 3, 2.0
+    g = torch.Generator().manual_seed(11)
+    zq = (torch.randn(V, generator=g) * 1.3).float()
+    zp = (zq * 0.8 + torch.randn(V, generator=g) * 0.6).float()
+    cb = W.make_codebook(V, 3, "f32", seed=5)
+    nbr, _ = oracle.neighbor_table(cb.to(torch.float64).numpy(), k)
+    q, _ = oracle.postprocess_row(zq.numpy(), None, 1.0, 1.0, 0)
+    p, _ = oracle.postprocess_row(zp.numpy(), None, 1.0, 1.0, 0)
+    law = np.zeros(V)
+    for a in range(V):
+        for b in range(V):
+            if a == b:
+                continue
+            w = p[a] * p[b] / (1.0 - p[a])
+            _, q_fin, tested = oracle.sibling_loop(q, p, [1, 2], [0, a, b], [0.0, 1.0, 1.0], nbr, k, lam, 0, V)
+            t1, t2 = tested[1][1], tested[2][1]
+            law[a] += w * t1
+            law[b] += w * (1 - t1) * t2
+            law += w * (1 - t1) * (1 - t2) * q_fin
+    assert abs(law.sum() - 1.0) < 1e-12
+    parent = [-1, 0, 0]
+    tree = L.Tree(parent)
+    tq = zq.cuda().repeat(3, 1).view(1, 3, V).expand(B, 3, V)          # stride 0 over the sequences
+    tp = zp.cuda().repeat(3, 1).view(1, 3, V).expand(B, 3, V)
+    par = L.Params(vocab=V, lam=lam, k=k, n_codes=V, seed=2024, step=3, kernels=kernels)
+    tok = L.sample_draft_tree(par, tree, tp, None)
+    out = L.verify_tree(par, tree, torch.from_numpy(nbr.astype(np.int32)).cuda(), tq, None, tp, None, tok)
+    torch.cuda.synchronize()
+    first = out["out_tokens"][:, 0].cpu().numpy()
+    counts = np.bincount(first, minlength=V).astype(np.float64)
+    chi2 = ((counts - B * law) ** 2 / (B * law)).sum()
+    assert chi2 < 50.0, (chi2, counts / B, law)            # 15 degrees of freedom: P(chi2 > 50) ~ 1e-5
+    # and it is not the unrelaxed law: the relaxation is visible at this sample size
+    plain = np.zeros(V)
+    for a in range(V):
+        for b in range(V):
+            if a == b:
+                continue
+            w = p[a] * p[b] / (1.0 - p[a])
+            _, q_fin, tested = oracle.sibling_loop(q, p, [1, 2], [0, a, b], [0.0, 1.0, 1.0], nbr, 0, 1.0, 0, V)
+            t1, t2 = tested[1][1], tested[2][1]
+            plain[a] += w * t1
+            plain[b] += w * (1 - t1) * t2
+            plain += w * (1 - t1) * (1 - t2) * q_fin
+    assert np.allclose(plain, q, atol=1e-12)               # standard speculative sampling emits q
+    assert ((counts - B * plain) ** 2 / (B * plain)).sum() > 200.0
