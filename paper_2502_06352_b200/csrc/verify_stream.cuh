@@ -379,20 +379,39 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
                           : uniform_halfopen(philox_stream(a.seed, a.step, static_cast<uint32_t>(out_b + fc + tid), kStreamAccept, 0).x);
   }
   // ---- gather: raw logits at every draft token and at its neighbours, 4-byte asynchronous
-  // copies into shared memory (in flight during the streaming pass)
+  // copies into shared memory (in flight during the streaming pass).  The children's tokens are
+  // staged first; the entries (child, list position) are then spread over all threads, four per
+  // thread at a time with their table reads issued together, so the chain token -> neighbour ->
+  // logit is walked once per node, not once per child.
+  int* ctok = sm.misc + 24;               // [LANTERN_MAX_CHILDREN] the children's draft tokens
+  if (tid < nc) ctok[tid] = tok_b[fc + tid];
+  __syncthreads();
   bool bad = false;
-  for (int ci = 0; ci < nc; ++ci) {
-    const int x = tok_b[fc + ci];
-    if (x < 0 || x >= a.V) continue;
-    const int code = x - a.code_offset;
-    const bool has_code = a.k > 0 && code >= 0 && code < a.n_codes;
-    const int cnt = has_code ? kp1 : 1;
-    for (int r = tid; r < cnt; r += ST) {
-      int t = x;
-      if (r > 0) t = a.code_offset + __ldg(a.nbr + static_cast<long long>(code) * a.k_table + (r - 1));
+  const int n_ent = nc * kp1;
+  for (int e0 = tid; e0 < n_ent; e0 += 4 * ST) {
+    int tt[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int e = e0 + i * ST;
+      tt[i] = -2;                                             // no such entry
+      if (e < n_ent) {
+        const int ci = e / kp1, r = e - ci * kp1;
+        const int x = ctok[ci];
+        const int code = x - a.code_offset;
+        if (x >= 0 && x < a.V) {
+          if (r == 0) tt[i] = x;
+          else if (a.k > 0 && code >= 0 && code < a.n_codes)
+            tt[i] = a.code_offset + __ldg(a.nbr + static_cast<long long>(code) * a.k_table + (r - 1));
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int e = e0 + i * ST;
+      if (e >= n_ent) continue;
+      const int t = tt[i];
       const bool ok = t >= 0 && t < a.V;
-      bad |= !ok;
-      const int e = ci * kp1 + r;
+      bad |= !ok && t != -2;
       sm.tok[e] = ok ? t : -1;
       if (ok) {
         const int w = sizeof(T) == 4 ? t : (t & ~1);
@@ -458,23 +477,67 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
       if (has_p) edge_sum(iop, ge, vbeg, vend, mx[1], sx[1]);
     }
   }
-  // common references, then the sums relative to them
-  float gm[2] = {warp_max(mx[0]), warp_max(mx[1])};
-  combine<2, true>(c, gm);
+  // one combination for both rows: per-warp (reference, sum) pairs -> CTA -> cluster; the sums are
+  // rescaled to the common reference in a fixed order, so every thread gets the same values
+  float gm[2], ws[2];
+  {
+    float wm[2] = {warp_max(mx[0]), warp_max(mx[1])};
+    float wsum[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+      wsum[i] = warp_sum(mx[i] == -INFINITY ? 0.f : sx[i] * ex2_approx((mx[i] - wm[i]) * kLog2e));
+    float* red = c.red + c.parity * (SW * 4);
+    if (lane == 0) { red[warp * 4] = wm[0]; red[warp * 4 + 1] = wsum[0]; red[warp * 4 + 2] = wm[1]; red[warp * 4 + 3] = wsum[1]; }
+    __syncthreads();
+    float cm[2] = {-INFINITY, -INFINITY}, cs2[2] = {0.f, 0.f};
+    for (int w2 = 0; w2 < SW; ++w2) { cm[0] = fmaxf(cm[0], red[w2 * 4]); cm[1] = fmaxf(cm[1], red[w2 * 4 + 2]); }
+    for (int w2 = 0; w2 < SW; ++w2) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const float m2 = red[w2 * 4 + 2 * i];
+        if (m2 != -INFINITY) cs2[i] += red[w2 * 4 + 2 * i + 1] * ex2_approx((m2 - cm[i]) * kLog2e);
+      }
+    }
+    gm[0] = cm[0]; gm[1] = cm[1]; ws[0] = cs2[0]; ws[1] = cs2[1];
+    if (c.nrank > 1) {
+      if (tid == 0) { c.xch[c.parity * 4] = cm[0]; c.xch[c.parity * 4 + 1] = cs2[0]; c.xch[c.parity * 4 + 2] = cm[1]; c.xch[c.parity * 4 + 3] = cs2[1]; }
+      cluster_sync();
+      float rm[2] = {-INFINITY, -INFINITY}, rs[2] = {0.f, 0.f};
+      for (uint32_t r = 0; r < c.nrank; ++r) {
+        const uint32_t base = dsmem_addr(smem_u32(&c.xch[c.parity * 4]), r);
+        const float v0 = dsmem_ld_f32(base), v1 = dsmem_ld_f32(base + 4), v2 = dsmem_ld_f32(base + 8), v3 = dsmem_ld_f32(base + 12);
+        if (tid == 0) { c.gath[r * 4] = v0; c.gath[r * 4 + 1] = v1; c.gath[r * 4 + 2] = v2; c.gath[r * 4 + 3] = v3; }
+        rm[0] = fmaxf(rm[0], v0); rm[1] = fmaxf(rm[1], v2);
+      }
+      for (uint32_t r = 0; r < c.nrank; ++r) {
+        const uint32_t base = dsmem_addr(smem_u32(&c.xch[c.parity * 4]), r);
+        const float v0 = dsmem_ld_f32(base), v1 = dsmem_ld_f32(base + 4), v2 = dsmem_ld_f32(base + 8), v3 = dsmem_ld_f32(base + 12);
+        if (v0 != -INFINITY) rs[0] += v1 * ex2_approx((v0 - rm[0]) * kLog2e);
+        if (v2 != -INFINITY) rs[1] += v3 * ex2_approx((v2 - rm[1]) * kLog2e);
+      }
+      gm[0] = rm[0]; gm[1] = rm[1]; ws[0] = rs[0]; ws[1] = rs[1];
+    }
+    // commit: the current target is q_0 (unnormalised, relative to gm[0])
+    if (tid < SW) {
+      const float m2 = red[tid * 4];
+      sm.wpart[tid] = m2 == -INFINITY ? 0.f : red[tid * 4 + 1] * ex2_approx((m2 - gm[0]) * kLog2e);
+    }
+    if (tid < static_cast<int>(c.nrank)) {
+      if (c.nrank > 1) {
+        const uint32_t base = dsmem_addr(smem_u32(&c.xch[c.parity * 4]), tid);
+        const float v0 = dsmem_ld_f32(base), v1 = dsmem_ld_f32(base + 4);
+        sm.rtot[tid] = v0 == -INFINITY ? 0.f : v1 * ex2_approx((v0 - gm[0]) * kLog2e);
+      } else {
+        sm.rtot[0] = ws[0];
+      }
+    }
+    c.parity ^= 1;
+  }
   if (gm[0] == -INFINITY || (has_p && gm[1] == -INFINITY)) {
     if (writer) vflag(a.status, LANTERN_DEV_EMPTY_ROW);
   }
   if (gm[0] == -INFINITY) gm[0] = 0.f;
   if (gm[1] == -INFINITY) gm[1] = 0.f;
-  float ws[2];
-  ws[0] = warp_sum(mx[0] == -INFINITY ? 0.f : sx[0] * ex2_approx((mx[0] - gm[0]) * kLog2e));
-  ws[1] = warp_sum(mx[1] == -INFINITY ? 0.f : sx[1] * ex2_approx((mx[1] - gm[1]) * kLog2e));
-  if (lane == 0) sm.wtmp[warp] = ws[0];
-  combine<2, false>(c, ws);
-  if (warp == 0) {                       // commit: the current target is q_0 (unnormalised)
-    if (lane < SW) sm.wpart[lane] = sm.wtmp[lane];
-    if (lane < static_cast<int>(c.nrank)) sm.rtot[lane] = c.gath[lane * 2];
-  }
   const float rq = ws[0] > 0.f ? 1.f / ws[0] : 0.f;
   const float rp = ws[1] > 0.f ? 1.f / ws[1] : 0.f;
   Cur cur;
@@ -488,30 +551,23 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
   // ---- gathered words -> (q_0, p_0) of every draft token and neighbour
   cp_async_wait<0>();
   __syncthreads();
-  for (int ci = 0; ci < nc; ++ci) {
-    const int x = tok_b[fc + ci];
-    if (x < 0 || x >= a.V) continue;
-    const int code = x - a.code_offset;
-    const int cnt = (a.k > 0 && code >= 0 && code < a.n_codes) ? kp1 : 1;
-    for (int r = tid; r < cnt; r += ST) {
-      const int e = ci * kp1 + r;
-      const int t = sm.tok[e];
-      float q0 = 0.f, p0 = 0.f;
-      if (t >= ge.alo && t < ge.ahi) {
-        const uint32_t* w = reinterpret_cast<const uint32_t*>(sm.ent + e * NOPS);
-        float v[4];
+  for (int e = tid; e < n_ent; e += ST) {
+    const int t = sm.tok[e];
+    float q0 = 0.f, p0 = 0.f;
+    if (t >= ge.alo && t < ge.ahi) {
+      const uint32_t* w = reinterpret_cast<const uint32_t*>(sm.ent + e * NOPS);
+      float v[4];
 #pragma unroll
-        for (int o = 0; o < NOPS; ++o) {
-          const uint32_t raw = w[o];
-          v[o] = sizeof(T) == 4 ? __uint_as_float(raw) : __uint_as_float((t & 1) ? (raw & 0xffff0000u) : (raw << 16));
-        }
-        const float zq = ioq.z1(v[0], CFG ? v[2] : 0.f);
-        q0 = ex2_approx(fmaf(zq, kLog2e, cur.cq)) * rq;
-        if (has_p) p0 = ex2_approx(fmaf(ioq.z1(v[1], CFG ? v[3] : 0.f), kLog2e, cur.cp)) * rp;
+      for (int o = 0; o < NOPS; ++o) {
+        const uint32_t raw = w[o];
+        v[o] = sizeof(T) == 4 ? __uint_as_float(raw) : __uint_as_float((t & 1) ? (raw & 0xffff0000u) : (raw << 16));
       }
-      sm.ent[e * NOPS] = q0;
-      sm.ent[e * NOPS + 1] = p0;
+      const float zq = ioq.z1(v[0], CFG ? v[2] : 0.f);
+      q0 = ex2_approx(fmaf(zq, kLog2e, cur.cq)) * rq;
+      if (has_p) p0 = ex2_approx(fmaf(ioq.z1(v[1], CFG ? v[3] : 0.f), kLog2e, cur.cp)) * rp;
     }
+    sm.ent[e * NOPS] = q0;
+    sm.ent[e * NOPS + 1] = p0;
   }
   __syncthreads();
 
@@ -521,7 +577,7 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
   int accepted = -1;
   for (int ci = 0; ci < nc; ++ci) {
     const int child = fc + ci;
-    const int x = tok_b[child];
+    const int x = ctok[ci];
     if (accepted >= 0 || x < 0 || x >= a.V) {
       if (accepted < 0 && x >= a.V && writer) vflag(a.status, LANTERN_DEV_BAD_INDEX);
       if (writer) {
@@ -536,20 +592,51 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
     const int* tk = sm.tok + ci * kp1;
     bool x_dropped = false;
     for (int d = 0; d < n_dropped; ++d) x_dropped |= dropped[d] == x;
+    // current target at entry r: exception tokens are zero
+    auto val = [&](int r) -> float {
+      const int t = tk[r];
+      if (t < 0) return 0.f;
+      if ((sm.bits[t >> 5] >> (t & 31)) & 1u) return 0.f;
+      return fmaxf(fmaf(-alpha, en[r * NOPS + 1], en[r * NOPS]), 0.f) * ibeta;
+    };
+    // Prefix rule over lists of up to 32 * SW entries, all warps at once: warp w scans entries
+    // [32w, 32w + 32); with the sums of the warps before it (added in list order, as the one-warp
+    // loop below does) it finds its first entry that would break the bound; the first warp that
+    // has one ends the prefix.
+    const bool par = has_code && !skip && a.k <= 32 * SW;
+    float* pcum = reinterpret_cast<float*>(sm.memb + 8);          // (the member mask is unused without skip)
+    if (par) {
+      const int r = warp * 32 + lane;
+      const float incl = warp_incl_scan(r < a.k ? val(1 + r) : 0.f, lane);
+      if (lane == 31) sm.scan[warp] = incl;
+      __syncthreads();
+      const float qx = val(0);
+      const float bound = a.delta > 0.f ? qx + a.delta : a.lambda * qx;
+      float base = qx;
+      for (int w2 = 0; w2 < warp; ++w2) base += sm.scan[w2];
+      const uint32_t ballot = __ballot_sync(0xffffffffu, r < a.k && (base + incl < bound));
+      const int ntake = __ffs(~ballot) - 1;
+      const int take = ntake < 0 ? 32 : ntake;
+      const float upto = take > 0 ? base + __shfl_sync(0xffffffffu, incl, take - 1) : base;
+      if (lane == 0) { sm.memb[warp] = static_cast<uint32_t>(take); pcum[warp] = upto; }
+      __syncthreads();
+    }
     if (warp == 0) {
-      // current target at entry r: exception tokens are zero
-      auto val = [&](int r) -> float {
-        const int t = tk[r];
-        if (t < 0) return 0.f;
-        if ((sm.bits[t >> 5] >> (t & 31)) & 1u) return 0.f;
-        return fmaxf(fmaf(-alpha, en[r * NOPS + 1], en[r * NOPS]), 0.f) * ibeta;
-      };
       const float qx = val(0);
       const float px = det ? 1.f : (x_dropped ? 0.f : en[1] * iW);
       const float bound = a.delta > 0.f ? qx + a.delta : a.lambda * qx;      // Sec. 2.2 / Sec. 4
       float cum = qx;
       int nA = 0;
       bool open = has_code;
+      if (par) {
+        for (int w2 = 0; w2 < SW && open; ++w2) {
+          const int take = static_cast<int>(sm.memb[w2]);
+          nA += take;
+          cum = pcum[w2];
+          if (take < 32) open = false;
+        }
+        open = false;
+      }
       if (skip && open) {
         // greedy-skip rule: a neighbour that would break the bound is passed over and the list
         // is searched on; the running sum is sequential, 32 entries at a time through shuffles
@@ -715,21 +802,32 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
       const float excl = before + (lane > 0 ? prev : 0.f);
       const float inc2 = before + incl;
       const bool mine = !fallback && !(E0 + excl > target) && (E0 + inc2 > target);
+      if (mine) {                                  // at most one thread: its piece holds the draw
+        sm.misc[4] = mb;
+        sm.misc[5] = me;
+        sm.misc[6] = lastpos;
+        fm[1] = E0 + excl;
+      }
       const int any = __syncthreads_or(mine ? 1 : 0);
-      if (mine) {
-        float run = E0 + excl;
+      if (any && warp == 0) {
+        // the 32 lanes walk that piece together, one token per lane and step
+        const int t0 = ge.j0 + sm.misc[4] * VN, t1 = ge.j0 + sm.misc[5] * VN;
+        float run = fm[1];
         int found = -1;
-        for (int vv = mb; vv < me && found < 0; ++vv) {
-          float tv[VN];
-          vec_terms(ioq, iop, ge, cur, sm.bits, vv, tv);
-#pragma unroll
-          for (int e = 0; e < VN; ++e) {
-            run += tv[e];
-            if (found < 0 && tv[e] > 0.f && run > target) found = ge.j0 + vv * VN + e;
+        for (int tb = t0; tb < t1 && found < 0; tb += 32) {
+          const int t = tb + lane;
+          float v = 0.f;
+          if (t < t1 && t >= ge.alo && t < ge.ahi && !((sm.bits[t >> 5] >> (t & 31)) & 1u)) {
+            v = ex2_approx(fmaf(ioq.z_at(t), kLog2e, cur.cq)) * cur.aq;
+            if (cur.has_p) v = fmaxf(fmaf(-ex2_approx(fmaf(iop.z_at(t), kLog2e, cur.cp)), cur.ap, v), 0.f);
           }
+          const float incl2 = warp_incl_scan(v, lane);
+          const uint32_t hit = __ballot_sync(0xffffffffu, v > 0.f && run + incl2 > target);
+          if (hit) found = tb + __ffs(hit) - 1;
+          run += __shfl_sync(0xffffffffu, incl2, 31);
         }
-        if (found < 0) found = lastpos;
-        a.node_token[out_b + n] = found;
+        if (found < 0) found = sm.misc[6];
+        if (lane == 0) a.node_token[out_b + n] = found;
       }
       if (!any) {
         // last positive entry of the range
