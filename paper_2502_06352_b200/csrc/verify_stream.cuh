@@ -248,7 +248,10 @@ __device__ __forceinline__ void pass_residual(const IO& ioq, const IO& iop, cons
   constexpr int VN = IO::VN;
   const int hb = max(vbeg, ge.vi0), he = min(vend, ge.vi1);
   float a0 = 0.f, a1 = 0.f, p0 = 0.f, p1 = 0.f;
-  for (int base = hb; base < he; base += 32 * U) {
+  // Backwards: the end of the range was streamed last, so it is what L2 still holds.
+  const int n_it = he > hb ? (he - hb + 32 * U - 1) / (32 * U) : 0;
+  for (int it = n_it - 1; it >= 0; --it) {
+    const int base = hb + it * 32 * U;
     uint4 qc[U], qu[U], pc[U], pu[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
