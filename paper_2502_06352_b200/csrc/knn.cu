@@ -21,6 +21,8 @@ constexpr int kDC = 32;             // embedding dims staged per step
 struct KnnArgs {
   const void* cb;
   int L, d, k, QT, CAP, q_double;
+  int f32acc;        // filter distances accumulated in float32 with an error margin (small d)
+  float margin;      // 1 + 3 (d + 2) 2^-24: the filter keeps everything within this factor of tau
   int32_t* nbr_idx;
   float* nbr_dist;
 };
@@ -187,20 +189,73 @@ __global__ void __launch_bounds__(kKnnThreads) knn_kernel(const KnnArgs a) {
   const int q0 = blockIdx.x * QT;
   const int nq = min(QT, L - q0);
 
-  for (int i = tid; i < QT * d; i += kKnnThreads) {
-    int q = i / d, t = i - q * d;
-    float v = (q < nq) ? widen<T>(cb[static_cast<long long>(q0 + q) * d + t]) : 0.f;
-    if (a.q_double) qd[i] = static_cast<double>(v); else qf[i] = v;
+  const int dpad = (d + 7) & ~7;
+  if (a.f32acc) {
+    for (int i = tid; i < QT * dpad; i += kKnnThreads) {
+      int q = i / dpad, t = i - q * dpad;
+      qf[i] = (q < nq && t < d) ? widen<T>(cb[static_cast<long long>(q0 + q) * d + t]) : 0.f;
+    }
+  } else {
+    for (int i = tid; i < QT * d; i += kKnnThreads) {
+      int q = i / d, t = i - q * d;
+      float v = (q < nq) ? widen<T>(cb[static_cast<long long>(q0 + q) * d + t]) : 0.f;
+      if (a.q_double) qd[i] = static_cast<double>(v); else qf[i] = v;
+    }
   }
   if (tid < QT) { tau[tid] = INFINITY; cnt[tid] = 0; ovf[tid] = 0; }
   __syncthreads();
 
   constexpr int MAXQT = 8;
+  // d <= 8 (one chunk of dimensions): the candidate row of the next tile is fetched while this
+  // tile is being processed
+  float cnext[8];
+  const bool prefetch = a.f32acc && d <= 8;
+  auto fetch_row = [&](int row, float (&out)[8]) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t) out[t] = (row < L && t < d) ? widen<T>(cb[static_cast<long long>(row) * d + t]) : 0.f;
+  };
+  if (prefetch) fetch_row(tid, cnext);
   for (int base = 0; base < L; base += kKnnThreads) {
     double acc[MAXQT];
 #pragma unroll
     for (int q = 0; q < MAXQT; ++q) acc[q] = 0.0;
     const int ncand = min(kKnnThreads, L - base);
+    if (a.f32acc) {
+      // Filter distances in float32: every thread reads its candidate's row straight from global
+      // memory, eight dimensions at a time, against the query rows in shared memory.  The relative
+      // error of such a sum is below (d + 2) 2^-24, so with the margin applied to tau nothing
+      // that can belong to the exact top k is dropped; exact duplicates still give 0.
+      float accf[MAXQT];
+#pragma unroll
+      for (int q = 0; q < MAXQT; ++q) accf[q] = 0.f;
+      for (int db = 0; db < d; db += 8) {
+        float cv[8];
+        if (prefetch) {
+#pragma unroll
+          for (int t = 0; t < 8; ++t) cv[t] = cnext[t];
+          fetch_row(base + kKnnThreads + tid, cnext);
+        } else {
+#pragma unroll
+          for (int t = 0; t < 8; ++t)
+            cv[t] = (tid < ncand && db + t < d) ? widen<T>(cb[static_cast<long long>(base + tid) * d + db + t]) : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < MAXQT; ++q) {
+          if (q < QT) {
+            const float4 qa = *reinterpret_cast<const float4*>(qf + q * dpad + db);
+            const float4 qb = *reinterpret_cast<const float4*>(qf + q * dpad + db + 4);
+            const float qv[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+              const float diff = qv[t] - cv[t];
+              accf[q] = fmaf(diff, diff, accf[q]);
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < MAXQT; ++q) acc[q] = static_cast<double>(accf[q]);
+    } else
     for (int db = 0; db < d; db += kDC) {
       const int dc = min(kDC, d - db);
       __syncthreads();
@@ -250,8 +305,9 @@ __global__ void __launch_bounds__(kKnnThreads) knn_kernel(const KnnArgs a) {
       // keep everything <= the k-th smallest rounded distance
       if (tid == 0) {
         uint32_t tb = static_cast<uint32_t>(bq[k - 1] >> 32);
+        if (a.f32acc) tb = __float_as_uint(__fmul_ru(__uint_as_float(tb), a.margin));     // (non-negative floats order as their bits)
         int m = k;
-        while (m < n && static_cast<uint32_t>(bq[m] >> 32) == tb) ++m;
+        while (m < n && static_cast<uint32_t>(bq[m] >> 32) <= tb) ++m;
         tau[q] = __uint_as_float(tb);
         cnt[q] = m;
         if (m > CAP - kKnnThreads) ovf[q] = 1;      // ties at tau fill the buffer
@@ -326,9 +382,11 @@ extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_
   auto smem_for = [&](int qt, int qdouble) {
     return static_cast<size_t>(qt) * cap * 8 + static_cast<size_t>(cap) * 12 + 8 * 12 +
            static_cast<size_t>(kKnnThreads) * (kDC + 1) * 4 + static_cast<size_t>(qt) * 12 + 16 +
-           static_cast<size_t>(qt) * d * (qdouble ? 8 : 4);
+           static_cast<size_t>(qt) * ((d + 7) & ~7) * (qdouble ? 8 : 4);
   };
-  a.q_double = smem_for(a.QT, 1) <= 160 * 1024 ? 1 : 0;
+  a.f32acc = d <= 64 ? 1 : 0;
+  a.margin = 1.0f + 3.0f * static_cast<float>(d + 2) * 5.9604644775390625e-8f;
+  a.q_double = (!a.f32acc && smem_for(a.QT, 1) <= 160 * 1024) ? 1 : 0;
   while (a.QT > 1 && smem_for(a.QT, a.q_double) > 220 * 1024) a.QT /= 2;
   size_t smem = smem_for(a.QT, a.q_double);
   if (smem > 227 * 1024) return LANTERN_ERR_UNSUPPORTED;
