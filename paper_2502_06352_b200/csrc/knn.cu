@@ -65,6 +65,76 @@ __device__ __forceinline__ void bitonic_pair(double* dv, int* iv, int n) {
   }
 }
 
+// Cut-back of one query's candidate buffer without sorting it.  Entries are 64-bit words whose
+// upper half is a monotone 32-bit key of the filter distance.  A most-significant-digit radix
+// select (4 passes of 8 bits, shared-memory histogram) finds the k-th smallest key; `limit_of`
+// turns it into the largest key that may stay (k-th key plus the caller's error margin); the
+// entries up to that limit are compacted through `tmp` (order is irrelevant: the final ranking
+// sorts).  Returns the number kept; *kth_key_out receives the k-th smallest key.  n >= k.
+template <typename F>
+__device__ __forceinline__ int radix_cut(unsigned long long* bq, int n, int k, unsigned long long* tmp, uint32_t* hist,
+                                         int* sel, F&& limit_of, uint32_t* limit_out) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  uint32_t prefix = 0;
+  int rem = k;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int i = tid; i < 256; i += kKnnThreads) hist[i] = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += kKnnThreads) {
+      const uint32_t key = static_cast<uint32_t>(bq[i] >> 32);
+      if (pass == 0 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid < 32) {
+      uint32_t c8[8], s = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c8[i] = hist[lane * 8 + i]; s += c8[i]; }
+      uint32_t incl = s;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      const uint32_t before = incl - s;
+      if (before < static_cast<uint32_t>(rem) && static_cast<uint32_t>(rem) <= incl) {     // exactly one lane
+        uint32_t run = before;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (run < static_cast<uint32_t>(rem) && static_cast<uint32_t>(rem) <= run + c8[i]) {
+            sel[0] = lane * 8 + i;
+            sel[1] = rem - static_cast<int>(run);
+          }
+          run += c8[i];
+        }
+      }
+    }
+    __syncthreads();
+    prefix = (prefix << 8) | static_cast<uint32_t>(sel[0]);
+    rem = sel[1];
+    __syncthreads();
+  }
+  const uint32_t limit = limit_of(prefix);          // prefix is now the k-th smallest key
+  if (tid == 0) sel[2] = 0;
+  __syncthreads();
+  for (int i0 = 0; i0 < n; i0 += kKnnThreads) {
+    const int i = i0 + tid;
+    const unsigned long long e = i < n ? bq[i] : ~0ull;
+    const bool keep = i < n && static_cast<uint32_t>(e >> 32) <= limit;
+    const uint32_t m = __ballot_sync(0xffffffffu, keep);
+    int pos0 = 0;
+    if (lane == 0 && m) pos0 = atomicAdd(&sel[2], __popc(m));
+    pos0 = __shfl_sync(0xffffffffu, pos0, 0);
+    if (keep) tmp[pos0 + __popc(m & ((1u << lane) - 1u))] = e;
+  }
+  __syncthreads();
+  const int kept = sel[2];
+  for (int i = tid; i < kept; i += kKnnThreads) bq[i] = tmp[i];
+  *limit_out = limit;
+  __syncthreads();
+  return kept;
+}
+
 template <typename T>
 __device__ __forceinline__ double exact_dist(const T* __restrict__ cb, int d, int i, int j) {
   const T* a = cb + static_cast<long long>(i) * d;
@@ -180,7 +250,9 @@ __global__ void __launch_bounds__(kKnnThreads) knn_kernel(const KnnArgs a) {
   int* cnt = reinterpret_cast<int*>(tau + QT);
   int* ovf = cnt + QT;
   int* redi = ovf + QT;
-  unsigned char* qraw = reinterpret_cast<unsigned char*>(redi + 8);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(redi + 8);       // [256] radix-select histogram
+  int* sel = reinterpret_cast<int*>(hist + 256);               // [4]
+  unsigned char* qraw = reinterpret_cast<unsigned char*>(sel + 4);
   qraw += (16 - (reinterpret_cast<uintptr_t>(qraw) & 15)) & 15;
   double* qd = reinterpret_cast<double*>(qraw);
   float* qf = reinterpret_cast<float*>(qraw);
@@ -299,16 +371,13 @@ __global__ void __launch_bounds__(kKnnThreads) knn_kernel(const KnnArgs a) {
       int n = cnt[q];
       if (n <= CAP - kKnnThreads || ovf[q]) continue;     // uniform: cnt/ovf are shared
       unsigned long long* bq = buf + static_cast<size_t>(q) * CAP;
-      for (int i = n + tid; i < CAP; i += kKnnThreads) bq[i] = ~0ull;
-      __syncthreads();
-      bitonic_u64(bq, CAP);
-      // keep everything <= the k-th smallest rounded distance
+      // keep everything up to the k-th smallest filter distance (times the margin in float32 mode)
+      uint32_t limit;
+      const float margin = a.f32acc ? a.margin : 1.0f;
+      const int m = radix_cut(bq, min(n, CAP), k, reinterpret_cast<unsigned long long*>(sortd), hist, sel,
+                              [&](uint32_t kth) { return __float_as_uint(__fmul_ru(__uint_as_float(kth), margin)); }, &limit);
       if (tid == 0) {
-        uint32_t tb = static_cast<uint32_t>(bq[k - 1] >> 32);
-        if (a.f32acc) tb = __float_as_uint(__fmul_ru(__uint_as_float(tb), a.margin));     // (non-negative floats order as their bits)
-        int m = k;
-        while (m < n && static_cast<uint32_t>(bq[m] >> 32) <= tb) ++m;
-        tau[q] = __uint_as_float(tb);
+        tau[q] = __uint_as_float(limit);      // (non-negative floats order as their bits)
         cnt[q] = m;
         if (m > CAP - kKnnThreads) ovf[q] = 1;      // ties at tau fill the buffer
       }
@@ -367,7 +436,8 @@ extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_
     ta.nbr_idx = nbr_idx; ta.nbr_dist = nbr_dist;
     const int ld = d + kTcPad;
     const size_t tsm = static_cast<size_t>(kTcQT) * ta.CAP * 8 + static_cast<size_t>(kTcQT) * ld * 2 +
-                       static_cast<size_t>(2) * kTcCT * ld * 2 + 2 * kTcCT * 4 + 5 * kTcQT * 4 + 64;
+                       static_cast<size_t>(2) * kTcCT * ld * 2 + 2 * kTcCT * 4 + 5 * kTcQT * 4 + 64 +
+                       260 * 4 + static_cast<size_t>(ta.CAP) * 8;
     if (cudaFuncSetAttribute(knn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tsm)) != cudaSuccess)
       return LANTERN_ERR_CUDA;
     knn_tc_kernel<<<(L + kTcQT - 1) / kTcQT, kKnnThreads, tsm, st>>>(ta);
@@ -381,7 +451,7 @@ extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_
   a.QT = cap <= 1024 ? 8 : 4;
   auto smem_for = [&](int qt, int qdouble) {
     return static_cast<size_t>(qt) * cap * 8 + static_cast<size_t>(cap) * 12 + 8 * 12 +
-           static_cast<size_t>(kKnnThreads) * (kDC + 1) * 4 + static_cast<size_t>(qt) * 12 + 16 +
+           static_cast<size_t>(kKnnThreads) * (kDC + 1) * 4 + static_cast<size_t>(qt) * 12 + 16 + 260 * 4 +
            static_cast<size_t>(qt) * ((d + 7) & ~7) * (qdouble ? 8 : 4);
   };
   a.f32acc = d <= 64 ? 1 : 0;

@@ -104,6 +104,9 @@ __global__ void __launch_bounds__(kKnnThreads) knn_tc_kernel(const KnnTcArgs a) 
   float* eps2 = thr + kTcQT;
   int* cnt = reinterpret_cast<int*>(eps2 + kTcQT);
   int* ovf = cnt + kTcQT;
+  uint32_t* hist = reinterpret_cast<uint32_t*>(ovf + kTcQT);                            // [256] radix-select histogram
+  int* sel = reinterpret_cast<int*>(hist + 256);                                        // [4]
+  unsigned long long* cut_tmp = reinterpret_cast<unsigned long long*>(sel + 4);         // [CAP]
   // after the main loop the tile buffers are reused by the exact ranking
   double* sortd = reinterpret_cast<double*>(Bs);
   double* redd = sortd + CAP;
@@ -183,20 +186,15 @@ __global__ void __launch_bounds__(kKnnThreads) knn_tc_kernel(const KnnTcArgs a) 
       const int n = cnt[q];
       if (n <= CAP - kTcCT || ovf[q]) continue;            // uniform: shared values
       unsigned long long* bq = buf + static_cast<size_t>(q) * CAP;
-      for (int i = n + tid; i < CAP; i += kKnnThreads) bq[i] = ~0ull;
-      __syncthreads();
-      bitonic_u64(bq, CAP);
+      // keep everything within the error margin of the k-th smallest approximate distance
+      uint32_t limit;
+      const float e2 = eps2[q];
+      const int kept = radix_cut(bq, min(n, CAP), k, cut_tmp, hist, sel,
+                                 [&](uint32_t kth) { return float_key(key_float(kth) + e2); }, &limit);
       if (tid == 0) {
-        const float tau = key_float(static_cast<uint32_t>(bq[k - 1] >> 32));
-        const float th = tau + eps2[q];
-        int lo = k, hi = n;                                 // first index in [k, n) whose f exceeds th
-        while (lo < hi) {
-          const int mid = (lo + hi) >> 1;
-          if (key_float(static_cast<uint32_t>(bq[mid] >> 32)) <= th) lo = mid + 1; else hi = mid;
-        }
-        thr[q] = th;
-        cnt[q] = lo;
-        if (lo > CAP - kTcCT) ovf[q] = 1;                   // too many rows within the error margin
+        thr[q] = key_float(limit);
+        cnt[q] = kept;
+        if (kept > CAP - kTcCT) ovf[q] = 1;                 // too many rows within the error margin
       }
       __syncthreads();
     }

@@ -95,7 +95,7 @@ static int stream_cluster_size(int nodes, int V, bool f32) {
   if (g_cluster_override > 0) return g_cluster_override;
   const int nvec = V / (f32 ? 4 : 8);
   int cs = 1;
-  while (cs < 16 && static_cast<long long>(nodes) * cs < 4 * sm_count() && nvec / (2 * cs * stream::SW) >= 32) cs *= 2;
+  while (cs < 16 && static_cast<long long>(nodes) * cs < 8 * sm_count() && nvec / (2 * cs * stream::SW) >= 32) cs *= 2;
   return cs;
 }
 
