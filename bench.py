@@ -352,7 +352,8 @@ def table_sweep(with_oracle):
                 rows.append({"L": n, "d": d, "k": k, "ms": round(best, 3), "rows_per_s": n / (best * 1e-3),
                              "gbs": alg / (best * 1e-3) / 1e9, "contraction_tflops": 2.0 * n * n * d / (best * 1e-3) / 1e12,
                              "candidates_per_s": float(n) * n / (best * 1e-3),
-                             "path": "tensor" if (d % 16 == 0 and 32 <= d <= 256 and k <= 320) else "brute",
+                             "path": ("tcgen05" if (n >= 8192 and d % 8 == 0 and d <= 256 and k <= 320)
+                                      else "mma.sync" if (d % 16 == 0 and 32 <= d <= 256 and k <= 320) else "brute"),
                              "oracle_rows_per_s": None if t_or is None else 1.0 / t_or})
     return rows, SWEEP_DUP_FRAC
 

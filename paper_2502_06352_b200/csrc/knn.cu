@@ -65,13 +65,20 @@ __device__ __forceinline__ void bitonic_pair(double* dv, int* iv, int n) {
   }
 }
 
+template <int NT, int BAR>
+__device__ __forceinline__ void knn_bar() {
+  if (BAR == 0) __syncthreads();
+  else asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
+}
+
 // Cut-back of one query's candidate buffer without sorting it.  Entries are 64-bit words whose
 // upper half is a monotone 32-bit key of the filter distance.  A most-significant-digit radix
 // select (4 passes of 8 bits, shared-memory histogram) finds the k-th smallest key; `limit_of`
 // turns it into the largest key that may stay (k-th key plus the caller's error margin); the
 // entries up to that limit are compacted through `tmp` (order is irrelevant: the final ranking
 // sorts).  Returns the number kept; *kth_key_out receives the k-th smallest key.  n >= k.
-template <typename F>
+// NT threads (threadIdx.x < NT) take part and meet at hardware barrier BAR (0 = the whole CTA).
+template <int NT = kKnnThreads, int BAR = 0, typename F>
 __device__ __forceinline__ int radix_cut(unsigned long long* bq, int n, int k, unsigned long long* tmp, uint32_t* hist,
                                          int* sel, F&& limit_of, uint32_t* limit_out) {
   const int tid = threadIdx.x, lane = tid & 31;
@@ -79,13 +86,13 @@ __device__ __forceinline__ int radix_cut(unsigned long long* bq, int n, int k, u
   int rem = k;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    for (int i = tid; i < 256; i += kKnnThreads) hist[i] = 0;
-    __syncthreads();
-    for (int i = tid; i < n; i += kKnnThreads) {
+    for (int i = tid; i < 256; i += NT) hist[i] = 0;
+    knn_bar<NT, BAR>();
+    for (int i = tid; i < n; i += NT) {
       const uint32_t key = static_cast<uint32_t>(bq[i] >> 32);
       if (pass == 0 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
     }
-    __syncthreads();
+    knn_bar<NT, BAR>();
     if (tid < 32) {
       uint32_t c8[8], s = 0;
 #pragma unroll
@@ -109,15 +116,15 @@ __device__ __forceinline__ int radix_cut(unsigned long long* bq, int n, int k, u
         }
       }
     }
-    __syncthreads();
+    knn_bar<NT, BAR>();
     prefix = (prefix << 8) | static_cast<uint32_t>(sel[0]);
     rem = sel[1];
-    __syncthreads();
+    knn_bar<NT, BAR>();
   }
   const uint32_t limit = limit_of(prefix);          // prefix is now the k-th smallest key
   if (tid == 0) sel[2] = 0;
-  __syncthreads();
-  for (int i0 = 0; i0 < n; i0 += kKnnThreads) {
+  knn_bar<NT, BAR>();
+  for (int i0 = 0; i0 < n; i0 += NT) {
     const int i = i0 + tid;
     const unsigned long long e = i < n ? bq[i] : ~0ull;
     const bool keep = i < n && static_cast<uint32_t>(e >> 32) <= limit;
@@ -127,11 +134,11 @@ __device__ __forceinline__ int radix_cut(unsigned long long* bq, int n, int k, u
     pos0 = __shfl_sync(0xffffffffu, pos0, 0);
     if (keep) tmp[pos0 + __popc(m & ((1u << lane) - 1u))] = e;
   }
-  __syncthreads();
+  knn_bar<NT, BAR>();
   const int kept = sel[2];
-  for (int i = tid; i < kept; i += kKnnThreads) bq[i] = tmp[i];
+  for (int i = tid; i < kept; i += NT) bq[i] = tmp[i];
   *limit_out = limit;
-  __syncthreads();
+  knn_bar<NT, BAR>();
   return kept;
 }
 
@@ -397,6 +404,7 @@ __global__ void __launch_bounds__(kKnnThreads) knn_kernel(const KnnArgs a) {
 }  // namespace lantern
 
 #include "knn_tc.cuh"
+#include "knn_t5.cuh"
 
 using namespace lantern;
 
@@ -406,11 +414,26 @@ static bool use_tensor_path(lantern_dtype dt, int L, int d, int k) {
   return dt == LANTERN_BF16 && d % 16 == 0 && d >= 32 && d <= kTcMaxD && k <= 320 && L >= 64;
 }
 
+// bfloat16 codebooks of at least this many rows, d a multiple of 8 up to 256, take the tcgen05 kernel
+// (tiles of 128 queries per CTA); smaller ones would leave most SMs without a tile and stay on the
+// mma.sync kernel (or, for d it does not serve, on the brute-force kernel).
+#ifndef LANTERN_T5_MIN_L
+#define LANTERN_T5_MIN_L 8192
+#endif
+constexpr int kT5GridCap = 160;          // CTAs the workspace is sized for (one per SM)
+static bool use_t5_path(lantern_dtype dt, int L, int d, int k) {
+  return dt == LANTERN_BF16 && d % 8 == 0 && d >= 8 && d <= 256 && k <= kT5MaxK && L >= LANTERN_T5_MIN_L;
+}
+static size_t norms_bytes(int L) { return ((static_cast<size_t>(L) + 64) * sizeof(float) + 255) / 256 * 256; }
+static size_t t5_cta_bytes(int k) { return static_cast<size_t>(kT5Q) * knn_t5_cap(k) * 8; }
+
 extern "C" size_t lantern_build_neighbors_workspace(lantern_dtype dt, int32_t L, int32_t d, int32_t k) {
   if (L < 2 || d < 1 || k < 1) return 0;
-  // squared norms of all rows and their maximum (tensor-core path); the brute-force kernel
-  // keeps all of its state on chip
-  return use_tensor_path(dt, L, d, k) ? (static_cast<size_t>(L) + 64) * sizeof(float) : 0;
+  // squared norms of all rows and their maximum (tensor-core paths), plus the per-CTA candidate
+  // lists of the tcgen05 kernel; the brute-force kernel keeps all of its state on chip
+  if (!use_t5_path(dt, L, d, k)) return use_tensor_path(dt, L, d, k) ? norms_bytes(L) : 0;
+  const int nqt = (L + kT5Q - 1) / kT5Q;
+  return norms_bytes(L) + static_cast<size_t>(nqt < kT5GridCap ? nqt : kT5GridCap) * t5_cta_bytes(k);
 }
 
 extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_dtype dt, int32_t L, int32_t d,
@@ -421,7 +444,7 @@ extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_
   if (L < 2 || d < 1 || k < 1 || k > L - 1) return LANTERN_ERR_INVALID_ARG;
   if (k > 1024 || d > 4096) return LANTERN_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (use_tensor_path(dt, L, d, k)) {
+  if (use_t5_path(dt, L, d, k) || use_tensor_path(dt, L, d, k)) {
     const size_t need = lantern_build_neighbors_workspace(dt, L, d, k);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) % 256)) return LANTERN_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(codebook) % 16) return LANTERN_ERR_INVALID_ARG;
@@ -429,6 +452,27 @@ extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_
     if (cudaMemsetAsync(nrm + L, 0, sizeof(float), st) != cudaSuccess) return LANTERN_ERR_CUDA;
     knn_norms_kernel<<<(L * 32 + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(codebook), L, d, nrm);
     if (cudaGetLastError() != cudaSuccess) return LANTERN_ERR_CUDA;
+    if (use_t5_path(dt, L, d, k)) {
+      KnnT5Args fa;
+      fa.cb = static_cast<const __nv_bfloat16*>(codebook); fa.nrm = nrm; fa.L = L; fa.d = d; fa.k = k;
+      fa.CAP = knn_t5_cap(k);
+      fa.lists = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(workspace) + norms_bytes(L));
+      fa.nbr_idx = nbr_idx; fa.nbr_dist = nbr_dist;
+      int dev = 0, sms = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        return LANTERN_ERR_CUDA;
+      const long long afford = static_cast<long long>((workspace_bytes - norms_bytes(L)) / t5_cta_bytes(k));
+      int grid = (L + kT5Q - 1) / kT5Q;
+      if (grid > sms) grid = sms;
+      if (grid > afford) grid = static_cast<int>(afford);
+      if (grid < 1) return LANTERN_ERR_WORKSPACE;
+      const size_t fsm = knn_t5_smem(d, fa.CAP);
+      if (cudaFuncSetAttribute(knn_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fsm)) != cudaSuccess)
+        return LANTERN_ERR_CUDA;
+      knn_t5_kernel<<<grid, kT5Threads, fsm, st>>>(fa);
+      return cudaGetLastError() == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
+    }
     KnnTcArgs ta;
     ta.cb = static_cast<const __nv_bfloat16*>(codebook); ta.nrm = nrm; ta.L = L; ta.d = d; ta.k = k;
     ta.CAP = 256;

@@ -93,3 +93,31 @@ def test_sweep_largest_shapes_sampled_rows(L, n, d, k):
     dup_rows = np.nonzero(cnt[inv.ravel()] > 1)[0]
     rows += [int(x) for x in dup_rows[:3]]
     _check(L, cb, k, rows=rows)
+
+
+@pytest.mark.parametrize("n,d,k", [(8192, 8, 10), (8200, 24, 100), (8325, 48, 320), (9000, 80, 64), (8500, 128, 200),
+                                   (16384, 8, 100)])
+def test_tcgen05_kernel_ragged_tiles_sampled_rows(L, n, d, k):
+    """Shapes served by the tcgen05 kernel (bf16, at least 8192 rows): a ragged last query and
+    candidate tile (n not a multiple of 128), d below and between multiples of 16 (rows are
+    zero-padded on chip), the smallest and the largest k of that kernel; rows of the first, an
+    inner and the ragged last tile, and the -1 abort marker never appears."""
+    cb = W.make_codebook(n, d, "bf16", seed=n + k, dup_frac=0.05)
+    rng = np.random.default_rng(2)
+    rows = [0, 127, 128, n - 1, n - 2, ((n - 1) // 128) * 128] + [int(x) for x in rng.integers(0, n, 12)]
+    idx, _ = _check(L, cb, k, rows=rows)
+    assert idx.min() >= 0 and idx.max() < n and not np.any(idx == np.arange(n)[:, None])
+    s = np.sort(idx, axis=1)
+    assert np.all(s[:, 1:] != s[:, :-1])
+
+
+def test_tcgen05_kernel_overflowing_lists_take_the_exact_fallback(L):
+    """A block of 1200 equal rows inside a large codebook: their lists hold more rows within the
+    error margin than the exact ranking takes, so those queries go through the arg-min fallback;
+    ties by index."""
+    n, d, k = 8300, 32, 20
+    cb = W.make_codebook(n, d, "bf16", seed=9)
+    cb[1000:2200] = cb[1000]
+    idx, dist = _check(L, cb, k, rows=[0, 999, 1000, 1001, 1500, 2199, 2200, n - 1])
+    assert list(idx[1000]) == list(range(1001, 1021)) and list(idx[1500]) == list(range(1000, 1020))
+    assert np.all(dist[1000:2200] == 0)
