@@ -125,10 +125,15 @@ typedef struct {
  *   codebook  [L][d] row-major, dt = F32 or BF16            nbr_idx  [L][k] int32
  *   nbr_dist  [L][k] float32 squared distances, or NULL
  *   workspace device scratch of at least lantern_build_neighbors_workspace() bytes, 256-B aligned
- *             (row norms for the tensor-core path; 0 bytes when that path is not taken)
- * bfloat16 codebooks with d a multiple of 16 in [32, 256] and k <= 320 take a tensor-core path:
- * approximate distances from bf16 MMAs select a superset of the neighbours (with a proven error
- * margin), which is then ranked exactly.  Everything else takes an exact brute-force kernel.
+ *             (row norms, and for the tcgen05 kernel the candidate lists of its CTAs: up to
+ *             160 * 128 * (k + 128 + max(k, 192)) * 8 bytes; 0 bytes for the brute-force kernel)
+ * bfloat16 codebooks with k <= 320 take a tensor-core path: approximate distances from bf16 MMAs
+ * select a superset of the neighbours (with a proven error margin), which is then ranked exactly.
+ * L >= 8192 and d a multiple of 8 up to 256: tcgen05 MMAs with accumulators in tensor memory; the
+ * codebook must be 16-byte aligned.  Smaller L with d a multiple of 16 in [32, 256]: mma.sync.
+ * Everything else takes an exact brute-force kernel.  The table is the same whichever kernel
+ * builds it.  Every wait inside the tcgen05 kernel is bounded; should one run out, the rows of the
+ * affected query tiles are written as -1 (never observed; callers may check nbr_idx[i][0] >= 0).
  * Requires 1 <= k <= min(L-1, 1024), 1 <= d <= 4096.                                            */
 size_t lantern_build_neighbors_workspace(lantern_dtype dt, int32_t L, int32_t d, int32_t k);
 lantern_status lantern_build_neighbors(const void* codebook, lantern_dtype dt, int32_t L, int32_t d,
