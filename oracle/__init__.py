@@ -19,3 +19,4 @@ from .tree import tree_children  # noqa: F401
 from .verify import relaxed_mass, moved_mass, sibling_loop, inverse_cdf, verify_node, verify_sequence, walk, verify_batch  # noqa: F401
 from .sampler import sample_children, sample_draft_tree  # noqa: F401
 from .philox import philox4x32_10, uniform_open, uniform_halfopen, stream_uniforms  # noqa: F401
+from .dynamic_tree import top_children, expand_frontier, trim, breadth_first, draft_dynamic_tree  # noqa: F401
