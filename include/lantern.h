@@ -260,6 +260,50 @@ lantern_status lantern_verify_tree_static(const lantern_params* params, const la
                                           float* node_mass, float* node_thresh,
                                           int32_t* device_status, void* stream);
 
+/* ---- (5) dynamic-tree drafting -------------------------------------------------------------
+ * Sec. 2.1, the dynamic variant of tree drafting: every draft node t_i carries the global accept
+ * value V_i = product of the drafter's confidences c_j along the path from the root (the
+ * confidence of a token is its probability in the drafter's post-processed row); a depth of
+ * drafting gives every frontier node its n_children most confident tokens and keeps the n_expand
+ * candidates with the largest V as the next frontier; at the end the nodes are trimmed by V
+ * (Sec. 3: with low confidences the product decays fast and the tree stays shallow).  The tokens
+ * are chosen deterministically, so such a tree is verified with draft_deterministic = 1.
+ *
+ * A sequence's candidates live in a pool of pool_size entries (entry 0 = the root: the caller sets
+ * pool_parent = -1, pool_token = -1, pool_logv = 0, pool_depth = 0).  Values are kept as log V in
+ * double.  Equal values rank by lower index: tokens of a row by (z descending, token ascending),
+ * candidates by (log V descending, pool index ascending), so a parent ranks before its children.
+ *
+ * lantern_expand_frontier, one depth:
+ *   draft_cond / draft_uncond  drafter rows of the frontier nodes: row of slot f of sequence b at
+ *             b * seq_stride + f * row_stride (elements); uncond NULL = no guidance.  Post-processing
+ *             as for every other entry point (guidance, temperature, allowed range); top_k_draft
+ *             must be 0 (LANTERN_ERR_UNSUPPORTED otherwise)
+ *   frontier  [batch][n_frontier] pool index of the node in each slot, -1 = empty slot
+ *   pool_*    [batch][pool_size]; the n_frontier * n_children candidates of this depth are written
+ *             at pool_offset + f * n_children + rank (parent = the slot's node, depth = `depth`,
+ *             log V = the parent's + ln c); candidates of empty slots get log V = -inf
+ *   next_frontier  [batch][n_expand] pool indices of the chosen candidates in rank order, -1 beyond
+ *             the number of candidates
+ * 1 <= n_children <= LANTERN_MAX_CHILDREN, n_frontier * n_children <= 2048, pool_size <= 2048.
+ *
+ * lantern_trim_tree: of the first pool_used entries keep the root and the max_nodes - 1 others with
+ * the largest log V, renumbered breadth first as lantern_tree_create wants them.
+ *   n_nodes [batch]; parent / token / pool_index / logv [batch][max_nodes] (unused tail: -1, -inf)
+ *   max_depth  the largest value in pool_depth (the number of depths drafted)                     */
+lantern_status lantern_expand_frontier(const lantern_params* params, const void* draft_cond,
+                                       const void* draft_uncond, lantern_dtype dt, int64_t row_stride,
+                                       int64_t seq_stride, int32_t batch, int32_t n_frontier,
+                                       int32_t n_children, int32_t n_expand, const int32_t* frontier,
+                                       int32_t pool_size, int32_t pool_offset, int32_t depth,
+                                       int32_t* pool_parent, int32_t* pool_token, double* pool_logv,
+                                       int32_t* pool_depth, int32_t* next_frontier, void* stream);
+lantern_status lantern_trim_tree(int32_t batch, int32_t pool_size, int32_t pool_used, int32_t max_depth,
+                                 const int32_t* pool_parent, const int32_t* pool_token,
+                                 const double* pool_logv, const int32_t* pool_depth, int32_t max_nodes,
+                                 int32_t* n_nodes, int32_t* parent, int32_t* token, int32_t* pool_index,
+                                 double* logv, void* stream);
+
 /* Raw Philox-4x32-10 words (Salmon et al., SC 2011) for counters (first + i, c1, c2, c3), i in
  * [0, n): out[i][0..3].  Exists so that the generator can be checked against other
  * implementations.  out is a device pointer to n*4 uint32.                                      */

@@ -17,5 +17,8 @@ from .binding import (  # noqa: F401
     set_cluster_size,
     verify_tree_path,
     sample_draft_tree_path,
+    DraftPool,
+    expand_frontier,
+    trim_tree,
     lib,
 )

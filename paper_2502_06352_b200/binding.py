@@ -107,6 +107,11 @@ def _load():
     L.lantern_verify_tree_path.argtypes = [ctypes.POINTER(_CParams), vp, i32]
     L.lantern_sample_draft_tree_path.restype = i32
     L.lantern_sample_draft_tree_path.argtypes = [ctypes.POINTER(_CParams), vp, i32]
+    L.lantern_expand_frontier.restype = ctypes.c_int
+    L.lantern_expand_frontier.argtypes = [ctypes.POINTER(_CParams), vp, vp, ctypes.c_int, i64, i64, i32, i32, i32, i32,
+                                          vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+    L.lantern_trim_tree.restype = ctypes.c_int
+    L.lantern_trim_tree.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     return L
 
 
@@ -265,6 +270,58 @@ def verify_tree_static(params: Params, tree: Tree, nbr_idx, target_cond, target_
             _ptr(out["out_nodes"]), _ptr(out.get("node_mass")), _ptr(out.get("node_thresh")),
             _ptr(device_status), _stream()), "lantern_verify_tree_static")
     return out
+
+
+class DraftPool:
+    """Candidate pool of dynamic-tree drafting: [B][P] parent / token / depth (int32) and log V
+    (float64) with entry 0 the root, plus the current frontier [B][F] of pool indices."""
+
+    def __init__(self, batch, n_depths, n_children, n_expand, device="cuda"):
+        self.B, self.K, self.E = batch, n_children, n_expand
+        # depth 1 expands the root alone, every later depth the n_expand chosen candidates
+        self.P = 1 + n_children + max(0, n_depths - 1) * n_expand * n_children
+        self.parent = torch.full((batch, self.P), -1, dtype=torch.int32, device=device)
+        self.token = torch.full((batch, self.P), -1, dtype=torch.int32, device=device)
+        self.depth = torch.zeros((batch, self.P), dtype=torch.int32, device=device)
+        self.logv = torch.full((batch, self.P), float("-inf"), dtype=torch.float64, device=device)
+        self.logv[:, 0] = 0.0
+        self.frontier = torch.zeros((batch, 1), dtype=torch.int32, device=device)
+        self.used, self.n_depths = 1, 0
+
+
+def expand_frontier(params: Params, pool: DraftPool, draft_cond, draft_uncond=None):
+    """lantern_expand_frontier: one depth of dynamic-tree drafting.  draft_cond [B][F][V] holds the
+    drafter rows of the nodes in pool.frontier (F = its width).  The pool and its frontier advance."""
+    B, F, V = pool.B, pool.frontier.shape[1], params.vocab
+    rs, ss = _rows(draft_cond, B, F, V)
+    if draft_uncond is not None and _rows(draft_uncond, B, F, V) != (rs, ss):
+        raise ValueError("cond and uncond rows must share strides")
+    nxt = torch.empty((B, pool.E), dtype=torch.int32, device=draft_cond.device)
+    cp = params.c()
+    with torch.cuda.device(draft_cond.device):
+        _check(lib.lantern_expand_frontier(
+            ctypes.byref(cp), _ptr(draft_cond), _ptr(draft_uncond), _dtype_code(draft_cond), rs, ss, B, F, pool.K, pool.E,
+            _ptr(pool.frontier), pool.P, pool.used, pool.n_depths + 1, _ptr(pool.parent), _ptr(pool.token),
+            _ptr(pool.logv), _ptr(pool.depth), _ptr(nxt), _stream()), "lantern_expand_frontier")
+    pool.used += F * pool.K
+    pool.n_depths += 1
+    pool.frontier = nxt
+    return nxt
+
+
+def trim_tree(pool: DraftPool, max_nodes: int):
+    """lantern_trim_tree: (n_nodes [B], parent, token, pool_index [B][max_nodes] int32, logv float64)."""
+    dev = pool.parent.device
+    n = torch.empty((pool.B,), dtype=torch.int32, device=dev)
+    parent = torch.empty((pool.B, max_nodes), dtype=torch.int32, device=dev)
+    token = torch.empty_like(parent)
+    index = torch.empty_like(parent)
+    logv = torch.empty((pool.B, max_nodes), dtype=torch.float64, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib.lantern_trim_tree(pool.B, pool.P, pool.used, pool.n_depths, _ptr(pool.parent), _ptr(pool.token),
+                                     _ptr(pool.logv), _ptr(pool.depth), max_nodes, _ptr(n), _ptr(parent), _ptr(token),
+                                     _ptr(index), _ptr(logv), _stream()), "lantern_trim_tree")
+    return n, parent, token, index, logv
 
 
 def philox_raw(seed, first, c1, c2, c3, n, device="cuda"):
