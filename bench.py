@@ -521,6 +521,55 @@ def config_entry(torch, L, W, cfg, dev, peak, allowed=None, use_graph=True, ring
     return ent
 
 
+def dynamic_tree_entry(torch, L, dev, peak):
+    """Dynamic-tree drafting (Sec. 2.1) on rows of the headline shape: B = 64 sequences, V = 65536 bf16 drafter rows,
+    6 depths, 8 children per node, frontier of 8, trimmed to 59 nodes (the node count the paper quotes for dynamic
+    trees); the frontier rows of a depth are synthetic stand-ins for the drafter's forward pass.  Timed: the six
+    expand calls and the trim as one CUDA graph, CUDA events around a replay, median of 20 after 3 warm-ups;
+    bytes = every frontier row once."""
+    B, V, D, K, E, m = 64, 65536, 6, 8, 8, 59
+    g = torch.Generator(device=dev).manual_seed(17)
+    rows = [(torch.randn((B, 1 if d == 0 else E, V), generator=g, device=dev) * 2.0).to(torch.bfloat16) for d in range(D)]
+    par = L.Params(vocab=V)
+    pool = L.DraftPool(B, D, K, E, device=dev)
+    root = pool.frontier
+
+    def run():
+        pool.used, pool.n_depths, pool.frontier = 1, 0, root
+        for d in range(D):
+            L.expand_frontier(par, pool, rows[d])
+        return L.trim_tree(pool, m)
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            run()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        n, parent, token, index, logv = run()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    for it in range(23):
+        ev0.record()
+        graph.replay()
+        ev1.record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            times.append(ev0.elapsed_time(ev1))
+    dep = torch.gather(pool.depth, 1, index.clamp(min=0).long()).float()
+    depth_mean = float((dep * (index >= 0)).sum() / (index >= 0).sum())
+    times.sort()
+    med = times[len(times) // 2]
+    alg = sum(int(r.numel()) * 2 for r in rows)
+    return {"workload": "f3_dynamic_tree: B=64, V=65536 bf16, 6 depths, top-8 children, frontier 8, trim to 59 nodes",
+            "kernels": "expand_rows_kernel + select_frontier_kernel (x6), trim_tree_kernel", "launches": 2 * D + 1,
+            "us_median": round(1e3 * med, 1), "us_min": round(1e3 * times[0], 1), "algorithmic_bytes": alg,
+            "gbs": round(alg / (med * 1e-3) / 1e9, 1), "frac_measured": round(alg / (med * 1e-3) / 1e9 / peak, 4),
+            "mean_nodes": float(n.float().mean()), "mean_node_depth": round(depth_mean, 3),
+            "note": "two passes per row (HBM, then L2); instruction-bound (about 20 instructions per logit and pass)"}
+
+
 def c1_three_numbers(torch, L, W, dev, peak, use_graph=True):
     """Config 1 is smaller than a launch: (i) latency of a single eager verify call on an idle
     stream, (ii) 256 decode steps over 256 distinct input sets replayed back to back in one CUDA
@@ -766,6 +815,7 @@ def main():
                 torch, L, W, c3, dev, peak, allowed=(c3.code_offset, c3.code_offset + c3.codebook_size), use_graph=use_graph,
                 ring=16, note="tokens restricted to the 8192 image codes; bytes counted for that slice of every row")
             cfgs["c1_tiny"]["three_numbers"] = c1_three_numbers(torch, L, W, dev, peak, use_graph)
+            cfgs["f3_dynamic_tree"] = dynamic_tree_entry(torch, L, dev, peak)
             rows, dup = table_sweep(False)
             cfgs["c5_table_sweep"] = {
                 "dup_frac": dup, "total_ms": round(sum(r["ms"] for r in rows), 2),

@@ -10,13 +10,9 @@
 // (log V descending, pool index ascending); a parent therefore always ranks before its children.
 #include <cmath>
 
-#include "common.cuh"
+#include "rowops.cuh"
 
 namespace lantern {
-
-template <typename T> __device__ __forceinline__ float dyn_widen(T x);
-template <> __device__ __forceinline__ float dyn_widen<float>(float x) { return x; }
-template <> __device__ __forceinline__ float dyn_widen<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
 
 constexpr int kDynThreads = 256;
 constexpr int kDynMaxPool = 2048;
@@ -50,11 +46,86 @@ __device__ __forceinline__ void block_best(float& z, int& j, float* sz, int* sj)
   __syncthreads();
 }
 
+constexpr int kDynList = 1024;          // tokens at or above the row's selection threshold
+
+// Visits every allowed token of a row once: 16-byte vector loads over the aligned middle (when the
+// row pointers allow it), scalar loads at the ragged ends.  fn(j, z) per token; fold() after every
+// vector and after every scalar token.
+template <typename T, typename F, typename G>
+__device__ __forceinline__ void for_each_z(const T* c, const T* u, float g, float inv_tau, int lo, int hi, F&& fn, G&& fold) {
+  constexpr int VN = Vec<T>::N;
+  auto z1 = [&](float cc, float uu) { return u ? combine<true>(cc, uu, g, inv_tau) : combine<false>(cc, 0.f, g, inv_tau); };
+  const bool aligned = (reinterpret_cast<uintptr_t>(c) % 16 == 0) && (!u || reinterpret_cast<uintptr_t>(u) % 16 == 0);
+  int v0 = lo, v1 = lo;                                 // vector part [v0, v1)
+  if (aligned) {
+    v0 = (lo + VN - 1) / VN * VN;
+    v1 = hi / VN * VN;
+    if (v1 < v0) v1 = v0;
+  }
+  const int tid = threadIdx.x;
+  for (int j = lo + tid; j < (aligned ? min(v0, hi) : hi); j += kDynThreads) {
+    fn(j, z1(Vec<T>::widen(c[j]), u ? Vec<T>::widen(u[j]) : 0.f));
+    fold();
+  }
+  if (!aligned) return;
+  constexpr int UV = 4;                                 // vectors a thread keeps in flight (more would only grow the code)
+  for (int j0 = v0 + tid * VN; j0 < v1; j0 += kDynThreads * VN * UV) {
+    uint4 rc[UV], ru[UV];
+#pragma unroll
+    for (int q = 0; q < UV; ++q) {
+      const int j = j0 + q * kDynThreads * VN;
+      if (j < v1) {
+        rc[q] = ldg_stream_u128(c + j);
+        if (u) ru[q] = ldg_stream_u128(u + j);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < UV; ++q) {
+      const int j = j0 + q * kDynThreads * VN;
+      if (j < v1) {
+        float cf[VN], uf[VN];
+        Vec<T>::unpack_raw(rc[q], cf);
+        if (u) Vec<T>::unpack_raw(ru[q], uf);
+#pragma unroll
+        for (int e = 0; e < VN; ++e) fn(j + e, z1(cf[e], u ? uf[e] : 0.f));
+        fold();
+      }
+    }
+  }
+  for (int j = max(v1, v0) + tid; j < hi; j += kDynThreads) {
+    fn(j, z1(Vec<T>::widen(c[j]), u ? Vec<T>::widen(u[j]) : 0.f));
+    fold();
+  }
+}
+
+// The round of the fallback path: best token after (pz, pj) over the whole row, scalar loads.  Kept out
+// of line so that this rarely used scan does not grow the kernel's main loops.
+template <typename T>
+__device__ __noinline__ void scan_row_after(const T* c, const T* u, float g, float inv_tau, int lo, int hi, float pz, int pj,
+                                            float& bz, int& bj) {
+  for (int j = lo + threadIdx.x; j < hi; j += kDynThreads) {
+    const float z = u ? combine<true>(Vec<T>::widen(c[j]), Vec<T>::widen(u[j]), g, inv_tau)
+                      : combine<false>(Vec<T>::widen(c[j]), 0.f, g, inv_tau);
+    const bool after = z < pz || (z == pz && j > pj);
+    if (after && (z > bz || (z == bz && j < bj))) { bz = z; bj = j; }
+  }
+}
+
+// One frontier row.  Pass 1 (from HBM): every thread's maximum; the K-th largest of the 256 thread
+// maxima is a lower bound tau of the row's K-th largest value.  Pass 2 (the row is in L2 now): the
+// softmax denominator, and the tokens with z >= tau go to a short list in shared memory, from which
+// K rounds pick the children in the order (z descending, token ascending).  A list that overflows
+// (thousands of equal values) falls back to K rounds over the row.
 template <typename T>
 __global__ void __launch_bounds__(kDynThreads) expand_rows_kernel(const ExpandArgs a) {
   __shared__ float sz[kDynThreads / 32];
   __shared__ int sj[kDynThreads / 32];
   __shared__ double sd[kDynThreads / 32];
+  __shared__ float tmax[kDynThreads];
+  __shared__ float lz[kDynList];
+  __shared__ int lj[kDynList];
+  __shared__ int lcount;
+  __shared__ float tau_s;
   const int f = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   const int node = a.frontier[b * a.F + f];
   const long long pbase = static_cast<long long>(b) * a.P + a.pool_off + f * a.K;
@@ -69,22 +140,37 @@ __global__ void __launch_bounds__(kDynThreads) expand_rows_kernel(const ExpandAr
   }
   const T* c = static_cast<const T*>(a.dc) + b * a.seq_stride + f * a.row_stride;
   const T* u = a.du ? static_cast<const T*>(a.du) + b * a.seq_stride + f * a.row_stride : nullptr;
-  // the float32 pre-softmax value of a token: the row post-processing of every other entry point
-  auto zof = [&](int j) {
-    const float cc = dyn_widen<T>(c[j]);
-    if (u) { const float uu = dyn_widen<T>(u[j]); return __fmul_rn(__fmaf_rn(a.g, __fsub_rn(cc, uu), uu), a.inv_tau); }
-    return __fmul_rn(cc, a.inv_tau);
-  };
-  // maximum, then the softmax denominator (terms in float32, sum in double)
+  // pass 1 (from HBM): maxima only
   float m = -INFINITY;
-  int mj = 0x7fffffff;
-  for (int j = a.allow_lo + tid; j < a.allow_hi; j += kDynThreads) {
-    const float z = zof(j);
-    if (z > m) { m = z; mj = j; }
+  for_each_z<T>(c, u, a.g, a.inv_tau, a.allow_lo, a.allow_hi, [&](int, float z) { m = fmaxf(m, z); }, [] {});
+  tmax[tid] = m;
+  if (tid == 0) lcount = 0;
+  float bm = m;
+  int bj = tid;
+  block_best(bm, bj, sz, sj);                       // bm: the row's maximum (the barriers inside publish tmax too)
+  // tau = K-th largest thread maximum (rank by counting; K <= 8 <= 256 thread maxima)
+  {
+    int r = 0;
+    for (int t = 0; t < kDynThreads; ++t) r += (tmax[t] > m || (tmax[t] == m && t < tid)) ? 1 : 0;
+    if (r == min(a.K, kDynThreads) - 1) tau_s = m;
   }
-  block_best(m, mj, sz, sj);
+  __syncthreads();
+  const float tau = tau_s;
+  // pass 2 (the row is in L2 now): softmax denominator relative to the row maximum, terms in float32,
+  // a vector's terms summed in float32 and folded into a double (double-precision work is slow on this
+  // part, so it stays at one addition per vector); tokens at or above tau go to the list
   double s = 0.0;
-  for (int j = a.allow_lo + tid; j < a.allow_hi; j += kDynThreads) s += static_cast<double>(expf(zof(j) - m));
+  float part = 0.f;
+  for_each_z<T>(c, u, a.g, a.inv_tau, a.allow_lo, a.allow_hi,
+                [&](int j, float z) {
+                  part += ex2_approx(__fmul_rn(__fsub_rn(z, bm), kLog2e));   // exp(z - max): the argument's rounding costs
+                                                                             // |z - max| 2^-24 relative on a term of weight exp(z - max)
+                  if (z >= tau) {
+                    const int pos = atomicAdd(&lcount, 1);
+                    if (pos < kDynList) { lz[pos] = z; lj[pos] = j; }
+                  }
+                },
+                [&] { s += static_cast<double>(part); part = 0.f; });
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
   if ((tid & 31) == 0) sd[tid >> 5] = s;
@@ -93,50 +179,63 @@ __global__ void __launch_bounds__(kDynThreads) expand_rows_kernel(const ExpandAr
   for (int w = 0; w < kDynThreads / 32; ++w) s += sd[w];
   const double ln_s = log(s);
   const double parent_logv = a.pool_logv[static_cast<long long>(b) * a.P + node];
-  // K rounds: the best token that comes after the last pick in the order (z descending, id ascending)
+  __syncthreads();
+  const int n = lcount;
+  const bool listed = n <= kDynList;
   float pz = INFINITY;
   int pj = -1;
   for (int r = 0; r < a.K; ++r) {
     float bz = -INFINITY;
-    int bj = 0x7fffffff;
-    for (int j = a.allow_lo + tid; j < a.allow_hi; j += kDynThreads) {
-      const float z = zof(j);
-      const bool after = z < pz || (z == pz && j > pj);
-      if (after && (z > bz || (z == bz && j < bj))) { bz = z; bj = j; }
+    int bjj = 0x7fffffff;
+    if (listed) {
+      for (int i = tid; i < n; i += kDynThreads) {
+        const float z = lz[i];
+        const int j = lj[i];
+        const bool after = z < pz || (z == pz && j > pj);
+        if (after && (z > bz || (z == bz && j < bjj))) { bz = z; bjj = j; }
+      }
+    } else {
+      scan_row_after<T>(c, u, a.g, a.inv_tau, a.allow_lo, a.allow_hi, pz, pj, bz, bjj);
     }
-    block_best(bz, bj, sz, sj);
+    block_best(bz, bjj, sz, sj);
     if (tid == 0) {
-      const bool found = bj != 0x7fffffff;          // fewer than K allowed tokens: the rest can never be chosen
+      const bool found = bjj != 0x7fffffff;         // fewer than K allowed tokens: the rest can never be chosen
       a.pool_parent[pbase + r] = found ? node : -1;
-      a.pool_token[pbase + r] = found ? bj : -1;
+      a.pool_token[pbase + r] = found ? bjj : -1;
       a.pool_depth[pbase + r] = a.depth;
-      a.pool_logv[pbase + r] = found ? parent_logv + ((static_cast<double>(bz) - static_cast<double>(m)) - ln_s) : -INFINITY;
+      a.pool_logv[pbase + r] = found ? parent_logv + ((static_cast<double>(bz) - static_cast<double>(bm)) - ln_s) : -INFINITY;
     }
     pz = bz;
-    pj = bj;
+    pj = bjj;
   }
 }
 
-// rank of entry i among n entries by (value descending, index ascending); -inf entries rank last
-__device__ __forceinline__ int rank_desc(const double* v, int n, int i) {
-  const double vi = v[i];
+// order-preserving map of a double to an unsigned 64-bit integer (compares then run on the integer pipe)
+__device__ __forceinline__ unsigned long long mono64(double x) {
+  const unsigned long long b = static_cast<unsigned long long>(__double_as_longlong(x));
+  return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+}
+
+// rank of entry i among n entries by (value descending, index ascending); v holds mono64 keys
+__device__ __forceinline__ int rank_desc(const unsigned long long* v, int n, int i) {
+  const unsigned long long vi = v[i];
   int r = 0;
   for (int j = 0; j < n; ++j) {
-    const double vj = v[j];
+    const unsigned long long vj = v[j];
     r += (vj > vi || (vj == vi && j < i)) ? 1 : 0;
   }
   return r;
 }
 
 __global__ void __launch_bounds__(kDynThreads) select_frontier_kernel(const ExpandArgs a) {
-  extern __shared__ double dyn_lv[];
+  extern __shared__ unsigned long long dyn_lv[];
   const int b = blockIdx.x, tid = threadIdx.x, T = a.F * a.K;
   const double* lv = a.pool_logv + static_cast<long long>(b) * a.P + a.pool_off;
-  for (int i = tid; i < T; i += kDynThreads) dyn_lv[i] = lv[i];
+  for (int i = tid; i < T; i += kDynThreads) dyn_lv[i] = mono64(lv[i]);
   for (int e = tid; e < a.E; e += kDynThreads) a.next_frontier[b * a.E + e] = -1;
   __syncthreads();
   for (int i = tid; i < T; i += kDynThreads) {
-    if (dyn_lv[i] == -INFINITY) continue;
+    if (dyn_lv[i] == mono64(-INFINITY)) continue;
     const int r = rank_desc(dyn_lv, T, i);
     if (r < a.E) a.next_frontier[b * a.E + r] = a.pool_off + i;
   }
@@ -151,33 +250,48 @@ struct TrimArgs {
 };
 
 __global__ void __launch_bounds__(kDynThreads) trim_tree_kernel(const TrimArgs a) {
-  extern __shared__ double dyn_lv[];                 // [used] log V | new id [used] | selected [used]
+  extern __shared__ unsigned long long dyn_lv[];     // [used] keys of log V | new id | selected | depth | parent, [used] each
   int* newid = reinterpret_cast<int*>(dyn_lv + a.used);
   int* sel = newid + a.used;
+  int* dep_s = sel + a.used;
+  int* par_s = dep_s + a.used;
   __shared__ int count, level_n;
   const int b = blockIdx.x, tid = threadIdx.x, n = a.used;
   const long long base = static_cast<long long>(b) * a.P;
   for (int i = tid; i < n; i += kDynThreads) {
-    dyn_lv[i] = i == 0 ? INFINITY : a.pool_logv[base + i];      // the root ranks first
+    dyn_lv[i] = mono64(i == 0 ? INFINITY : a.pool_logv[base + i]);      // the root ranks first
     newid[i] = -1;
+    dep_s[i] = a.pool_depth[base + i];
+    par_s[i] = a.pool_parent[base + i];
   }
   __syncthreads();
   for (int i = tid; i < n; i += kDynThreads)
-    sel[i] = (i == 0 || (dyn_lv[i] != -INFINITY && rank_desc(dyn_lv, n, i) < a.m)) ? 1 : 0;
+    sel[i] = (i == 0 || (dyn_lv[i] != mono64(-INFINITY) && rank_desc(dyn_lv, n, i) < a.m)) ? 1 : 0;
   if (tid == 0) { count = 1; newid[0] = 0; }
   __syncthreads();
+  // the selected entries, compacted (order irrelevant); at most m of them
+  int* lst = reinterpret_cast<int*>(dyn_lv);        // the keys are no longer needed
+  __shared__ int nsel;
+  if (tid == 0) nsel = 0;
+  __syncthreads();
+  for (int i = 1 + tid; i < n; i += kDynThreads)
+    if (sel[i]) lst[atomicAdd(&nsel, 1)] = i;
+  __syncthreads();
+  const int ns = nsel;
   // breadth-first numbering: a level is ordered by (new id of the parent, pool index)
   for (int dep = 1; dep <= a.max_depth; ++dep) {
     if (tid == 0) level_n = 0;
     __syncthreads();
     const int start = count;
-    for (int i = tid; i < n; i += kDynThreads) {
-      if (!sel[i] || a.pool_depth[base + i] != dep) continue;
-      const int pi = newid[a.pool_parent[base + i]];
+    for (int t = tid; t < ns; t += kDynThreads) {
+      const int i = lst[t];
+      if (dep_s[i] != dep) continue;
+      const int pi = newid[par_s[i]];
       int pos = 0;
-      for (int j = 1; j < n; ++j) {
-        if (!sel[j] || j == i || a.pool_depth[base + j] != dep) continue;
-        const int pj = newid[a.pool_parent[base + j]];
+      for (int t2 = 0; t2 < ns; ++t2) {
+        const int j = lst[t2];
+        if (j == i || dep_s[j] != dep) continue;
+        const int pj = newid[par_s[j]];
         pos += (pj < pi || (pj == pi && j < i)) ? 1 : 0;
       }
       const int id = start + pos;
@@ -187,12 +301,13 @@ __global__ void __launch_bounds__(kDynThreads) trim_tree_kernel(const TrimArgs a
       a.pool_index[o] = i;
       a.logv[o] = a.pool_logv[base + i];
       atomicAdd(&level_n, 1);
-      // the id is published after the level is complete (below), so this level's reads see parents only
-      sel[i] = 2 + id;
+      sel[i] = 2 + id;                               // the id is published once the level is complete (below)
     }
     __syncthreads();
-    for (int i = tid; i < n; i += kDynThreads)
+    for (int t = tid; t < ns; t += kDynThreads) {
+      const int i = lst[t];
       if (sel[i] >= 2) { newid[i] = sel[i] - 2; sel[i] = 1; }
+    }
     if (tid == 0) count = start + level_n;
     __syncthreads();
   }
@@ -258,6 +373,6 @@ extern "C" lantern_status lantern_trim_tree(int32_t batch, int32_t pool_size, in
   a.B = batch; a.P = pool_size; a.used = pool_used; a.m = max_nodes; a.max_depth = max_depth;
   a.pool_parent = pool_parent; a.pool_token = pool_token; a.pool_depth = pool_depth; a.pool_logv = pool_logv;
   a.n_nodes = n_nodes; a.parent = parent; a.token = token; a.pool_index = pool_index; a.logv = logv;
-  trim_tree_kernel<<<batch, kDynThreads, static_cast<size_t>(pool_used) * 16, static_cast<cudaStream_t>(stream)>>>(a);
+  trim_tree_kernel<<<batch, kDynThreads, static_cast<size_t>(pool_used) * 24, static_cast<cudaStream_t>(stream)>>>(a);
   return cudaGetLastError() == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
 }
