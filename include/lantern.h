@@ -69,6 +69,17 @@ lantern_status lantern_tree_create(const int32_t* parent /* host [n_nodes] */, i
                                    lantern_tree** out);
 lantern_status lantern_tree_destroy(lantern_tree* tree);
 int32_t lantern_tree_max_depth(const lantern_tree* tree);  /* depth of the deepest node */
+/* A forest: one tree per sequence (Sec. 2.1, dynamic tree drafting: the shape of the draft tree
+ * depends on the sequence), each numbered as above and padded to max_nodes.  parent is a HOST
+ * array [batch][max_nodes] of which row b uses its first n_nodes[b] entries (host [batch]).  The
+ * handle is used like a tree with max_nodes nodes by lantern_verify_tree (and _static) for exactly
+ * `batch` sequences: per-node arrays are [batch][max_nodes], entries of padding nodes are ignored
+ * on input and -1 on output.  Served by the streaming kernels' eager launch only: rows that a
+ * top-k truncates, lazy_walk = 1 and kernels = 2 return LANTERN_ERR_UNSUPPORTED, and so does
+ * lantern_sample_draft_tree (such trees are drafted deterministically; verify them with
+ * draft_deterministic = 1).  Destroyed with lantern_tree_destroy.                               */
+lantern_status lantern_forest_create(const int32_t* parent /* host */, const int32_t* n_nodes /* host */,
+                                     int32_t batch, int32_t max_nodes, lantern_tree** out);
 
 /* ---- parameters (App. B "Models": guidance, temperature, top-k; Sec. 4: k, lambda) ---------
  * Row post-processing, identical for target rows (-> q) and drafter rows (-> p):

@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     LanternError,
     Params,
     Tree,
+    Forest,
     build_neighbors,
     sample_draft_tree,
     verify_tree,

@@ -75,6 +75,8 @@ def _load():
     L.lantern_status_string.argtypes = [ctypes.c_int]
     L.lantern_tree_create.restype = ctypes.c_int
     L.lantern_tree_create.argtypes = [vp, i32, ctypes.POINTER(vp)]
+    L.lantern_forest_create.restype = ctypes.c_int
+    L.lantern_forest_create.argtypes = [vp, vp, i32, i32, ctypes.POINTER(vp)]
     L.lantern_tree_destroy.restype = ctypes.c_int
     L.lantern_tree_destroy.argtypes = [vp]
     L.lantern_tree_max_depth.restype = i32
@@ -156,6 +158,25 @@ class Tree:
         if h is not None and lib is not None:
             lib.lantern_tree_destroy(h)
             self.handle = None
+
+
+class Forest(Tree):
+    """One tree per sequence, padded to max_nodes (lantern_forest_create); used like a Tree."""
+
+    def __init__(self, parents, n_nodes, max_nodes=None):
+        B = len(n_nodes)
+        self.n_nodes = int(max_nodes if max_nodes is not None else max(int(n) for n in n_nodes))
+        flat = []
+        for b in range(B):
+            row = [int(x) for x in parents[b][:int(n_nodes[b])]]
+            flat += row + [-1] * (self.n_nodes - len(row))
+        self.parent = flat
+        arr = (ctypes.c_int32 * len(flat))(*flat)
+        cnt = (ctypes.c_int32 * B)(*[int(n) for n in n_nodes])
+        h = ctypes.c_void_p()
+        _check(lib.lantern_forest_create(arr, cnt, B, self.n_nodes, ctypes.byref(h)), "lantern_forest_create")
+        self.handle = h
+        self.max_depth = lib.lantern_tree_max_depth(h)
 
 
 def _rows(t: torch.Tensor, B, N, V):

@@ -19,6 +19,7 @@ struct TreeDev {
   int32_t max_depth;
   int32_t max_children;
   int32_t n_internal;
+  int32_t per_seq;          // 0: one tree for every sequence.  B > 0: a forest of B trees padded to n_nodes, arrays [B][N]
   int32_t* d_first_child;   // [N] first child id, or -1
   int32_t* d_n_child;       // [N]
   int32_t* d_order;         // [N] node ids, internal nodes first (launch order)
@@ -195,6 +196,7 @@ struct VerifyArgs {
   int32_t* done;           // one counter, zero before the launch and again after it
   int32_t *accept_len, *out_tokens, *out_nodes;
   int D1;
+  int tree_stride;         // 0: the tree arrays are shared by all sequences; N: sequence b's arrays start at b * N (a forest)
 };
 
 // ---- walk (Sec. 2.1): follow accepted children from the root of one sequence.  nx / nt are the

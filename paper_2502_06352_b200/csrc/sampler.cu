@@ -457,6 +457,7 @@ extern "C" lantern_status lantern_sample_draft_tree(
   if (batch <= 0 || p->vocab <= 0 || !(p->temperature > 0.f) || p->top_k_draft < 0) return LANTERN_ERR_INVALID_ARG;
   if (dt != LANTERN_F32 && dt != LANTERN_BF16) return LANTERN_ERR_INVALID_ARG;
   if (parent_begin < 0 || parent_end > t->n_nodes || parent_begin > parent_end) return LANTERN_ERR_INVALID_ARG;
+  if (t->per_seq) return LANTERN_ERR_UNSUPPORTED;      // a forest holds deterministically drafted trees: nothing to sample
   const int V = p->vocab;
   const int allow_lo = p->allowed_begin, allow_hi = p->allowed_end == 0 ? V : p->allowed_end;
   if (allow_lo < 0 || allow_hi > V || allow_lo >= allow_hi) return LANTERN_ERR_INVALID_ARG;

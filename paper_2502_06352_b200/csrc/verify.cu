@@ -76,7 +76,7 @@ static cudaError_t launch_stream_k(const VerifyArgs& a, int cs, size_t smem, cud
 }
 template <typename T, bool CFG, bool TAU1>
 static cudaError_t launch_stream_t(const VerifyArgs& a, int cs, size_t smem, cudaStream_t st) {
-  return (a.lazy || a.skip || a.det) ? launch_stream_k<T, CFG, TAU1, true>(a, cs, smem, st)
+  return (a.lazy || a.skip || a.det || a.tree_stride) ? launch_stream_k<T, CFG, TAU1, true>(a, cs, smem, st)
                                      : launch_stream_k<T, CFG, TAU1, false>(a, cs, smem, st);
 }
 static cudaError_t launch_stream_any(const VerifyArgs& a, int cs, size_t smem, bool f32, bool cfg, cudaStream_t st) {
@@ -185,7 +185,7 @@ bool verify_uses_stream(const lantern_params* p, const TreeDev* t, int batch, bo
 extern "C" int32_t lantern_verify_tree_path(const lantern_params* p, const lantern_tree* tree, int32_t batch) {
   if (!p || !tree || batch <= 0) return -1;
   const TreeDev* t = reinterpret_cast<const TreeDev*>(tree);
-  if (verify_uses_stream(p, t, batch, true)) return LANTERN_PATH_STREAM;
+  if (t->per_seq || verify_uses_stream(p, t, batch, true)) return LANTERN_PATH_STREAM;
   return verify_uses_lists(p, t) ? LANTERN_PATH_LISTS : LANTERN_PATH_DENSE;
 }
 
@@ -213,6 +213,9 @@ extern "C" lantern_status lantern_verify_tree(
   if (t->n_internal > 0 && !draft_cond && !det) return LANTERN_ERR_INVALID_ARG;
   if ((target_uncond != nullptr) != (draft_uncond != nullptr) && t->n_internal > 0 && !det) return LANTERN_ERR_INVALID_ARG;
   if ((det || p->subset_rule) && !stream_applies(p, t)) return LANTERN_ERR_UNSUPPORTED;
+  // a forest (one tree per sequence) is served by the streaming kernel's eager launch only
+  if (t->per_seq && (batch != t->per_seq || p->lazy_walk || p->kernels == 2 || !stream_applies(p, t)))
+    return batch != t->per_seq ? LANTERN_ERR_INVALID_ARG : LANTERN_ERR_UNSUPPORTED;
   if (p->kernels < 0 || p->kernels > 2) return LANTERN_ERR_INVALID_ARG;
   if (p->k < 0 || p->top_k_target < 0 || p->top_k_draft < 0) return LANTERN_ERR_INVALID_ARG;
   if (!(p->delta >= 0.f) || p->delta > 4.f) return LANTERN_ERR_INVALID_ARG;      // also rejects NaN
@@ -261,6 +264,7 @@ extern "C" lantern_status lantern_verify_tree(
   a.only = nullptr;
   a.done = nullptr;
   a.lazy = p->lazy_walk ? 1 : 0;
+  a.tree_stride = t->per_seq ? t->n_nodes : 0;
   const int D1 = t->max_depth + 1;
   a.accept_len = accept_len; a.out_tokens = out_tokens; a.out_nodes = out_nodes; a.D1 = D1;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -272,7 +276,7 @@ extern "C" lantern_status lantern_verify_tree(
   cudaError_t e;
   // Rows truncated to a moderate top-k on every side that is read take the sparse kernel; the
   // dense kernel then repairs the nodes it could not hold (a.only) and usually finds none.
-  const bool use_sparse = redo && !a.lazy && verify_uses_lists(p, t);
+  const bool use_sparse = redo && !a.lazy && !t->per_seq && verify_uses_lists(p, t);
   if (use_sparse) {
     const int se = V <= sparse::ST * 8 ? 8 : (V <= sparse::ST * 16 ? 16 : 32);
     a.done = redo + static_cast<size_t>(batch) * t->n_nodes;       // the sparse kernel clears it
@@ -280,7 +284,7 @@ extern "C" lantern_status lantern_verify_tree(
     if (e != cudaSuccess) return LANTERN_ERR_CUDA;
     a.only = redo;
   }
-  if (!use_sparse && verify_uses_stream(p, t, batch, dense_fits(p, t, f32, cfg))) {
+  if (!use_sparse && (t->per_seq || verify_uses_stream(p, t, batch, dense_fits(p, t, f32, cfg)))) {
     const int cs = stream_cluster_size(a.lazy ? batch : batch * t->n_nodes, allow_hi - allow_lo, f32);
     e = launch_stream_any(a, cs, stream::smem_bytes(V, t->max_children, p->k + 1, cfg), f32, cfg, st);
     if (e != cudaSuccess) return LANTERN_ERR_CUDA;

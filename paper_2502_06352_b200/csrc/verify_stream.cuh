@@ -336,7 +336,8 @@ __device__ __forceinline__ int stream_node(const VerifyArgs& a, const int b, con
   constexpr int U1 = CFG ? 2 : 4;       // vectors in flight per thread and operand, single row
   constexpr int U2 = CFG ? 1 : 2;       // ... when two rows are read together
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int fc = a.first_child[n], nc = a.n_child[n];
+  const int toff = VAR ? b * a.tree_stride : 0;            // a forest keeps one set of tree arrays per sequence
+  const int fc = a.first_child[toff + n], nc = a.n_child[toff + n];
   const long long row_off = static_cast<long long>(b) * a.seq_stride + static_cast<long long>(n) * a.row_stride;
   const int32_t* tok_b = a.tokens + static_cast<long long>(b) * a.N;
   const long long out_b = static_cast<long long>(b) * a.N;
@@ -886,7 +887,17 @@ __global__ void __launch_bounds__(ST, LANTERN_STREAM_MINB) verify_stream_kernel(
   // nodes are not written.
   const bool lazy = GENERAL && a.lazy != 0;
   const int b = lazy ? idx : idx % a.B;
-  int cur = lazy ? 0 : a.order[idx / a.B];
+  int cur = lazy ? 0 : a.order[(GENERAL ? b * a.tree_stride : 0) + idx / a.B];
+  if (GENERAL && cur < 0) {            // padding of a forest's shorter tree: nothing to verify (the whole cluster leaves)
+    if (c.rank == 0 && threadIdx.x == 0) {
+      const long long o = static_cast<long long>(b) * a.N + idx / a.B;       // padding sits at the end of the order
+      a.node_next[o] = -1;
+      a.node_token[o] = -1;
+      if (a.node_mass) a.node_mass[o] = -1.f;
+      if (a.node_thresh) a.node_thresh[o] = -1.f;
+    }
+    return;
+  }
   int len = 0;
   for (;;) {
     const int acc = stream_node<T, CFG, TAU1, GENERAL>(a, b, cur, c, sm);

@@ -6,7 +6,7 @@ import torch
 
 import oracle
 from oracle import dynamic_tree as DT
-from gpu_cases import Case, small_config
+from gpu_cases import Case, small_config, f64
 from parity_util import compare_verify, check_walk
 
 pytestmark = pytest.mark.gpu
@@ -145,3 +145,47 @@ def test_drafted_trees_are_verified_with_deterministic_drafts(L):
         stats = compare_verify(res, o, case.parent, case.u_accept.numpy(), case.seqs, rerun=case.oracle_node)
         check_walk(res, case.tokens, tree.max_depth, o, stats["dirty_sequences"], case.seqs, stats["patched"])
     assert len(shapes) > 1            # the trees really differ from sequence to sequence
+
+
+@pytest.mark.parametrize("dtype,guided", [("f32", False), ("bf16", True)])
+def test_a_forest_of_drafted_trees_is_verified_in_one_call(L, dtype, guided):
+    """lantern_forest_create: every sequence keeps its own tree (padded to the largest); one verify call
+    covers the batch; each sequence is compared with the oracle run on its own tree."""
+    g = torch.Generator().manual_seed(33)
+    D, B, E, V, K, m = 5, 4, 6, 1200, 4, 30
+    data = torch.randn((D, B, E, V), generator=g) * torch.tensor([0.5, 1.5, 3.0, 6.0]).view(1, B, 1, 1)
+    gpu, orc = _draft(L, data, None, K, E, m, torch.float32)
+    assert _compare(gpu, orc, m) == 0
+    n_nodes = [int(x) for x in gpu["n"]]
+    parents = [[int(x) for x in gpu["parent"][b][:n_nodes[b]]] for b in range(B)]
+    assert len({tuple(p) for p in parents}) > 1
+    Nmax = max(n_nodes)
+    cfg = small_config(batch=B, n_nodes=Nmax, vocab=V, codebook_size=V, k=8, lam=3.0, dtype=dtype,
+                       cfg_scale=3.0 if guided else None)
+    # the inputs of one [B][Nmax] call; a dummy chain tree only sizes the generators
+    base = Case(cfg, parent=[-1] + list(range(Nmax - 1)), seed=70, det_draft=True, tokens="random")
+    for b in range(B):
+        base.tokens[b, 1:n_nodes[b]] = gpu["token"][b][1:n_nodes[b]]
+    gi, par, nbr, tok = base.gpu_inputs(L)
+    forest = L.Forest(parents, n_nodes, Nmax)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = L.verify_tree(par, forest, nbr, gi["target_cond"], gi["target_uncond"], None, None, tok,
+                        base.u_accept.cuda(), base.u_resample.cuda(), debug=True, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    res = {k: v.cpu().numpy() for k, v in out.items()}
+    lg = base.logits
+    for b in range(B):
+        n = n_nodes[b]
+        o = oracle.verify_sequence(
+            parents[b], f64(lg["target_cond"][b][:n]), None if lg["target_uncond"] is None else f64(lg["target_uncond"][b][:n]),
+            None, None, base.tokens[b][:n], base.u_accept[b].numpy()[:n], base.u_resample[b].numpy()[:n], base.nbr,
+            **base.params)
+        stats = compare_verify(res, [o], parents[b], base.u_accept.numpy(), [b])
+        assert stats["tie_accept"] + stats["tie_cut"] + stats["tie_resample"] == 0
+        # the walk: accepted path and its length as the oracle walks them
+        assert int(res["accept_len"][b]) == o["accept_len"]
+        L1 = o["accept_len"] + 1
+        assert list(res["out_tokens"][b][:L1]) == list(o["out_tokens"][:L1])
+        # padding nodes: -1 on output
+        assert np.all(res["node_next"][b][n:] == -1) and np.all(res["node_token"][b][n:] == -1)
