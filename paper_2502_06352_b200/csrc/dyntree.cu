@@ -51,11 +51,11 @@ constexpr int kDynList = 1024;          // tokens at or above the row's selectio
 // Visits every allowed token of a row once: 16-byte vector loads over the aligned middle (when the
 // row pointers allow it), scalar loads at the ragged ends.  fn(j, z) per token; fold() after every
 // vector and after every scalar token.
-template <typename T, typename F, typename G>
+template <typename T, bool CFG, typename F, typename G>
 __device__ __forceinline__ void for_each_z(const T* c, const T* u, float g, float inv_tau, int lo, int hi, F&& fn, G&& fold) {
   constexpr int VN = Vec<T>::N;
-  auto z1 = [&](float cc, float uu) { return u ? combine<true>(cc, uu, g, inv_tau) : combine<false>(cc, 0.f, g, inv_tau); };
-  const bool aligned = (reinterpret_cast<uintptr_t>(c) % 16 == 0) && (!u || reinterpret_cast<uintptr_t>(u) % 16 == 0);
+  auto z1 = [&](float cc, float uu) { return combine<CFG>(cc, uu, g, inv_tau); };
+  const bool aligned = (reinterpret_cast<uintptr_t>(c) % 16 == 0) && (!CFG || reinterpret_cast<uintptr_t>(u) % 16 == 0);
   int v0 = lo, v1 = lo;                                 // vector part [v0, v1)
   if (aligned) {
     v0 = (lo + VN - 1) / VN * VN;
@@ -64,7 +64,7 @@ __device__ __forceinline__ void for_each_z(const T* c, const T* u, float g, floa
   }
   const int tid = threadIdx.x;
   for (int j = lo + tid; j < (aligned ? min(v0, hi) : hi); j += kDynThreads) {
-    fn(j, z1(Vec<T>::widen(c[j]), u ? Vec<T>::widen(u[j]) : 0.f));
+    fn(j, z1(Vec<T>::widen(c[j]), CFG ? Vec<T>::widen(u[j]) : 0.f));
     fold();
   }
   if (!aligned) return;
@@ -76,7 +76,7 @@ __device__ __forceinline__ void for_each_z(const T* c, const T* u, float g, floa
       const int j = j0 + q * kDynThreads * VN;
       if (j < v1) {
         rc[q] = ldg_stream_u128(c + j);
-        if (u) ru[q] = ldg_stream_u128(u + j);
+        if (CFG) ru[q] = ldg_stream_u128(u + j);
       }
     }
 #pragma unroll
@@ -85,15 +85,15 @@ __device__ __forceinline__ void for_each_z(const T* c, const T* u, float g, floa
       if (j < v1) {
         float cf[VN], uf[VN];
         Vec<T>::unpack_raw(rc[q], cf);
-        if (u) Vec<T>::unpack_raw(ru[q], uf);
+        if (CFG) Vec<T>::unpack_raw(ru[q], uf);
 #pragma unroll
-        for (int e = 0; e < VN; ++e) fn(j + e, z1(cf[e], u ? uf[e] : 0.f));
+        for (int e = 0; e < VN; ++e) fn(j + e, z1(cf[e], CFG ? uf[e] : 0.f));
         fold();
       }
     }
   }
   for (int j = max(v1, v0) + tid; j < hi; j += kDynThreads) {
-    fn(j, z1(Vec<T>::widen(c[j]), u ? Vec<T>::widen(u[j]) : 0.f));
+    fn(j, z1(Vec<T>::widen(c[j]), CFG ? Vec<T>::widen(u[j]) : 0.f));
     fold();
   }
 }
@@ -116,7 +116,7 @@ __device__ __noinline__ void scan_row_after(const T* c, const T* u, float g, flo
 // softmax denominator, and the tokens with z >= tau go to a short list in shared memory, from which
 // K rounds pick the children in the order (z descending, token ascending).  A list that overflows
 // (thousands of equal values) falls back to K rounds over the row.
-template <typename T>
+template <typename T, bool CFG>
 __global__ void __launch_bounds__(kDynThreads) expand_rows_kernel(const ExpandArgs a) {
   __shared__ float sz[kDynThreads / 32];
   __shared__ int sj[kDynThreads / 32];
@@ -139,10 +139,10 @@ __global__ void __launch_bounds__(kDynThreads) expand_rows_kernel(const ExpandAr
     return;
   }
   const T* c = static_cast<const T*>(a.dc) + b * a.seq_stride + f * a.row_stride;
-  const T* u = a.du ? static_cast<const T*>(a.du) + b * a.seq_stride + f * a.row_stride : nullptr;
+  const T* u = CFG ? static_cast<const T*>(a.du) + b * a.seq_stride + f * a.row_stride : nullptr;
   // pass 1 (from HBM): maxima only
   float m = -INFINITY;
-  for_each_z<T>(c, u, a.g, a.inv_tau, a.allow_lo, a.allow_hi, [&](int, float z) { m = fmaxf(m, z); }, [] {});
+  for_each_z<T, CFG>(c, u, a.g, a.inv_tau, a.allow_lo, a.allow_hi, [&](int, float z) { m = fmaxf(m, z); }, [] {});
   tmax[tid] = m;
   if (tid == 0) lcount = 0;
   float bm = m;
@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(kDynThreads) expand_rows_kernel(const ExpandAr
   // part, so it stays at one addition per vector); tokens at or above tau go to the list
   double s = 0.0;
   float part = 0.f;
-  for_each_z<T>(c, u, a.g, a.inv_tau, a.allow_lo, a.allow_hi,
+  for_each_z<T, CFG>(c, u, a.g, a.inv_tau, a.allow_lo, a.allow_hi,
                 [&](int j, float z) {
                   part += ex2_approx(__fmul_rn(__fsub_rn(z, bm), kLog2e));   // exp(z - max): the argument's rounding costs
                                                                              // |z - max| 2^-24 relative on a term of weight exp(z - max)
@@ -354,8 +354,14 @@ extern "C" lantern_status lantern_expand_frontier(const lantern_params* p, const
   a.next_frontier = next_frontier;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid(n_frontier, batch);
-  if (dt == LANTERN_F32) expand_rows_kernel<float><<<grid, kDynThreads, 0, st>>>(a);
-  else expand_rows_kernel<__nv_bfloat16><<<grid, kDynThreads, 0, st>>>(a);
+  const bool cfg = draft_uncond != nullptr;
+  if (dt == LANTERN_F32) {
+    if (cfg) expand_rows_kernel<float, true><<<grid, kDynThreads, 0, st>>>(a);
+    else expand_rows_kernel<float, false><<<grid, kDynThreads, 0, st>>>(a);
+  } else {
+    if (cfg) expand_rows_kernel<__nv_bfloat16, true><<<grid, kDynThreads, 0, st>>>(a);
+    else expand_rows_kernel<__nv_bfloat16, false><<<grid, kDynThreads, 0, st>>>(a);
+  }
   if (cudaGetLastError() != cudaSuccess) return LANTERN_ERR_CUDA;
   select_frontier_kernel<<<batch, kDynThreads, static_cast<size_t>(T) * sizeof(double), st>>>(a);
   return cudaGetLastError() == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
