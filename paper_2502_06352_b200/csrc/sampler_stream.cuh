@@ -101,6 +101,43 @@ __device__ __forceinline__ float cut_list(const SampSmem& s, int R, float T) {
   return got == R ? pk : T;
 }
 
+// The same cut for a short list, by warp 0 alone (no barriers inside the rounds); every thread
+// calls it between two barriers' worth of quiet: nobody appends while it runs.  R <= 15.
+__device__ __forceinline__ float cut_small(const SampSmem& s, int R, float T) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int n = min(*s.cnt, kListCap);
+  __syncthreads();                               // every thread has read the count
+  if (tid < 32) {
+    float pk = INFINITY;
+    int pt = -1;
+    int got = 0;
+    for (int round = 0; round < R; ++round) {
+      float bk = -INFINITY;
+      int bt = 0x7fffffff;
+      for (int i = lane; i < n; i += 32) {
+        const uint2 en = s.list[i];
+        const float k = __uint_as_float(en.x);
+        const int t = static_cast<int>(en.y);
+        if (key_before(pk, pt, k, t) && key_before(k, t, bk, bt)) { bk = k; bt = t; }
+      }
+      warp_key_first(bk, bt);
+      if (bt == 0x7fffffff) break;               // fewer than R entries (the same in every lane)
+      if (lane == 0) s.top[round] = make_uint2(__float_as_uint(bk), static_cast<uint32_t>(bt));
+      pk = bk;
+      pt = bt;
+      ++got;
+    }
+    __syncwarp();
+    if (lane < got) s.list[lane] = s.top[lane];
+    if (lane == 0) {
+      *s.cnt = got;
+      s.top[15].x = __float_as_uint(got == R ? pk : T);
+    }
+  }
+  __syncthreads();
+  return __uint_as_float(s.top[15].x);
+}
+
 template <typename T, bool CFG, bool TAU1>
 __global__ void __launch_bounds__(ST, 4) sample_stream_kernel(const SampleArgs a) {
   grid_dependency_sync();
@@ -184,9 +221,18 @@ __global__ void __launch_bounds__(ST, 4) sample_stream_kernel(const SampleArgs a
     return near_one;
   };
 
-  // Optimistic pass: after the first cut the threshold is high and appends are rare, so the
-  // remaining chunks run without barriers or further cuts; if the list overflows all the same
-  // (keys that keep growing along the row), the row is redone with a check after every chunk.
+  // One entry for the list (appends are rare after the first cut: a shared-memory atomic each)
+  auto append = [&](float k, int tok) {
+    const int pos = atomicAdd(s.cnt, 1);
+    if (pos < kListCap) s.list[pos] = make_uint2(__float_as_uint(k), static_cast<uint32_t>(tok));
+  };
+  // Optimistic pass.  In the first chunk every thread enters only its best key: 256 entries from
+  // distinct tokens bound the R-th best key from below, a cut of that short list gives the first
+  // threshold, and the chunk's other keys above it (kept in registers meanwhile) follow.  Further
+  // cuts after chunks 1, 3 and 7 (each doubles the share of the row behind the threshold, so the
+  // chance that a vector holds a key above it halves each time); the chunks in between run without
+  // barriers.  If the list overflows all the same (keys that keep growing along the row), the
+  // row is redone with a check after every chunk.
   float Tk = -INFINITY;                               // every element left out has key <= Tk
   float mx = -INFINITY, sx = 0.f;
   const int iters = (ge.vw + 32 * UV - 1) / (32 * UV);
@@ -202,13 +248,17 @@ __global__ void __launch_bounds__(ST, 4) sample_stream_kernel(const SampleArgs a
         const int vv = base + 32 * u + lane;
         if (vv < vend && vv >= ge.vi0 && vv < ge.vi1) io.load(vv, rc[u], ru[u]);
       }
+      float first[UV][VN];                              // keys of the first chunk
+      float tbk = -INFINITY;                            // ... and the thread's best of them
+      int tbj = 0x7fffffff;
 #pragma unroll
       for (int u = 0; u < UV; ++u) {
         const int vv = base + 32 * u + lane;
         const bool active = vv < vend;
         const int j = ge.j0 + vv * VN;
         float z[VN], key[VN];
-        bool any = false;
+#pragma unroll
+        for (int e = 0; e < VN; ++e) key[e] = -INFINITY;
         if (active) {
           if (vv >= ge.vi0 && vv < ge.vi1) {
             io.z(rc[u], ru[u], z);
@@ -225,32 +275,43 @@ __global__ void __launch_bounds__(ST, 4) sample_stream_kernel(const SampleArgs a
             for (int e = 0; e < VN; ++e)
               if (U[e] > 0.999f) key[e] = careful_key(z[e], U[e]);
           }
+          if (want_prob) acc_exp<VN>(z, mx, sx);
+        }
+        if (it == 0) {
+#pragma unroll
+          for (int e = 0; e < VN; ++e) {
+            first[u][e] = key[e];
+            if (key_before(key[e], j + e, tbk, tbj)) { tbk = key[e]; tbj = j + e; }
+          }
+        } else {
           float best = key[0];
 #pragma unroll
           for (int e = 1; e < VN; ++e) best = fmaxf(best, key[e]);
-          any = best > Tk;
-          if (want_prob) acc_exp<VN>(z, mx, sx);
-        }
-        if (__any_sync(0xffffffffu, any)) {
+          if (best > Tk) {                              // rare, and rarer after every cut
 #pragma unroll
-          for (int e = 0; e < VN; ++e) {
-            const bool take = active && key[e] > Tk;
-            const uint32_t m = __ballot_sync(0xffffffffu, take);
-            if (m) {
-              int pos0 = 0;
-              if (lane == 0) pos0 = atomicAdd(s.cnt, __popc(m));
-              pos0 = __shfl_sync(0xffffffffu, pos0, 0);
-              const int pos = pos0 + __popc(m & ((1u << lane) - 1u));
-              if (take && pos < kListCap) s.list[pos] = make_uint2(__float_as_uint(key[e]), static_cast<uint32_t>(j + e));
-            }
+            for (int e = 0; e < VN; ++e)
+              if (key[e] > Tk) append(key[e], j + e);
           }
         }
       }
-      if (it == 0 || mode == 1) {
+      if (it == 0) {
+        if (tbk > -INFINITY) append(tbk, tbj);
         __syncthreads();
-        const bool full = *s.cnt > kListCap - kIterElems;
+        if (*s.cnt > R) Tk = cut_small(s, R, Tk);       // (the count is the same for every thread: nobody appends here)
+        else __syncthreads();
+#pragma unroll
+        for (int u = 0; u < UV; ++u) {
+          const int j = ge.j0 + (base + 32 * u + lane) * VN;
+#pragma unroll
+          for (int e = 0; e < VN; ++e)
+            if (first[u][e] > Tk && j + e != tbj) append(first[u][e], j + e);
+        }
+      } else if (it == 1 || it == 3 || it == 7 || mode == 1) {
+        __syncthreads();
+        const int cn = *s.cnt;
+        const bool do_cut = mode == 1 ? cn > kListCap - kIterElems : cn > R;
         __syncthreads();                                // everyone has read the count before it moves again
-        if (full) Tk = cut_list(s, R, Tk);
+        if (do_cut) Tk = cn <= 1024 ? cut_small(s, R, Tk) : cut_list(s, R, Tk);
       }
     }
     __syncthreads();
