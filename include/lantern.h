@@ -224,7 +224,8 @@ lantern_status lantern_verify_tree(const lantern_params* params, const lantern_t
  * the dense kernels that redoes the nodes whose rows did not fit the lists' fixed buffers (massive
  * ties; usually none).  All other calls (top-k on wide vocabularies, the path walk) run the dense
  * kernels alone (LANTERN_PATH_DENSE: rows held in shared memory).  So do small calls without top-k
- * (fewer than 128 tree nodes, or 256 expanded parents, in the whole batch) whose rows fit the dense
+ * (fewer than 128 tree nodes, or fewer than both 256 and 4 Mi / vocab expanded parents, in the whole
+ * batch) whose rows fit the dense
  * kernels: a handful of nodes is a chain of dependent steps, which shared-memory rows shorten.
  * params->kernels overrides the choice by size.  Results are the same either way; these queries
  * only tell which it will be for a batch of `batch` sequences (lantern_verify_tree additionally

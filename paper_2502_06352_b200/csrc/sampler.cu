@@ -430,14 +430,17 @@ bool sampler_uses_lists(const lantern_params* p) {
 }  // namespace
 
 // Rows that no top-k truncates can take the streaming kernel; it does when the call expands at
-// least kStreamMinParents parents (fewer are a chain of dependent steps that the dense kernel's
-// shared-memory row shortens), when the dense kernel cannot hold the row, or when asked to.
+// least kStreamMinParents parents or kStreamMinLogits / V of them (fewer fit the dense kernel's one
+// wave of CTAs, or of CTA clusters for wide rows, whose shared-memory row shortens the chain of
+// dependent steps: the measured cross-over lies between 2.6 M and 5.2 M parents x V for V = 16384
+// and 65536, whatever the allowed range), when the dense kernel cannot hold the row, or when asked to.
 constexpr int kStreamMinParents = 256;
+constexpr long long kStreamMinLogits = 4ll << 20;
 static bool sampler_uses_stream(const lantern_params* p, long long parents, bool fits_dense) {
   if ((p->top_k_draft > 0 && p->top_k_draft < p->vocab) || p->vocab > stream::kMaxV) return false;
   if (p->kernels == 2) return !fits_dense;
   if (p->kernels == 1) return true;
-  return parents >= kStreamMinParents || !fits_dense;
+  return parents >= kStreamMinParents || parents * p->vocab >= kStreamMinLogits || !fits_dense;
 }
 
 extern "C" int32_t lantern_sample_draft_tree_path(const lantern_params* p, const lantern_tree* tree, int32_t batch) {
