@@ -226,16 +226,16 @@ __global__ void __launch_bounds__(ST, 4) sample_stream_kernel(const SampleArgs a
     const int pos = atomicAdd(s.cnt, 1);
     if (pos < kListCap) s.list[pos] = make_uint2(__float_as_uint(k), static_cast<uint32_t>(tok));
   };
-  // Optimistic pass.  In the first chunk every thread enters only its best key: 256 entries from
-  // distinct tokens bound the R-th best key from below, a cut of that short list gives the first
-  // threshold, and the chunk's other keys above it (kept in registers meanwhile) follow.  Further
-  // cuts after chunks 1, 3 and 7 (each doubles the share of the row behind the threshold, so the
-  // chance that a vector holds a key above it halves each time); the chunks in between run without
-  // barriers.  If the list overflows all the same (keys that keep growing along the row), the
+  // Optimistic pass.  The first chunk's keys stay in registers until a first threshold is known: the
+  // R-th best of the warps' two best keys each (distinct tokens, so a lower bound of the row's R-th
+  // best key), found with one barrier; the chunk's keys above it then enter the list.  One cut of the
+  // (short) list after a third of the row tightens the threshold (more cuts cost more in barriers than
+  // they save in appends); the other chunks run without barriers.  If the list overflows all the same (keys that keep growing along the row), the
   // row is redone with a check after every chunk.
   float Tk = -INFINITY;                               // every element left out has key <= Tk
   float mx = -INFINITY, sx = 0.f;
   const int iters = (ge.vw + 32 * UV - 1) / (32 * UV);
+  const int cut_it = max(1, iters / 3);                // the one scheduled cut of the optimistic pass
   for (int mode = 0; mode < 2; ++mode) {
     Tk = -INFINITY;
     mx = -INFINITY;
@@ -295,18 +295,41 @@ __global__ void __launch_bounds__(ST, 4) sample_stream_kernel(const SampleArgs a
         }
       }
       if (it == 0) {
-        if (tbk > -INFINITY) append(tbk, tbj);
+        // the two best of every warp's thread-bests: 2 * SW keys of distinct tokens, whose R-th best is a
+        // lower bound of the row's R-th best key (R <= 12 <= 2 * SW); every warp ranks them for itself
+        float k1 = tbk, k2;
+        int j1 = tbj, j2;
+        warp_key_first(k1, j1);
+        k2 = (tbj == j1) ? -INFINITY : tbk;
+        j2 = (tbj == j1) ? 0x7fffffff : tbj;
+        warp_key_first(k2, j2);
+        if (lane == 0) {
+          s.pk[2 * warp] = make_uint2(__float_as_uint(k1), static_cast<uint32_t>(j1));
+          s.pk[2 * warp + 1] = make_uint2(__float_as_uint(k2), static_cast<uint32_t>(j2));
+        }
         __syncthreads();
-        if (*s.cnt > R) Tk = cut_small(s, R, Tk);       // (the count is the same for every thread: nobody appends here)
-        else __syncthreads();
+        {
+          const uint2 en = s.pk[lane & (2 * SW - 1)];
+          const float mk = __uint_as_float(en.x);
+          const int mt = static_cast<int>(en.y);
+          int rank = 0;
+#pragma unroll
+          for (int i = 0; i < 2 * SW; ++i) {
+            const float ok = __shfl_sync(0xffffffffu, mk, i);
+            const int ot = __shfl_sync(0xffffffffu, mt, i);
+            rank += key_before(ok, ot, mk, mt) ? 1 : 0;
+          }
+          const uint32_t hit = __ballot_sync(0xffffffffu, lane < 2 * SW && rank == R - 1 && mt != 0x7fffffff && mk > -INFINITY);
+          if (hit) Tk = __shfl_sync(0xffffffffu, mk, __ffs(hit) - 1);
+        }
 #pragma unroll
         for (int u = 0; u < UV; ++u) {
           const int j = ge.j0 + (base + 32 * u + lane) * VN;
 #pragma unroll
           for (int e = 0; e < VN; ++e)
-            if (first[u][e] > Tk && j + e != tbj) append(first[u][e], j + e);
+            if (first[u][e] > Tk) append(first[u][e], j + e);
         }
-      } else if (it == 1 || it == 3 || it == 7 || mode == 1) {
+      } else if (it == cut_it || mode == 1) {
         __syncthreads();
         const int cn = *s.cnt;
         const bool do_cut = mode == 1 ? cn > kListCap - kIterElems : cn > R;
