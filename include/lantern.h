@@ -15,7 +15,7 @@
  *    (a table index out of range, a copy that did not complete in time) are
  *    OR-ed into *device_status as LANTERN_DEV_* bits; the kernels never trap.
  *  - Same inputs and same uniforms / seed give the same bytes.
- *  - Only lantern_tree_create allocates (a few hundred bytes per tree).
+ *  - Only lantern_tree_create and lantern_forest_create allocate (a few hundred bytes per tree).
  *  - Entry points may be called from several host threads at once as long as the calls do not
  *    share output buffers or a workspace; lantern_set_cluster_size is the exception (see there).
  *  - The neighbour table must not list a token among its own neighbours and a row's entries

@@ -189,3 +189,32 @@ def test_a_forest_of_drafted_trees_is_verified_in_one_call(L, dtype, guided):
         assert list(res["out_tokens"][b][:L1]) == list(o["out_tokens"][:L1])
         # padding nodes: -1 on output
         assert np.all(res["node_next"][b][n:] == -1) and np.all(res["node_token"][b][n:] == -1)
+
+
+def test_argument_errors_are_reported_before_anything_runs(L):
+    """Error behaviour of the dynamic-tree entry points and of the forest handle (host-side checks)."""
+    V = 512
+    rows = torch.randn((1, 1, V)).cuda()
+    pool = L.DraftPool(1, 2, 4, 4)
+    with pytest.raises(L.LanternError):                       # truncated rows: confidences of a top-k row are not built
+        L.expand_frontier(L.Params(vocab=V, top_k_draft=10), pool, rows)
+    assert pool.used == 1 and pool.n_depths == 0              # nothing advanced
+    with pytest.raises(L.LanternError):                       # more children than a tree node may have
+        L.expand_frontier(L.Params(vocab=V), L.DraftPool(1, 2, 9, 4), rows)
+    with pytest.raises(L.LanternError):                       # parents must be numbered breadth first
+        L.Forest([[-1, 0, 0], [-1, 0, 1, 0]], [3, 4], 4)
+    forest = L.Forest([[-1, 0, 0], [-1, 0, 1, 1]], [3, 4], 4)
+    par = L.Params(vocab=V, k=0, draft_deterministic=1)
+    tc = torch.randn((2, 4, V)).cuda()
+    tok = torch.zeros((2, 4), dtype=torch.int32).cuda()
+    u = torch.rand((2, 4)).cuda()
+    with pytest.raises(L.LanternError):                       # a forest serves exactly its own number of sequences
+        L.verify_tree(par, forest, None, tc[:1], None, None, None, tok[:1], u[:1], u[:1])
+    with pytest.raises(L.LanternError):                       # ... on the streaming kernels only
+        L.verify_tree(L.Params(vocab=V, k=0, draft_deterministic=1, top_k_target=50), forest, None, tc, None, None, None,
+                      tok, u, u)
+    with pytest.raises(L.LanternError):                       # ... and is never sampled
+        L.sample_draft_tree(L.Params(vocab=V), forest, tc)
+    out = L.verify_tree(par, forest, None, tc, None, None, None, tok, u, u)
+    torch.cuda.synchronize()
+    assert out["accept_len"].shape == (2,)
