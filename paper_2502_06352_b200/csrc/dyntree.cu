@@ -111,8 +111,8 @@ __device__ __noinline__ void scan_row_after(const T* c, const T* u, float g, flo
   }
 }
 
-// One frontier row.  Pass 1 (from HBM): every thread's maximum; the K-th largest of the 256 thread
-// maxima is a lower bound tau of the row's K-th largest value.  Pass 2 (the row is in L2 now): the
+// One frontier row.  Pass 1 (from HBM): every thread's maximum; the K-th largest of the warps' two
+// largest thread maxima each is a lower bound tau of the row's K-th largest value.  Pass 2 (the row is in L2 now): the
 // softmax denominator, and the tokens with z >= tau go to a short list in shared memory, from which
 // K rounds pick the children in the order (z descending, token ascending).  A list that overflows
 // (thousands of equal values) falls back to K rounds over the row.
@@ -121,11 +121,10 @@ __global__ void __launch_bounds__(kDynThreads) expand_rows_kernel(const ExpandAr
   __shared__ float sz[kDynThreads / 32];
   __shared__ int sj[kDynThreads / 32];
   __shared__ double sd[kDynThreads / 32];
-  __shared__ float tmax[kDynThreads];
+  __shared__ float tmax[2 * (kDynThreads / 32)];
   __shared__ float lz[kDynList];
   __shared__ int lj[kDynList];
   __shared__ int lcount;
-  __shared__ float tau_s;
   const int f = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   const int node = a.frontier[b * a.F + f];
   const long long pbase = static_cast<long long>(b) * a.P + a.pool_off + f * a.K;
@@ -143,19 +142,33 @@ __global__ void __launch_bounds__(kDynThreads) expand_rows_kernel(const ExpandAr
   // pass 1 (from HBM): maxima only
   float m = -INFINITY;
   for_each_z<T, CFG>(c, u, a.g, a.inv_tau, a.allow_lo, a.allow_hi, [&](int, float z) { m = fmaxf(m, z); }, [] {});
-  tmax[tid] = m;
+  // the two largest thread maxima of every warp: 16 values of distinct tokens, whose K-th largest
+  // (K <= 8) is a lower bound tau of the row's K-th largest value; every warp ranks them for itself
+  {
+    const int lane = tid & 31, warp = tid >> 5;
+    const float w1 = warp_max(m);
+    const int wl = __ffs(__ballot_sync(0xffffffffu, m == w1)) - 1;
+    const float w2 = warp_max(lane == wl ? -INFINITY : m);
+    if (lane == 0) { tmax[2 * warp] = w1; tmax[2 * warp + 1] = w2; }
+  }
   if (tid == 0) lcount = 0;
   float bm = m;
   int bj = tid;
-  block_best(bm, bj, sz, sj);                       // bm: the row's maximum (the barriers inside publish tmax too)
-  // tau = K-th largest thread maximum (rank by counting; K <= 8 <= 256 thread maxima)
+  block_best(bm, bj, sz, sj);                       // bm: the row's maximum (the barriers inside publish tmax and lcount too)
+  float tau = -INFINITY;
   {
+    const int lane = tid & 31;
+    constexpr int NV = 2 * (kDynThreads / 32);
+    const float v = lane < NV ? tmax[lane] : -INFINITY;
     int r = 0;
-    for (int t = 0; t < kDynThreads; ++t) r += (tmax[t] > m || (tmax[t] == m && t < tid)) ? 1 : 0;
-    if (r == min(a.K, kDynThreads) - 1) tau_s = m;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const float o = __shfl_sync(0xffffffffu, v, i);
+      r += (o > v || (o == v && i < lane)) ? 1 : 0;
+    }
+    const uint32_t hit = __ballot_sync(0xffffffffu, lane < NV && r == min(a.K, NV) - 1);
+    tau = __shfl_sync(0xffffffffu, v, __ffs(hit) - 1);
   }
-  __syncthreads();
-  const float tau = tau_s;
   // pass 2 (the row is in L2 now): softmax denominator relative to the row maximum, terms in float32,
   // a vector's terms summed in float32 and folded into a double (double-precision work is slow on this
   // part, so it stays at one addition per vector); tokens at or above tau go to the list
