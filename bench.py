@@ -372,6 +372,23 @@ def run_table_sweep(args):
                       "gpu_launches": 4 * 2 * len(rows)}))
 
 
+def run_dynamic_tree(args):
+    """--workload f3_dynamic_tree: dynamic-tree drafting as the headline of its own JSON line."""
+    import torch
+    import paper_2502_06352_b200 as L
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    peak, peak_kind = peak_hbm()
+    ent = dynamic_tree_entry(torch, L, dev, peak)
+    rows = 64 * (1 + 5 * 8)
+    print(json.dumps({"metric": "drafter rows expanded/sec", "value": rows / (ent["us_median"] * 1e-6), "unit": "rows/s",
+                      "n_gpus": 1, "steps": 20, "warmup": 3, "ms_per_step": ent["us_median"] * 1e-3, "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "f32 (log V in f64)", "data": "synthetic",
+                      "config": {"workload": ent["workload"]}, "roofline": {"bound": "hbm", "achieved": ent["gbs"], "peak": peak,
+                      "unit": "GB/s", "frac": ent["frac_measured"], "peak_kind": peak_kind, "traffic": None,
+                      "kernel": ent["kernels"]}, "gpu_launches": ent["launches"] * 20, "detail": ent}))
+
+
 # ------------------------------------------------------------------------------------------------
 # one configuration on the device
 
@@ -567,7 +584,7 @@ def dynamic_tree_entry(torch, L, dev, peak):
             "us_median": round(1e3 * med, 1), "us_min": round(1e3 * times[0], 1), "algorithmic_bytes": alg,
             "gbs": round(alg / (med * 1e-3) / 1e9, 1), "frac_measured": round(alg / (med * 1e-3) / 1e9 / peak, 4),
             "mean_nodes": float(n.float().mean()), "mean_node_depth": round(depth_mean, 3),
-            "note": "two passes per row (HBM, then L2); instruction-bound (about 20 instructions per logit and pass)"}
+            "note": "two passes per row (HBM, then L2); about 10 instructions per logit and pass, latency-bound chain per row"}
 
 
 def c1_three_numbers(torch, L, W, dev, peak, use_graph=True):
@@ -609,6 +626,9 @@ def main():
     import workloads as W
     if args.workload == "c5_table_sweep":
         run_table_sweep(args)
+        return
+    if args.workload == "f3_dynamic_tree":
+        run_dynamic_tree(args)
         return
     cfg = W.CONFIGS[args.workload]
     if args.batch > 0:
