@@ -121,3 +121,16 @@ def test_tcgen05_kernel_overflowing_lists_take_the_exact_fallback(L):
     idx, dist = _check(L, cb, k, rows=[0, 999, 1000, 1001, 1500, 2199, 2200, n - 1])
     assert list(idx[1000]) == list(range(1001, 1021)) and list(idx[1500]) == list(range(1000, 1020))
     assert np.all(dist[1000:2200] == 0)
+
+
+@pytest.mark.parametrize("n,d,k", [(8192, 16, 50), (9000, 40, 200)])
+def test_tcgen05_and_brute_force_kernels_build_the_same_table(L, n, d, k):
+    """Every row, not a sample: the same codebook as bfloat16 (tcgen05 kernel) and widened to float32 (exact
+    brute-force kernel; the widening is exact) must give the same indices and the same distances, twice."""
+    cb = W.make_codebook(n, d, "bf16", seed=n + d, dup_frac=0.05).cuda()
+    i1, d1 = L.build_neighbors(cb, k, return_dist=True)
+    i2, d2 = L.build_neighbors(cb.to(torch.float32), k, return_dist=True)
+    i3, d3 = L.build_neighbors(cb, k, return_dist=True)
+    torch.cuda.synchronize()
+    assert torch.equal(i1, i3) and torch.equal(d1, d3)          # run to run
+    assert torch.equal(i1, i2) and torch.equal(d1, d2)          # kernel to kernel
