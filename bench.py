@@ -718,6 +718,11 @@ def main():
     clk = clocks.stop()
     verify_med_ms = tv[len(tv) // 2]
     accept_mean = float(w.out["accept_len"].float().mean().item())
+    # accepted path lengths of the last step: how many sequences accepted exactly d draft tokens, and the
+    # share of sequences that got past each depth (the per-depth accept rate of the walk, Sec. 2.1)
+    al = w.out["accept_len"].cpu().tolist()
+    hist = [al.count(d) for d in range(max(al) + 1)]
+    reach = [sum(1 for x in al if x >= d) / len(al) for d in range(1, max(al) + 1)]
     dev_status = int(w.status.item())
     total_nodes = world * B * N * K
     value = total_nodes / (elapsed_ms * 1e-3)
@@ -819,7 +824,8 @@ def main():
             "gpu_launches": launches_per_step * K,
             "clocks": clk,
             "table_build": table,
-            "stats": {"mean_accept_len": accept_mean, "tokens_per_step": accept_mean + 1.0, "device_status": dev_status},
+            "stats": {"mean_accept_len": accept_mean, "tokens_per_step": accept_mean + 1.0, "device_status": dev_status,
+                      "accept_len_hist": hist, "reached_depth_share": [round(x, 4) for x in reach]},
         }
         if world == 1 and args.configs == "all" and args.walk == "eager":
             cfgs = {}

@@ -11,6 +11,8 @@ from .binding import (  # noqa: F401
     Tree,
     Forest,
     build_neighbors,
+    save_neighbors,
+    load_neighbors,
     sample_draft_tree,
     verify_tree,
     verify_tree_static,

@@ -202,6 +202,35 @@ def build_neighbors(codebook: torch.Tensor, k: int, return_dist=False):
     return (idx, dist) if return_dist else idx
 
 
+def save_neighbors(path: str, nbr_idx: torch.Tensor, codebook: torch.Tensor = None):
+    """Writes a neighbour table ([L][k] int32) to `path` (numpy .npz) with a SHA-256 of its bytes and,
+    if the codebook is given, of the codebook's bytes, so that a table is never paired with another codebook."""
+    import hashlib
+    import numpy as np
+    t = nbr_idx.detach().cpu().contiguous().numpy().astype(np.int32)
+    meta = {"table_sha256": hashlib.sha256(t.tobytes()).hexdigest()}
+    if codebook is not None:
+        cb = codebook.detach().cpu().contiguous()
+        meta["codebook_sha256"] = hashlib.sha256(cb.view(torch.uint8).numpy().tobytes()).hexdigest()
+    np.savez(path, nbr_idx=t, **{k: np.array(v) for k, v in meta.items()})
+
+
+def load_neighbors(path: str, codebook: torch.Tensor = None, device="cuda"):
+    """Reads a table written by save_neighbors; raises ValueError if the bytes do not match their checksum or
+    (when a codebook is given and one was recorded) the table belongs to another codebook."""
+    import hashlib
+    import numpy as np
+    with np.load(path) as z:
+        t = np.ascontiguousarray(z["nbr_idx"], dtype=np.int32)
+        if hashlib.sha256(t.tobytes()).hexdigest() != str(z["table_sha256"]):
+            raise ValueError("neighbour table does not match its checksum: " + path)
+        if codebook is not None and "codebook_sha256" in z.files:
+            cb = codebook.detach().cpu().contiguous()
+            if hashlib.sha256(cb.view(torch.uint8).numpy().tobytes()).hexdigest() != str(z["codebook_sha256"]):
+                raise ValueError("neighbour table was built from another codebook: " + path)
+    return torch.from_numpy(t).to(device)
+
+
 def sample_draft_tree(params: Params, tree: Tree, draft_cond, draft_uncond=None, *, tokens=None,
                       parent_begin=0, parent_end=None, gumbel_uniforms=None, draft_prob=None,
                       device_status=None):

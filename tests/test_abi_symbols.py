@@ -42,3 +42,27 @@ def test_host_side_rejections_need_no_gpu():
     assert L.lib.lantern_sample_draft_tree(None, None, None, None, 0, 0, 0, 0, 0, 0, None, None, None, None, None) == 1
     assert L.lib.lantern_verify_tree_workspace(None, 4) == 0
     assert L.set_cluster_size(3) == 0 and L.set_cluster_size(0) == 0        # 3 is refused
+
+
+def test_neighbour_table_file_round_trip_and_checksums(tmp_path):
+    """save_neighbors / load_neighbors (host utilities): bytes come back, a flipped entry or another codebook is refused."""
+    import numpy as np
+    import pytest
+    import torch
+    import paper_2502_06352_b200 as L
+    g = torch.Generator().manual_seed(0)
+    idx = torch.randint(0, 100, (100, 7), generator=g, dtype=torch.int32)
+    cb = torch.randn((100, 4), generator=g)
+    path = str(tmp_path / "table.npz")
+    L.save_neighbors(path, idx, cb)
+    back = L.load_neighbors(path, cb, device="cpu")
+    assert torch.equal(back, idx)
+    with pytest.raises(ValueError):
+        L.load_neighbors(path, cb + 1.0, device="cpu")
+    with np.load(path) as z:
+        d = {k: z[k] for k in z.files}
+    d["nbr_idx"] = d["nbr_idx"].copy()
+    d["nbr_idx"][3, 2] ^= 1
+    np.savez(path, **d)
+    with pytest.raises(ValueError):
+        L.load_neighbors(path, device="cpu")

@@ -134,3 +134,27 @@ def test_tcgen05_and_brute_force_kernels_build_the_same_table(L, n, d, k):
     torch.cuda.synchronize()
     assert torch.equal(i1, i3) and torch.equal(d1, d3)          # run to run
     assert torch.equal(i1, i2) and torch.equal(d1, d2)          # kernel to kernel
+
+
+def test_outputs_stay_inside_their_extent(L):
+    """Guard words before and after the table and the distance array (one allocation each) survive a build
+    by the tcgen05 kernel (ragged last tile) and by the brute-force kernel."""
+    import ctypes
+    from paper_2502_06352_b200.binding import lib, _check
+    for n, d, k, dt in ((8200, 24, 33, torch.bfloat16), (700, 5, 9, torch.float32)):
+        cb = W.make_codebook(n, d, "bf16" if dt == torch.bfloat16 else "f32", seed=3).cuda()
+        pad = 64
+        gi = torch.full((n * k + 2 * pad,), 0x5a5a5a5a, dtype=torch.int32, device="cuda")
+        gd = torch.full((n * k + 2 * pad,), -7.0, dtype=torch.float32, device="cuda")
+        code = 1 if dt == torch.bfloat16 else 0
+        wb = lib.lantern_build_neighbors_workspace(code, n, d, k)
+        ws = torch.empty(max(wb, 256), dtype=torch.uint8, device="cuda")
+        _check(lib.lantern_build_neighbors(ctypes.c_void_p(cb.data_ptr()), code, n, d, k,
+                                           ctypes.c_void_p(gi.data_ptr() + 4 * pad), ctypes.c_void_p(gd.data_ptr() + 4 * pad),
+                                           ctypes.c_void_p(ws.data_ptr()), ws.numel(),
+                                           ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)), "lantern_build_neighbors")
+        torch.cuda.synchronize()
+        assert torch.all(gi[:pad] == 0x5a5a5a5a) and torch.all(gi[-pad:] == 0x5a5a5a5a)
+        assert torch.all(gd[:pad] == -7.0) and torch.all(gd[-pad:] == -7.0)
+        body = gi[pad:-pad].view(n, k)
+        assert int(body.min()) >= 0 and int(body.max()) < n
