@@ -233,19 +233,20 @@ __device__ __forceinline__ double t5_bf16_to_double(uint32_t b16) {
 // st[base + 32 u + lane], u < kT5Chains, each the sum of exact_dist_bf16x8 term by term in the same
 // order.  A double-precision FMA has a long latency and each sum is one dependent chain, so a lane
 // runs the chains of its candidates side by side.  Entries in [n, p2) are padded with +inf.
-constexpr int kT5Chains = 6;
+constexpr int kT5Chains = 7;
 __device__ __forceinline__ void t5_exact_block(const double* qd, const __nv_bfloat16* __restrict__ cb, int d,
-                                               const unsigned long long* st, int n, int p2, int base,
+                                               const unsigned long long* st, int n, int p2, int base, int nch,
                                                unsigned long long* sortd, int* sorti) {
   const int lane = threadIdx.x & 31;
-  const int nu = min(kT5Chains, (min(n, p2) - base + 31) / 32);      // chains with at least one candidate in the warp
+  // this call covers entries [base, base + 32 nch); nu of its chains hold at least one candidate
+  const int nu = min(nch, (min(n, p2) - base + 31) / 32);
   const __nv_bfloat16* row[kT5Chains];
   int idx[kT5Chains];
   double acc[kT5Chains];
 #pragma unroll
   for (int u = 0; u < kT5Chains; ++u) {
     const int i = base + 32 * u + lane;
-    idx[u] = i < n ? static_cast<int>(st[i] & 0xffffffffu) : -1;
+    idx[u] = (u < nch && i < n) ? static_cast<int>(st[i] & 0xffffffffu) : -1;
     row[u] = cb + static_cast<long long>(idx[u] < 0 ? 0 : idx[u]) * d;
     acc[u] = 0.0;
   }
@@ -274,7 +275,7 @@ __device__ __forceinline__ void t5_exact_block(const double* qd, const __nv_bflo
 #pragma unroll
   for (int u = 0; u < kT5Chains; ++u) {
     const int i = base + 32 * u + lane;
-    if (i < p2) {
+    if (u < nch && i < p2) {
       sorti[i] = idx[u] < 0 ? 0x7fffffff : idx[u];
       sortd[i] = idx[u] < 0 ? 0x7ff0000000000000ull : static_cast<unsigned long long>(__double_as_longlong(acc[u]));
     }
@@ -553,7 +554,16 @@ __global__ void __launch_bounds__(kT5Threads, 1) knn_t5_kernel(const KnnT5Args a
         const __nv_bfloat16* q_row = cb + static_cast<long long>(qi) * d;
         for (int t = lane; t < d; t += 32) qd[t] = t5_bf16_to_double(__bfloat16_as_ushort(q_row[t]));
         __syncwarp();
-        for (int base = 0; base < p2; base += 32 * kT5Chains) t5_exact_block(qd, cb, d, st, n, p2, base, sortd, sorti);
+        {
+          // groups of 32 candidates, spread evenly over as few calls as the chains per lane allow
+          const int groups = max((n + 31) / 32, 1), calls = (groups + kT5Chains - 1) / kT5Chains;
+          const int nch = (groups + calls - 1) / calls;
+          for (int c2 = 0; c2 < calls; ++c2) t5_exact_block(qd, cb, d, st, n, p2, c2 * 32 * nch, nch, sortd, sorti);
+          for (int i = calls * 32 * nch + lane; i < p2; i += 32) {       // padding of the sort beyond the calls' range
+            sorti[i] = 0x7fffffff;
+            sortd[i] = 0x7ff0000000000000ull;
+          }
+        }
         __syncwarp();
         t5_warp_sort(sortd, sorti, p2);
         for (int r = lane; r < k; r += 32) {
