@@ -170,3 +170,32 @@ def test_first_child_follows_p_chi_square(L):
     n = counts.sum()
     chi2 = ((counts - n * p) ** 2 / (n * p)).sum()
     assert chi2 < 44.3       # 15 dof, p ~ 1e-4
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+@pytest.mark.parametrize("kw", [dict(vocab=65536, codebook_size=1024, dtype="bf16", cfg_scale=None),
+                                dict(vocab=16384, codebook_size=1024, temperature=0.7),
+                                dict(vocab=5000, codebook_size=1024, n_nodes=26, cfg_scale=None)])
+def test_streaming_kernel_over_seeds_and_row_shapes(L, seed, kw):
+    """The streaming sampler (forced) on rows of the benchmark's width and smaller, several seeds: first
+    threshold from the warps' best keys, the scheduled cut, the exact ranking."""
+    case = Case(small_config(batch=2, **kw), seed=100 + seed, tokens="random", kernels=1)
+    gum = W.make_gumbel_uniforms(case.B, case.N, case.V, 4321 + seed)
+    gtok, gprob, _ = _gpu_sample(L, case, gumbel=gum)
+    assert _compare(case, gum.numpy(), gtok, gprob) <= 1
+
+
+@pytest.mark.parametrize("shape", ["rising", "falling", "flat"])
+def test_streaming_kernel_on_monotone_and_constant_rows(L, shape):
+    """Rows whose logits rise along the row keep producing keys above every earlier threshold (the candidate
+    list overflows and the row is redone with a cut after every chunk); falling rows never do; constant rows
+    leave everything to the uniforms.  All must agree with the oracle."""
+    case = Case(small_config(batch=2, vocab=65536, codebook_size=1024, dtype="f32", cfg_scale=None), seed=77,
+                tokens="random", kernels=1)
+    V = case.V
+    ramp = torch.linspace(-30.0, 30.0, V)
+    row = {"rising": ramp, "falling": ramp.flip(0), "flat": torch.zeros(V)}[shape]
+    case.padded["draft_cond"][:, :, :V] = row
+    gum = W.make_gumbel_uniforms(case.B, case.N, V, 99)
+    gtok, gprob, _ = _gpu_sample(L, case, gumbel=gum)
+    assert _compare(case, gum.numpy(), gtok, gprob) <= 1
