@@ -158,3 +158,18 @@ def test_outputs_stay_inside_their_extent(L):
         assert torch.all(gd[:pad] == -7.0) and torch.all(gd[-pad:] == -7.0)
         body = gi[pad:-pad].view(n, k)
         assert int(body.min()) >= 0 and int(body.max()) < n
+
+
+def test_tcgen05_kernel_on_clustered_rows_with_many_near_ties(L):
+    """64 tight clusters of about 130 rows (noise of a few bf16 steps, so many rows coincide after rounding):
+    inside a cluster the approximate distances are nearly equal, the cut-backs work on keys that differ in their
+    last bits only, and k reaches past the query's own cluster."""
+    g = torch.Generator().manual_seed(12)
+    n, d, k = 8320, 32, 150
+    centres = torch.randn((64, d), generator=g) * 4
+    cb = (centres[torch.arange(n) % 64] + torch.randn((n, d), generator=g) * 0.02).to(torch.bfloat16)
+    rows = [0, 1, 63, 64, 4000, n - 1] + [int(x) for x in np.random.default_rng(3).integers(0, n, 10)]
+    idx, _ = _check(L, cb, k, rows=rows)
+    assert idx.min() >= 0 and idx.max() < n
+    # the first 129 neighbours of a row lie in its own cluster (same index modulo 64)
+    assert np.all(idx[:, :100] % 64 == (np.arange(n) % 64)[:, None])
