@@ -432,7 +432,7 @@ extern "C" size_t lantern_build_neighbors_workspace(lantern_dtype dt, int32_t L,
   // squared norms of all rows and their maximum (tensor-core paths), plus the per-CTA candidate
   // lists of the tcgen05 kernel; the brute-force kernel keeps all of its state on chip
   if (!use_t5_path(dt, L, d, k)) return use_tensor_path(dt, L, d, k) ? norms_bytes(L) : 0;
-  const int nqt = (L + kT5Q - 1) / kT5Q;
+  const int nqt = (L + 63) / 64;                   // the kernel may run tiles of 64 queries (see the launch)
   return norms_bytes(L) + static_cast<size_t>(nqt < kT5GridCap ? nqt : kT5GridCap) * t5_cta_bytes(k);
 }
 
@@ -463,7 +463,10 @@ extern "C" lantern_status lantern_build_neighbors(const void* codebook, lantern_
           cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
         return LANTERN_ERR_CUDA;
       const long long afford = static_cast<long long>((workspace_bytes - norms_bytes(L)) / t5_cta_bytes(k));
-      int grid = (L + kT5Q - 1) / kT5Q;
+      // tiles of 128 queries, or of 64 (half of the tensor-memory lanes idle: the contraction is a small part
+      // of the kernel) when that is what it takes to give every SM a tile
+      fa.qtile = (L + kT5Q - 1) / kT5Q * 2 <= sms ? kT5Q / 2 : kT5Q;
+      int grid = (L + fa.qtile - 1) / fa.qtile;
       if (grid > sms) grid = sms;
       if (grid > afford) grid = static_cast<int>(afford);
       if (grid < 1) return LANTERN_ERR_WORKSPACE;

@@ -45,6 +45,7 @@ struct KnnT5Args {
   const float* nrm;                 // [L] squared norms, nrm[L] = their maximum
   unsigned long long* lists;        // [gridDim.x][kT5Q][CAP] candidate lists (key << 32 | index)
   int L, d, k, CAP;
+  int qtile;                        // queries a CTA tile really holds: 128, or 64 (the other lanes idle) when 128 would leave SMs without a tile
   int32_t* nbr_idx;
   float* nbr_dist;
 };
@@ -109,7 +110,7 @@ __device__ __forceinline__ void t5_arrive(uint32_t mbar) {
 // 8 rows of a chunk are one contiguous core matrix (conflict-free), each row reads 64 contiguous
 // bytes.  A warp walks along the rows of its row groups, so addresses advance by additions only.
 __device__ __forceinline__ void t5_load_tile(const __nv_bfloat16* __restrict__ cb, int L, int d, int row0,
-                                             unsigned char* dst, int ltid) {
+                                             unsigned char* dst, int ltid) {      // L: rows at or beyond it read as zero
   const int lane = ltid & 31, lw = ltid >> 5;
   const int r = lane & 7, c = lane >> 3;                          // row in the group, chunk in the quad
   const int nch = d >> 3, pch = knn_t5_dpad(d) >> 3;               // 16-byte chunks per row: real, padded
@@ -344,7 +345,8 @@ __global__ void __launch_bounds__(kT5Threads, 1) knn_t5_kernel(const KnnT5Args a
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tbase = static_cast<uint32_t>(misc[0]);
 
-  const int nqt = (L + kT5Q - 1) / kT5Q;            // query tiles
+  const int QT = a.qtile;
+  const int nqt = (L + QT - 1) / QT;                // query tiles
   const int nct = (L + kT5C - 1) / kT5C;            // candidate tiles per query tile
   const float nmax = a.nrm[L];
   unsigned long long* my_lists = a.lists + static_cast<size_t>(blockIdx.x) * kT5Q * CAP;
@@ -352,13 +354,13 @@ __global__ void __launch_bounds__(kT5Threads, 1) knn_t5_kernel(const KnnT5Args a
   uint32_t tiles_done = 0, qtiles_done = 0;         // per role: candidate tiles / query tiles handled so far
 
   for (int qt = blockIdx.x; qt < nqt; qt += gridDim.x) {
-    const int q0 = qt * kT5Q;
+    const int q0 = qt * QT;
     if (warp >= 5) {
       // ---------------------------------------------------------------- loaders (warps 5-7)
       const int ltid = tid - 160;
       uint32_t pending;                              // barrier of the copy group committed last
       if (!dead) dead = !t5_wait_warp(aempty, (qtiles_done & 1u) ^ 1u, abort);
-      if (!dead) t5_load_tile(cb, L, d, q0, As, ltid);
+      if (!dead) t5_load_tile(cb, min(L, q0 + QT), d, q0, As, ltid);
       cp_async_commit();
       pending = afull;
       for (int t = 0; t < nct; ++t) {
@@ -418,7 +420,7 @@ __global__ void __launch_bounds__(kT5Threads, 1) knn_t5_kernel(const KnnT5Args a
     } else {
       // ---------------------------------------------------------------- selection (warps 0-3): thread = query
       const int qi = q0 + tid;
-      const bool active = qi < L;
+      const bool active = qi < L && tid < QT;
       const float nq = active ? a.nrm[qi] : 0.f;
       const float e2 = 2.f * static_cast<float>(d + 8) * 4.76837158203125e-7f * (nq + nmax);     // 2 eps, 2^-21
       eps2s[tid] = e2;
@@ -433,7 +435,7 @@ __global__ void __launch_bounds__(kT5Threads, 1) knn_t5_kernel(const KnnT5Args a
       bool ovf = false;
       for (int t = 0; t < nct; ++t) {
         const uint32_t b = tiles_done & 1u;
-        const bool special = t == nct - 1 || t == qt;
+        const bool special = t == nct - 1 || t == q0 / kT5C;
         if (!dead) dead = !t5_wait_warp(tfull(b), (tiles_done >> 1) & 1u, abort);   // warp-uniform
         if (!dead) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -522,7 +524,7 @@ __global__ void __launch_bounds__(kT5Threads, 1) knn_t5_kernel(const KnnT5Args a
       unsigned long long* sortd = reinterpret_cast<unsigned long long*>(hist + 256);   // bit patterns of doubles >= 0
       int* sorti = reinterpret_cast<int*>(sortd + kT5Sort);
       double* qd = reinterpret_cast<double*>(sorti + kT5Sort);
-      for (int q = warp; q < kT5Q; q += kT5Threads / 32) {
+      for (int q = warp; q < QT; q += kT5Threads / 32) {
         const int qi = q0 + q;
         if (qi >= L) break;
         int32_t* out_i = a.nbr_idx + static_cast<long long>(qi) * k;
@@ -578,7 +580,7 @@ __global__ void __launch_bounds__(kT5Threads, 1) knn_t5_kernel(const KnnT5Args a
     if (!dead) {
       double* redd = reinterpret_cast<double*>(bars + 16);
       int* redi = misc + 16;
-      for (int q = 0; q < kT5Q && q0 + q < L; ++q) {
+      for (int q = 0; q < QT && q0 + q < L; ++q) {
         if (cnts[q] != -2) continue;                 // shared value: the same decision in every thread
         const int qi = q0 + q;
         rank_query<__nv_bfloat16>(cb, L, d, k, qi, nullptr, 0, true, 0, nullptr, nullptr, redd, redi,
