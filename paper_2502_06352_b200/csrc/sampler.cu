@@ -503,7 +503,8 @@ extern "C" lantern_status lantern_sample_draft_tree(
   const bool fits_dense = sampler_shape(V, batch * (i1 - i0), dt == LANTERN_F32 ? 4 : 8, ov, &cs_d, &e_d, &smem_d);
   if (p->kernels < 0 || p->kernels > 2) return LANTERN_ERR_INVALID_ARG;
   if (sampler_uses_stream(p, static_cast<long long>(batch) * (i1 - i0), fits_dense)) {
-    // CTAs per parent: one when the parents alone fill the machine
+    // CTAs per parent: the smallest power of two that gives every SM a CTA (measured on rows of 65536 logits:
+    // 80 and 100 parents run fastest split in two, 200 unsplit; wider clusters pay for their merge)
     int cs = ov;
     if (cs <= 0) {
       int dev = 0, sms = 0;
@@ -512,7 +513,7 @@ extern "C" lantern_status lantern_sample_draft_tree(
         sms = 148;
       const int nvec = (allow_hi - allow_lo) / (dt == LANTERN_F32 ? 4 : 8);
       cs = 1;
-      while (cs < 16 && static_cast<long long>(batch) * (i1 - i0) * cs < 4 * sms && nvec / (2 * cs * stream::SW) >= 32) cs *= 2;
+      while (cs < 16 && static_cast<long long>(batch) * (i1 - i0) * cs < sms && nvec / (2 * cs * stream::SW) >= 32) cs *= 2;
     }
     return launch_sample_stream(a, cs, dt == LANTERN_F32, cfg, st) == cudaSuccess ? LANTERN_OK : LANTERN_ERR_CUDA;
   }
