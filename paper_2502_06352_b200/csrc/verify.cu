@@ -90,12 +90,13 @@ static cudaError_t launch_stream_any(const VerifyArgs& a, int cs, size_t smem, b
               : launch_stream_t<__nv_bfloat16, false, false>(a, cs, smem, st);
 }
 // CTAs per node: one when the nodes alone fill the machine, else the smallest power of two that
-// does, as long as every warp keeps at least one full 512-byte step of the row
+// does, as long as every warp of the wider cluster keeps at least two full 512-byte steps of the row
+// (narrow rows, e.g. an allowed range of 8192 tokens, run faster on fewer, busier CTAs)
 static int stream_cluster_size(int nodes, int V, bool f32) {
   if (g_cluster_override > 0) return g_cluster_override;
   const int nvec = V / (f32 ? 4 : 8);
   int cs = 1;
-  while (cs < 16 && static_cast<long long>(nodes) * cs < 8 * sm_count() && nvec / (2 * cs * stream::SW) >= 32) cs *= 2;
+  while (cs < 16 && static_cast<long long>(nodes) * cs < 8 * sm_count() && nvec / (4 * cs * stream::SW) >= 32) cs *= 2;
   return cs;
 }
 
